@@ -1,0 +1,162 @@
+/*
+ * sol_attn3d -- 3D-RoPE joint self-attention of a video DiT block on NVIDIA B200 (sm_100a).
+ *
+ * The operation (per sequence, per head):
+ *
+ *     q~_i = RoPE3D(q_i, pos_i),  k~_j = RoPE3D(k_j, pos_j)        (video tokens only)
+ *     out_i = sum_j softmax_j( <q~_i, k~_j> / sqrt(head_dim) ) v_j   over valid keys j
+ *
+ * This is the dense attention ("SDPA") that Section 3.2 of the paper ("Optimized attention
+ * collectives") reports as the dominant cost of a denoising step, combined with the rotary
+ * embedding of fusion group (2) in Section 3.5 ("QK normalization with partial RoPE"), on the
+ * prefix-first packed token order of Section 3.4 ("Safety rails and the exact prefix KV sink")
+ * and the flat (total, heads, head_dim) activation layout of Section 3.2.
+ *
+ * Conventions (the paper prints no formula; these are the definitions this library implements):
+ *   - a sequence is text_len prefix tokens followed by T*H*W video tokens, t slowest, w fastest;
+ *   - prefix tokens carry no rotary embedding; V is never rotated;
+ *   - rope_dims = {d_T, d_H, d_W}: head dims [0,d_T) rotate with t, [d_T,d_T+d_H) with h, the next
+ *     d_W with w; dims beyond d_T+d_H+d_W pass through ("partial" RoPE).  Inside an axis of width
+ *     d_a the ADJACENT pair (2j, 2j+1) rotates by pos_a * theta^(-2j/d_a), counter-clockwise;
+ *   - non-causal; the only masks are the key-padding mask and the block-diagonal structure of a
+ *     packed batch (a query attends to the keys of its own sequence only);
+ *   - a query row whose sequence has no valid key returns zeros.
+ *
+ * All tensors are bf16.  Math: rotation in fp32 from fp64-built tables, QK^T and PV on tcgen05
+ * tensor cores (bf16 operands, fp32 accumulation in tensor memory), softmax in fp32.
+ *
+ * Every function returns 0 on success or a negative sol_attn3d_error.  No function throws, aborts
+ * or synchronises the device unless stated.  There is no CPU fallback: without a B200 the device
+ * calls fail with SOL_ATTN3D_ERR_NO_DEVICE / SOL_ATTN3D_ERR_UNSUPPORTED_ARCH.
+ */
+#ifndef SOL_ATTN3D_H_
+#define SOL_ATTN3D_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sol_attn3d_plan_s* sol_attn3d_plan_t;
+/* A cudaStream_t, passed as an opaque pointer so this header needs no CUDA include. */
+typedef void* sol_attn3d_stream_t;
+
+typedef enum {
+  SOL_ATTN3D_OK = 0,
+  SOL_ATTN3D_ERR_INVALID_ARG = -1,      /* NULL where a pointer is required, non-positive size, odd rope dim ... */
+  SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE = -2,/* head_dim not 64/128, strides not 16-byte multiples, size overflow */
+  SOL_ATTN3D_ERR_NO_WORKSPACE = -3,     /* forward before set_workspace, or workspace too small / misaligned */
+  SOL_ATTN3D_ERR_NO_DEVICE = -4,        /* no CUDA device / driver */
+  SOL_ATTN3D_ERR_UNSUPPORTED_ARCH = -5, /* current device is not compute capability 10.x */
+  SOL_ATTN3D_ERR_CUDA = -6,             /* a CUDA call failed; sol_attn3d_last_cuda_error() has the code */
+  SOL_ATTN3D_ERR_DEVICE_TIMEOUT = -7,   /* a bounded wait inside a kernel ran out (status word) */
+  SOL_ATTN3D_ERR_NO_MEMORY = -8         /* host allocation failed */
+} sol_attn3d_error;
+
+/*
+ * Extended problem description (packed / ragged batches, strided tensors).
+ *   size       sizeof(sol_attn3d_desc), for versioning.
+ *   n_seqs     number of packed sequences (>= 1).
+ *   grids      n_seqs x 3 ints {T, H, W}, each >= 1 ... or T*H*W may be 0 only via T=0 (prefix-only sequence).
+ *   text_lens  n_seqs prefix lengths (>= 0).  Sequence s holds text_lens[s] + T*H*W tokens and starts
+ *              where sequence s-1 ends (cu_seqlens is derived; see sol_attn3d_cu_seqlens).
+ *   theta      rotary base (> 1); the benchmark configurations use 10000.
+ *   *_strides  element strides {token, head} of q, k, v, out; {0,0} means contiguous
+ *              {heads*head_dim, head_dim}.  head_dim is always contiguous.  Strides let Q, K and V be
+ *              views into one packed QKV buffer (Section 3.2).  Byte strides must be multiples of 16.
+ */
+typedef struct {
+  uint32_t size;
+  int32_t n_seqs;
+  const int32_t* grids;
+  const int32_t* text_lens;
+  int32_t heads;
+  int32_t head_dim;
+  int32_t rope_dims[3];
+  double theta;
+  int64_t q_strides[2];
+  int64_t k_strides[2];
+  int64_t v_strides[2];
+  int64_t out_strides[2];
+} sol_attn3d_desc;
+
+/*
+ * Plan for B equal sequences (Section 3.2's attention over [prefix | T*H*W video tokens]).
+ * Host-only: validates, derives the token layout, the tile schedule and the fp64-computed cos/sin
+ * tables.  Allocates no device memory.  theta = 10000.  Tensors are [B, N, heads, head_dim] with
+ * N = text_len + T*H*W, contiguous.  *plan is written only on success; free with sol_attn3d_destroy.
+ */
+int sol_attn3d_plan(sol_attn3d_plan_t* plan, int B, int heads, int head_dim, int T, int H, int W,
+                    int text_len, const int rope_dims[3]);
+
+/* Same for a packed ragged batch and/or strided tensors ([total_tokens, heads, head_dim]). */
+int sol_attn3d_plan_ex(sol_attn3d_plan_t* plan, const sol_attn3d_desc* desc);
+
+/* Derived token offsets: *cu points at n_seqs+1 int64 values owned by the plan (host memory). */
+int sol_attn3d_cu_seqlens(sol_attn3d_plan_t plan, const int64_t** cu, int* n_seqs);
+
+/*
+ * Device scratch the caller must provide (the library never allocates device memory).  Holds the
+ * rotated Q and K (the rotary prologue writes them once per forward), the rotary tables, the
+ * per-128-key-tile validity bits and a status word.
+ */
+size_t sol_attn3d_workspace_bytes(sol_attn3d_plan_t plan);
+
+/*
+ * Binds caller-owned device memory (256-byte aligned, >= workspace_bytes) to the plan and uploads
+ * the plan's tables into it on the current device (synchronous copy; checks that the device is
+ * compute capability 10.x).  The workspace must stay alive and untouched until the plan is
+ * destroyed or rebound.  One plan supports one forward in flight at a time.
+ */
+int sol_attn3d_set_workspace(sol_attn3d_plan_t plan, void* device_ptr, size_t bytes);
+
+/*
+ * out = attention(q, k, v) as defined at the top of this file.  Steps, all enqueued on `stream`
+ * without host synchronisation: key-validity bits per 128-key tile (Section 3.2 layout; only when
+ * the mask may have changed), rotary prologue on Q and K (Section 3.5 group (2)), attention main
+ * kernel (Section 3.2 "SDPA").
+ *
+ *   q, k, v, out  DEVICE pointers, bf16, [total_tokens, heads, head_dim] with the plan's strides,
+ *                 16-byte aligned; q and k are UN-rotated.  out must not alias q, k or v.
+ *   key_mask      DEVICE pointer, uint8 [total_tokens] (i.e. [B, N]), nonzero = attend; applies to
+ *                 keys only, broadcast over heads and queries; NULL = all keys valid.
+ *   K and V values at masked positions must be finite (0 * inf inside the tensor core is NaN).
+ * Errors: INVALID_ARG (NULL / misaligned pointer), NO_WORKSPACE, CUDA.  Device-side time-outs are
+ * reported by sol_attn3d_status after the caller has synchronised the stream.
+ */
+int sol_attn3d_forward(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out,
+                       const uint8_t* key_mask, sol_attn3d_stream_t stream);
+
+/*
+ * The rotary prologue alone (Section 3.5 group (2), rotation part): q_rot / k_rot receive the rotated
+ * bf16 tensors, contiguous [total_tokens, heads, head_dim].  DEVICE pointers, 16-byte aligned; either
+ * input may be NULL together with its output.  Needs a bound workspace (tables).  Asynchronous.
+ */
+int sol_attn3d_rope_qk(sol_attn3d_plan_t plan, const void* q, const void* k, void* q_rot, void* k_rot,
+                       sol_attn3d_stream_t stream);
+
+/*
+ * Reads the device status word (synchronous 4-byte copy; call after synchronising the stream).
+ * 0 = no fault; SOL_ATTN3D_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up, in which
+ * case `out` is undefined.  The word is cleared by the next sol_attn3d_set_workspace.
+ */
+int sol_attn3d_status(sol_attn3d_plan_t plan);
+
+/* Number of kernels one sol_attn3d_forward with / without a key mask enqueues (for launch accounting). */
+int sol_attn3d_launches_per_forward(sol_attn3d_plan_t plan, int with_mask);
+
+/* cudaError_t of the last failing CUDA call made on behalf of this plan (0 if none). */
+int sol_attn3d_last_cuda_error(sol_attn3d_plan_t plan);
+
+/* Static string for an error code. */
+const char* sol_attn3d_strerror(int code);
+
+/* Frees host state.  Never frees caller memory.  NULL is a no-op.  Does not synchronise. */
+int sol_attn3d_destroy(sol_attn3d_plan_t plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOL_ATTN3D_H_ */

@@ -1,0 +1,246 @@
+"""ctypes binding of the C-ABI library, one Python function per exported call.
+
+Argument marshalling only: every step of the attention path runs in the CUDA
+kernels behind ``libsol_attn3d.so``.  PyTorch appears here only as the owner
+of device memory and streams.  There is no CPU fallback: loading fails loudly
+if the library has not been built, and device calls fail on a machine without
+a B200.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.environ.get("SOL_ATTN3D_LIB") or os.path.join(_HERE, "libsol_attn3d.so")
+
+
+class SolAttn3dError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = _lib().sol_attn3d_strerror(code).decode() if _LIB is not None else "?"
+        super().__init__(f"{where}: {msg} (code {code})")
+
+
+class sol_attn3d_desc(ctypes.Structure):
+    _fields_ = [
+        ("size", ctypes.c_uint32),
+        ("n_seqs", ctypes.c_int32),
+        ("grids", ctypes.POINTER(ctypes.c_int32)),
+        ("text_lens", ctypes.POINTER(ctypes.c_int32)),
+        ("heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32),
+        ("rope_dims", ctypes.c_int32 * 3),
+        ("theta", ctypes.c_double),
+        ("q_strides", ctypes.c_int64 * 2),
+        ("k_strides", ctypes.c_int64 * 2),
+        ("v_strides", ctypes.c_int64 * 2),
+        ("out_strides", ctypes.c_int64 * 2),
+    ]
+
+
+# error codes (mirror include/sol_attn3d.h)
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED_SHAPE = -2
+ERR_NO_WORKSPACE = -3
+ERR_NO_DEVICE = -4
+ERR_UNSUPPORTED_ARCH = -5
+ERR_CUDA = -6
+ERR_DEVICE_TIMEOUT = -7
+ERR_NO_MEMORY = -8
+
+_LIB = None
+
+
+def _lib():
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2609_35110_b200.build` "
+            "(there is no CPU fallback for the attention path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+    lib.sol_attn3d_plan.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
+    lib.sol_attn3d_plan.restype = i32
+    lib.sol_attn3d_plan_ex.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(sol_attn3d_desc)]
+    lib.sol_attn3d_plan_ex.restype = i32
+    lib.sol_attn3d_cu_seqlens.argtypes = [vp, ctypes.POINTER(ctypes.POINTER(i64)), ctypes.POINTER(i32)]
+    lib.sol_attn3d_cu_seqlens.restype = i32
+    lib.sol_attn3d_workspace_bytes.argtypes = [vp]
+    lib.sol_attn3d_workspace_bytes.restype = ctypes.c_size_t
+    lib.sol_attn3d_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    lib.sol_attn3d_set_workspace.restype = i32
+    lib.sol_attn3d_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.sol_attn3d_forward.restype = i32
+    lib.sol_attn3d_rope_qk.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.sol_attn3d_rope_qk.restype = i32
+    lib.sol_attn3d_status.argtypes = [vp]
+    lib.sol_attn3d_status.restype = i32
+    lib.sol_attn3d_launches_per_forward.argtypes = [vp, i32]
+    lib.sol_attn3d_launches_per_forward.restype = i32
+    lib.sol_attn3d_last_cuda_error.argtypes = [vp]
+    lib.sol_attn3d_last_cuda_error.restype = i32
+    lib.sol_attn3d_strerror.argtypes = [i32]
+    lib.sol_attn3d_strerror.restype = ctypes.c_char_p
+    lib.sol_attn3d_destroy.argtypes = [vp]
+    lib.sol_attn3d_destroy.restype = i32
+    _LIB = lib
+    return lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise SolAttn3dError(code, where)
+
+
+# ----------------------------------------------------------------- 1:1 wrappers
+def sol_attn3d_plan(B: int, heads: int, head_dim: int, T: int, H: int, W: int, text_len: int,
+                    rope_dims: Sequence[int]) -> ctypes.c_void_p:
+    h = ctypes.c_void_p()
+    rd = (ctypes.c_int * 3)(*[int(x) for x in rope_dims])
+    _check(_lib().sol_attn3d_plan(ctypes.byref(h), B, heads, head_dim, T, H, W, text_len, rd), "sol_attn3d_plan")
+    return h
+
+
+def sol_attn3d_plan_ex(seqs: Sequence[Tuple[int, int, int, int]], heads: int, head_dim: int,
+                       rope_dims: Sequence[int], theta: float = 10000.0,
+                       q_strides=(0, 0), k_strides=(0, 0), v_strides=(0, 0), out_strides=(0, 0)) -> ctypes.c_void_p:
+    """seqs: [(text_len, T, H, W), ...]; strides are (token, head) element strides, 0 = contiguous."""
+    n = len(seqs)
+    grids = (ctypes.c_int32 * (3 * max(n, 1)))()
+    lens = (ctypes.c_int32 * max(n, 1))()
+    for i, (L, T, H, W) in enumerate(seqs):
+        grids[3 * i], grids[3 * i + 1], grids[3 * i + 2] = T, H, W
+        lens[i] = L
+    d = sol_attn3d_desc()
+    d.size = ctypes.sizeof(sol_attn3d_desc)
+    d.n_seqs = n
+    d.grids = ctypes.cast(grids, ctypes.POINTER(ctypes.c_int32))
+    d.text_lens = ctypes.cast(lens, ctypes.POINTER(ctypes.c_int32))
+    d.heads, d.head_dim = heads, head_dim
+    for a in range(3):
+        d.rope_dims[a] = int(rope_dims[a])
+    d.theta = float(theta)
+    for name, val in (("q_strides", q_strides), ("k_strides", k_strides), ("v_strides", v_strides),
+                      ("out_strides", out_strides)):
+        arr = getattr(d, name)
+        arr[0], arr[1] = int(val[0]), int(val[1])
+    h = ctypes.c_void_p()
+    _check(_lib().sol_attn3d_plan_ex(ctypes.byref(h), ctypes.byref(d)), "sol_attn3d_plan_ex")
+    return h
+
+
+def sol_attn3d_cu_seqlens(plan) -> list:
+    p = ctypes.POINTER(ctypes.c_int64)()
+    n = ctypes.c_int()
+    _check(_lib().sol_attn3d_cu_seqlens(plan, ctypes.byref(p), ctypes.byref(n)), "sol_attn3d_cu_seqlens")
+    return [int(p[i]) for i in range(n.value + 1)]
+
+
+def sol_attn3d_workspace_bytes(plan) -> int:
+    return int(_lib().sol_attn3d_workspace_bytes(plan))
+
+
+def sol_attn3d_set_workspace(plan, workspace: torch.Tensor) -> None:
+    _check(_lib().sol_attn3d_set_workspace(plan, workspace.data_ptr(), workspace.numel() * workspace.element_size()),
+           "sol_attn3d_set_workspace")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def sol_attn3d_forward(plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                       key_mask: Optional[torch.Tensor] = None, stream=None) -> None:
+    for t in (q, k, v, out):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v, out must be CUDA bf16 tensors")
+    if key_mask is not None and (not key_mask.is_cuda or key_mask.dtype != torch.uint8 or not key_mask.is_contiguous()):
+        raise ValueError("key_mask must be a contiguous CUDA uint8 tensor")
+    _check(_lib().sol_attn3d_forward(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask), _stream(stream)),
+           "sol_attn3d_forward")
+
+
+def sol_attn3d_rope_qk(plan, q, k, q_rot, k_rot, stream=None) -> None:
+    _check(_lib().sol_attn3d_rope_qk(plan, _ptr(q), _ptr(k), _ptr(q_rot), _ptr(k_rot), _stream(stream)),
+           "sol_attn3d_rope_qk")
+
+
+def sol_attn3d_status(plan) -> int:
+    return int(_lib().sol_attn3d_status(plan))
+
+
+def sol_attn3d_launches_per_forward(plan, with_mask: bool) -> int:
+    return int(_lib().sol_attn3d_launches_per_forward(plan, 1 if with_mask else 0))
+
+
+def sol_attn3d_last_cuda_error(plan) -> int:
+    return int(_lib().sol_attn3d_last_cuda_error(plan))
+
+
+def sol_attn3d_strerror(code: int) -> str:
+    return _lib().sol_attn3d_strerror(code).decode()
+
+
+def sol_attn3d_destroy(plan) -> None:
+    _check(_lib().sol_attn3d_destroy(plan), "sol_attn3d_destroy")
+
+
+# ----------------------------------------------------------------- convenience holder
+class Attn3d:
+    """Owns a plan and its torch-allocated workspace.  ``forward`` = one DiT-block attention."""
+
+    def __init__(self, seqs, heads, head_dim, rope_dims, theta=10000.0, device="cuda", **strides):
+        self.seqs = [tuple(int(x) for x in s) for s in seqs]
+        self.heads, self.head_dim = heads, head_dim
+        self.plan = sol_attn3d_plan_ex(self.seqs, heads, head_dim, rope_dims, theta, **strides)
+        self.cu_seqlens = sol_attn3d_cu_seqlens(self.plan)
+        self.total_tokens = self.cu_seqlens[-1]
+        self.workspace = None
+        if device is not None:
+            nbytes = sol_attn3d_workspace_bytes(self.plan)
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+            assert self.workspace.data_ptr() % 256 == 0
+            sol_attn3d_set_workspace(self.plan, self.workspace)
+
+    @classmethod
+    def from_workload(cls, w, device="cuda"):
+        return cls([(s.text_len, s.T, s.H, s.W) for s in w.seqs], w.heads, w.head_dim, w.rope_dims, w.theta, device)
+
+    def forward(self, q, k, v, key_mask=None, out=None, stream=None):
+        if out is None:
+            out = torch.empty((self.total_tokens, self.heads, self.head_dim), dtype=torch.bfloat16, device=q.device)
+        sol_attn3d_forward(self.plan, q, k, v, out, key_mask, stream)
+        return out
+
+    def rope_qk(self, q, k, stream=None):
+        q_rot = torch.empty((self.total_tokens, self.heads, self.head_dim), dtype=torch.bfloat16, device=q.device)
+        k_rot = torch.empty_like(q_rot)
+        sol_attn3d_rope_qk(self.plan, q, k, q_rot, k_rot, stream)
+        return q_rot, k_rot
+
+    def status(self) -> int:
+        return sol_attn3d_status(self.plan)
+
+    def close(self):
+        if self.plan is not None:
+            sol_attn3d_destroy(self.plan)
+            self.plan = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,368 @@
+// Attention main kernel for sm_100a: S = Q~ K~^T and O += P V on tcgen05 tensor cores with the
+// accumulators in tensor memory, TMA-fed shared-memory ring, online softmax in registers.
+//
+// One CTA = one (sequence, head, pair of 128-row query tiles).  Warp roles:
+//   warps 0-3   softmax / correction / epilogue of query tile 0 (thread = one query row)
+//   warps 4-7   the same for query tile 1
+//   warp  8     TMA producer (one elected lane)
+//   warp  9     tcgen05.mma issuer (one elected lane), owns the TMEM allocation
+//   warps 10-11 idle (complete the third warpgroup)
+// The two query tiles ping-pong: while the softmax of one tile runs on the ALUs, the tensor core
+// works on the other tile's QK^T / PV.
+//
+// Tensor memory (512 columns x 128 lanes x 32 bit):
+//   [0,128)    S0  (fp32 scores of tile 0);  P0 (bf16, 64 columns) overwrites its first half
+//   [128,256)  S1 / P1
+//   [256,256+D)       O0 (fp32)
+//   [256+D,256+2D)    O1
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "device_types.cuh"
+#include "ptx_sm100.cuh"
+
+namespace sol {
+
+constexpr int kAttnThreads = 384;
+
+template <int D>
+struct AttnSmem {
+  static constexpr int kTile = 128 * D * 2;               // bytes of one 128 x D bf16 tile
+  static constexpr int kHalves = D / 64;                  // 64-column (128-byte) swizzle boxes per row
+  static constexpr int kHalfBytes = 128 * 128;            // one box: 128 rows x 128 bytes
+  static constexpr int kStages = (D == 128) ? 5 : 10;     // K/V ring (K and V tiles alternate)
+  static constexpr int kOffQ = 0;
+  static constexpr int kOffKV = 2 * kTile;
+  static constexpr int kOffBars = kOffKV + kStages * kTile;
+  static constexpr int kNumBars = 1 + 2 * kStages + 7;  // q_full, kv_full/empty, s_full, p_full, o_done, drain
+  static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
+  static constexpr int kBytes = kOffTmemPtr + 16;
+  static constexpr int kDynBytes = kBytes + 1024;         // slack to align the base to 1024 bytes
+};
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+  using L = AttnSmem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t sbase = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (sbase - raw_addr);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  const uint32_t sQ = sbase + L::kOffQ;
+  const uint32_t sKV = sbase + L::kOffKV;
+  const uint32_t bars = sbase + L::kOffBars;
+  const uint32_t bar_q_full = bars;
+  auto bar_kv_full = [&](int s) { return bars + 8u * (1 + s); };
+  auto bar_kv_empty = [&](int s) { return bars + 8u * (1 + L::kStages + s); };
+  auto bar_s_full = [&](int t) { return bars + 8u * (1 + 2 * L::kStages + t); };
+  auto bar_p_full = [&](int t) { return bars + 8u * (3 + 2 * L::kStages + t); };
+  auto bar_o_done = [&](int t) { return bars + 8u * (5 + 2 * L::kStages + t); };
+  const uint32_t bar_drain = bars + 8u * (7 + 2 * L::kStages);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + L::kOffTmemPtr);
+
+  // A fault recorded by an earlier CTA stops later ones at the door (read once, CTA-uniform).
+  if (threadIdx.x == 0) tmem_ptr_smem[1] = *reinterpret_cast<volatile unsigned int*>(p.status);
+  __syncthreads();
+  if (tmem_ptr_smem[1] != 0) return;
+
+  // ---- which work item
+  int si = 0;
+  while (si + 1 < p.n_seqs && (int)blockIdx.x >= p.seqs[si + 1].work_start) ++si;
+  const SeqDev sq = p.seqs[si];
+  const int local = (int)blockIdx.x - sq.work_start;
+  const int head = local / sq.n_qpairs;
+  const int pair = local - head * sq.n_qpairs;
+  const int n_proc = p.ktile_count[si];
+  const int* __restrict__ ktiles = p.ktile_list + sq.ktile_start;
+  const uint4* __restrict__ keybits = p.keybits + sq.ktile_start;
+  const int q_row0 = pair * 256;                       // first local query row of the CTA
+  const int tok0 = (int)sq.tok_start;                  // TMA token coordinate of the sequence start
+  const unsigned long long limit = p.wait_limit_ns;
+
+  if (warp == 8 && lane == 0) {
+    mbar_init(bar_q_full, 1);
+    for (int s = 0; s < L::kStages; ++s) {
+      mbar_init(bar_kv_full(s), 1);
+      mbar_init(bar_kv_empty(s), 1);
+    }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(bar_s_full(t), 1);
+      mbar_init(bar_p_full(t), 128);
+      mbar_init(bar_o_done(t), 1);
+    }
+    mbar_init(bar_drain, 1);
+    fence_mbar_init();
+    prefetch_tensormap(&tm_q);
+    prefetch_tensormap(&tm_k);
+    prefetch_tensormap(&tm_v);
+  }
+  if (warp == 9) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_ptr_smem[0];
+
+  if (warp < 8) {
+    // =========================================================== softmax / correction / epilogue
+    const int t = warp >> 2;
+    const int wq = warp & 3;
+    const int row = wq * 32 + lane;
+    const uint32_t lane_off = static_cast<uint32_t>(wq * 32) << 16;
+    const uint32_t tS = tmem_base + lane_off + t * 128;
+    const uint32_t tO = tmem_base + lane_off + 256 + t * D;
+    const float c = p.scale_log2;
+    float m_ref = -CUDART_INF_F;
+    float l = 0.f;
+    bool ok = true;
+
+    for (int i = 0; i < n_proc; ++i) {
+      const int jt = __ldg(&ktiles[i]);
+      const uint4 kb = __ldg(&keybits[jt]);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full(t), i & 1, limit));
+      if (!ok) break;
+      tc_fence_after();
+
+      uint32_t r[128];
+#pragma unroll
+      for (int cch = 0; cch < 4; ++cch) tmem_ld32(tS + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[cch * 32]));
+      tmem_wait_ld();
+
+      if (p.dbg_scores != nullptr && i == 0) {
+        float* dst = p.dbg_scores + ((size_t)blockIdx.x * 2 + t) * 128 * 128 + (size_t)row * 128;
+#pragma unroll
+        for (int cc = 0; cc < 128; ++cc) dst[cc] = __uint_as_float(r[cc]);
+      }
+
+      if ((kb.x & kb.y & kb.z & kb.w) != 0xffffffffu) {
+        // mixed tile: masked or out-of-range keys get -inf
+#pragma unroll
+        for (int cc = 0; cc < 128; ++cc) {
+          const uint32_t w = cc < 32 ? kb.x : cc < 64 ? kb.y : cc < 96 ? kb.z : kb.w;
+          if (((w >> (cc & 31)) & 1u) == 0) r[cc] = __float_as_uint(-CUDART_INF_F);
+        }
+      }
+
+      float mx0 = __uint_as_float(r[0]), mx1 = __uint_as_float(r[1]);
+      float mx2 = __uint_as_float(r[2]), mx3 = __uint_as_float(r[3]);
+#pragma unroll
+      for (int cc = 4; cc < 128; cc += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(r[cc]));
+        mx1 = fmaxf(mx1, __uint_as_float(r[cc + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(r[cc + 2]));
+        mx3 = fmaxf(mx3, __uint_as_float(r[cc + 3]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+
+      // Lazy rescale: the reference maximum only moves when the row maximum has grown by more than
+      // 2^8 in the exp2 domain, so stale-reference terms stay <= 256 and O is rarely touched.
+      if (i == 0) {
+        m_ref = mx;
+      } else {
+        const bool grow = (mx - m_ref) * c > 8.0f;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
+          if (grow) m_ref = mx;
+          l *= f;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (i - 1) & 1, limit));
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int cch = 0; cch < D / 32; ++cch) {
+            uint32_t o[32];
+            tmem_ld32(tO + cch * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
+            tmem_st32(tO + cch * 32, o);
+          }
+        }
+      }
+
+      const float mc = m_ref * c;
+      float sum0 = 0.f, sum1 = 0.f;
+      uint32_t pk[64];
+#pragma unroll
+      for (int cc = 0; cc < 64; ++cc) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(r[2 * cc]), c, -mc));
+        const float p1 = ex2_approx(fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc));
+        sum0 += p0;
+        sum1 += p1;
+        pk[cc] = pack_bf16x2(p0, p1);
+      }
+      l += sum0 + sum1;
+      tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p_full(t));
+    }
+
+    // ---- epilogue: O / l -> bf16 -> global (rows beyond the sequence are not stored)
+    if (ok && n_proc > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (n_proc - 1) & 1, limit));
+      if (ok) tc_fence_after();
+    }
+    if (ok) {
+      const int qrow = q_row0 + t * 128 + row;
+      const bool store = qrow < sq.n_tokens;
+      const float inv = (n_proc > 0) ? 1.0f / l : 0.f;
+      __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
+                           (sq.tok_start + qrow) * p.o_tok_stride + (long long)head * p.o_head_stride;
+#pragma unroll
+      for (int cch = 0; cch < D / 32; ++cch) {
+        uint32_t o[32];
+        if (n_proc > 0) {
+          tmem_ld32(tO + cch * 32, o);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int cc = 0; cc < 32; ++cc) o[cc] = 0u;
+        }
+        if (store) {
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(o[8 * v4 + 0]) * inv, __uint_as_float(o[8 * v4 + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(o[8 * v4 + 2]) * inv, __uint_as_float(o[8 * v4 + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(o[8 * v4 + 4]) * inv, __uint_as_float(o[8 * v4 + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(o[8 * v4 + 6]) * inv, __uint_as_float(o[8 * v4 + 7]) * inv);
+            *reinterpret_cast<uint4*>(dst + cch * 32 + v4 * 8) = w;
+          }
+        }
+      }
+    } else if (lane == 0) {
+      atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);
+    }
+  } else if (warp == 8) {
+    // =========================================================== TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      mbar_arrive_expect_tx(bar_q_full, 2 * L::kTile);
+#pragma unroll
+      for (int t = 0; t < 2; ++t)
+#pragma unroll
+        for (int hf = 0; hf < L::kHalves; ++hf)
+          tma_load_3d(sQ + t * L::kTile + hf * L::kHalfBytes, &tm_q, bar_q_full, hf * 64, head,
+                      tok0 + q_row0 + t * 128);
+      uint32_t it = 0;
+      for (int i = 0; i < n_proc && ok; ++i) {
+        const int jt = __ldg(&ktiles[i]);
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+          const uint32_t stage = it % L::kStages;
+          const uint32_t par = (it / L::kStages) & 1u;
+          if (!mbar_wait(bar_kv_empty(stage), par ^ 1u, limit)) { ok = false; break; }
+          mbar_arrive_expect_tx(bar_kv_full(stage), L::kTile);
+          const CUtensorMap* tm = kv ? &tm_v : &tm_k;
+#pragma unroll
+          for (int hf = 0; hf < L::kHalves; ++hf)
+            tma_load_3d(sKV + stage * L::kTile + hf * L::kHalfBytes, tm, bar_kv_full(stage), hf * 64, head,
+                        tok0 + jt * 128);
+          ++it;
+        }
+      }
+      if (!ok) {
+        atomicCAS(p.status, 0u, kStatusTimeoutProducer);
+        // let the copies already in flight land before the CTA gives its shared memory back
+        mbar_wait(bar_q_full, 0, limit);
+        const uint32_t first = it > (uint32_t)L::kStages ? it - L::kStages : 0u;
+        for (uint32_t j = first; j < it; ++j) mbar_wait(bar_kv_full(j % L::kStages), (j / L::kStages) & 1u, limit);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 9) {
+    // =========================================================== MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, true);
+      bool ok = true;
+      const uint32_t v_lbo = p.v_lbo, v_sbo = p.v_sbo;
+      auto issue_qk = [&](int t, uint32_t kaddr) {
+        const uint32_t qaddr = sQ + t * L::kTile;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t off = (k >> 2) * L::kHalfBytes + (k & 3) * 32;
+          mma_ss(tmem_base + t * 128, smem_desc_sw128(qaddr + off, 16, 1024), smem_desc_sw128(kaddr + off, 16, 1024),
+                 idesc_qk, k > 0 ? 1u : 0u);
+        }
+      };
+      auto issue_pv = [&](int t, uint32_t vaddr, bool acc) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          mma_ts(tmem_base + 256 + t * D, tmem_base + t * 128 + k * 8, smem_desc_sw128(vaddr + k * 2048, v_lbo, v_sbo),
+                 idesc_pv, (acc || k > 0) ? 1u : 0u);
+        }
+      };
+      auto stage_addr = [&](uint32_t it) { return sKV + (it % L::kStages) * L::kTile; };
+      auto wait_full = [&](uint32_t it) {
+        return mbar_wait(bar_kv_full(it % L::kStages), (it / L::kStages) & 1u, limit);
+      };
+
+      if (n_proc > 0) {
+        uint32_t it = 0;
+        ok = mbar_wait(bar_q_full, 0, limit) && wait_full(it);
+        if (ok) {
+          tc_fence_after();
+          issue_qk(0, stage_addr(it));
+          tc_commit(bar_s_full(0));
+          issue_qk(1, stage_addr(it));
+          tc_commit(bar_s_full(1));
+          tc_commit(bar_kv_empty(it % L::kStages));
+          ++it;
+        }
+        for (int i = 0; i < n_proc && ok; ++i) {
+          const uint32_t it_v = it++;
+          const bool more = i + 1 < n_proc;
+          const uint32_t it_k = more ? it++ : 0;
+          if (!(wait_full(it_v) && mbar_wait(bar_p_full(0), i & 1, limit))) { ok = false; break; }
+          tc_fence_after();
+          issue_pv(0, stage_addr(it_v), i > 0);
+          tc_commit(bar_o_done(0));
+          if (more) {
+            if (!wait_full(it_k)) { ok = false; break; }
+            tc_fence_after();
+            issue_qk(0, stage_addr(it_k));
+            tc_commit(bar_s_full(0));
+          }
+          if (!mbar_wait(bar_p_full(1), i & 1, limit)) { ok = false; break; }
+          tc_fence_after();
+          issue_pv(1, stage_addr(it_v), i > 0);
+          tc_commit(bar_o_done(1));
+          tc_commit(bar_kv_empty(it_v % L::kStages));
+          if (more) {
+            issue_qk(1, stage_addr(it_k));
+            tc_commit(bar_s_full(1));
+            tc_commit(bar_kv_empty(it_k % L::kStages));
+          }
+        }
+      }
+      if (!ok) {
+        atomicCAS(p.status, 0u, kStatusTimeoutMma);
+        // tensor-core work already issued must finish before tensor memory is released
+        tc_commit(bar_drain);
+        mbar_wait(bar_drain, 0, limit);
+      }
+    }
+    __syncwarp();
+  }
+
+  // ---- teardown: everyone is done with tensor memory before it is released
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace sol

@@ -1,0 +1,50 @@
+// Plain structs shared between the host-side plan and the kernels.
+#pragma once
+#include <stdint.h>
+
+namespace sol {
+
+// One packed sequence as the kernels see it.  The array is in SCHEDULE order (longest first).
+struct SeqDev {
+  long long tok_start;  // first token of the sequence in the packed tensors
+  int n_tokens;         // text_len + T*H*W
+  int text_len;
+  int T, H, W;
+  int n_qpairs;         // ceil(n_tokens / 256): one CTA handles two 128-row query tiles
+  int n_ktiles;         // ceil(n_tokens / 128)
+  int work_start;       // first CTA index of this sequence (CTAs: head-major, query pair fastest)
+  int ktile_start;      // offset of this sequence in keybits / ktile_list
+  int seq_id;           // index in the caller's order
+};
+
+// Rotary tables: for axis a, entry [tab_off[a] + pos * (rope[a]/2) + j] = (cos, sin)(pos * theta^(-2j/rope[a])).
+struct RopeGeom {
+  int rope[3];
+  int tab_off[3];
+  int head_dim;
+  int heads;
+};
+
+struct AttnParams {
+  const SeqDev* seqs;
+  int n_seqs;
+  int heads;
+  const uint4* keybits;     // [ktile] 128 validity bits (bit b of word w = key 32*w + b of the tile)
+  const int* ktile_list;    // per sequence, tiles that hold at least one valid key, ascending
+  const int* ktile_count;   // per sequence (schedule order)
+  void* out;
+  long long o_tok_stride, o_head_stride;  // in elements
+  float scale_log2;         // log2(e) / sqrt(head_dim)
+  unsigned int* status;     // 0 = fine; written once on a wait time-out
+  unsigned long long wait_limit_ns;
+  unsigned int v_lbo, v_sbo;  // byte offsets of the V (MN-major) shared-memory descriptor
+  float* dbg_scores;        // optional: raw QK^T of the first processed key tile, [cta][2][128][128]
+};
+
+enum : unsigned int {
+  kStatusTimeoutProducer = 1,
+  kStatusTimeoutMma = 2,
+  kStatusTimeoutSoftmax = 3,
+};
+
+}  // namespace sol

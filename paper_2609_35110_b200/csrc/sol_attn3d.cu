@@ -1,0 +1,454 @@
+// Host side of the C-ABI library: plan (pure host), workspace binding, forward.
+#include "../../include/sol_attn3d.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "attn_fwd_sm100.cuh"
+#include "device_types.cuh"
+#include "prologue_kernels.cuh"
+
+namespace {
+
+using sol::SeqDev;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+struct Strides {
+  long long tok, head;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct sol_attn3d_plan_s {
+  int n_seqs = 0, heads = 0, head_dim = 0;
+  int rope[3] = {0, 0, 0};
+  double theta = 10000.0;
+  Strides sq{}, sk{}, sv{}, so{};
+  std::vector<int64_t> cu;            // caller order
+  std::vector<SeqDev> sched;          // schedule order (longest first)
+  long long total_tokens = 0;
+  int total_work = 0;
+  int total_ktiles = 0;
+  std::vector<float2> tables;
+  int tab_off[3] = {0, 0, 0};
+
+  // workspace layout (byte offsets)
+  size_t off_status = 0, off_tables = 0, off_seqs = 0, off_keybits = 0, off_list = 0, off_count = 0, off_qrot = 0,
+         off_krot = 0, ws_bytes = 0;
+  unsigned char* ws = nullptr;
+
+  EncodeTiledFn encode = nullptr;
+  CUtensorMap tm_q{}, tm_k{}, tm_v{};
+  const void* v_cached = nullptr;
+  int keybits_state = 0;              // 0 unknown, 1 built for "no mask", 2 built from a mask
+  int last_cuda = 0;
+  unsigned long long wait_limit_ns = 2000000000ull;
+  unsigned int v_lbo = 0, v_sbo = 1024;
+  float* dbg_scores = nullptr;
+};
+
+namespace {
+
+int fail_cuda(sol_attn3d_plan_t p, cudaError_t e) {
+  p->last_cuda = (int)e;
+  (void)cudaGetLastError();
+  return SOL_ATTN3D_ERR_CUDA;
+}
+
+bool stride_ok(long long s) { return s > 0 && (s * 2) % 16 == 0 && (s * 2) < (1ll << 40); }
+
+int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
+  if (out == nullptr || d == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (d->size != sizeof(sol_attn3d_desc)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (d->n_seqs < 1 || d->grids == nullptr || d->text_lens == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (d->heads < 1 || d->head_dim < 1) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (!(d->theta > 1.0) || !std::isfinite(d->theta)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  int rope_sum = 0;
+  for (int a = 0; a < 3; ++a) {
+    if (d->rope_dims[a] < 0 || (d->rope_dims[a] & 1)) return SOL_ATTN3D_ERR_INVALID_ARG;
+    rope_sum += d->rope_dims[a];
+  }
+  if (d->head_dim != 64 && d->head_dim != 128) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;
+  if (rope_sum > d->head_dim) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (d->heads > 65535) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;
+
+  sol_attn3d_plan_s* p = new (std::nothrow) sol_attn3d_plan_s();
+  if (p == nullptr) return SOL_ATTN3D_ERR_NO_MEMORY;
+  int rc = SOL_ATTN3D_OK;
+  try {
+    p->n_seqs = d->n_seqs;
+    p->heads = d->heads;
+    p->head_dim = d->head_dim;
+    p->theta = d->theta;
+    for (int a = 0; a < 3; ++a) p->rope[a] = d->rope_dims[a];
+
+    const long long dense_tok = (long long)d->heads * d->head_dim;
+    auto take = [&](const int64_t s[2], Strides* dst) {
+      dst->tok = s[0] == 0 ? dense_tok : s[0];
+      dst->head = s[1] == 0 ? d->head_dim : s[1];
+      return stride_ok(dst->tok) && stride_ok(dst->head);
+    };
+    if (!take(d->q_strides, &p->sq) || !take(d->k_strides, &p->sk) || !take(d->v_strides, &p->sv) ||
+        !take(d->out_strides, &p->so)) {
+      delete p;
+      return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;
+    }
+
+    int max_pos[3] = {1, 1, 1};
+    p->cu.assign(1, 0);
+    std::vector<SeqDev> seqs((size_t)d->n_seqs);
+    for (int s = 0; s < d->n_seqs; ++s) {
+      const int T = d->grids[3 * s], H = d->grids[3 * s + 1], W = d->grids[3 * s + 2];
+      const int L = d->text_lens[s];
+      if (T < 0 || H < 1 || W < 1 || L < 0) { rc = SOL_ATTN3D_ERR_INVALID_ARG; break; }
+      const long long nv = (long long)T * H * W;
+      const long long n = nv + L;
+      if (n < 1) { rc = SOL_ATTN3D_ERR_INVALID_ARG; break; }
+      if (n > (1ll << 30)) { rc = SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE; break; }
+      SeqDev& q = seqs[(size_t)s];
+      q.tok_start = p->cu.back();
+      q.n_tokens = (int)n;
+      q.text_len = L;
+      q.T = T; q.H = H; q.W = W;
+      q.n_qpairs = (int)((n + 255) / 256);
+      q.n_ktiles = (int)((n + 127) / 128);
+      q.seq_id = s;
+      p->cu.push_back(p->cu.back() + n);
+      max_pos[0] = std::max(max_pos[0], T);
+      max_pos[1] = std::max(max_pos[1], H);
+      max_pos[2] = std::max(max_pos[2], W);
+    }
+    if (rc == SOL_ATTN3D_OK) {
+      p->total_tokens = p->cu.back();
+      if (p->total_tokens >= (1ll << 31) - 256) rc = SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;
+    }
+    if (rc != SOL_ATTN3D_OK) {
+      delete p;
+      return rc;
+    }
+
+    // schedule: longest sequence first; inside a sequence head-major with the query pair fastest,
+    // so that CTAs running together stream the same head's K/V through L2
+    std::stable_sort(seqs.begin(), seqs.end(), [](const SeqDev& a, const SeqDev& b) { return a.n_tokens > b.n_tokens; });
+    long long work = 0;
+    long long ktiles = 0;
+    for (SeqDev& q : seqs) {
+      q.work_start = (int)work;
+      q.ktile_start = (int)ktiles;
+      work += (long long)q.n_qpairs * d->heads;
+      ktiles += q.n_ktiles;
+      if (work > 0x7fffffffll) break;
+    }
+    if (work > 0x7fffffffll) {
+      delete p;
+      return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;
+    }
+    p->sched = seqs;
+    p->total_work = (int)work;
+    p->total_ktiles = (int)ktiles;
+
+    // cos/sin tables, built in fp64 and rounded once to fp32
+    size_t n_entries = 0;
+    for (int a = 0; a < 3; ++a) {
+      p->tab_off[a] = (int)n_entries;
+      n_entries += (size_t)max_pos[a] * (size_t)(p->rope[a] / 2);
+    }
+    p->tables.resize(std::max<size_t>(n_entries, 1));
+    for (int a = 0; a < 3; ++a) {
+      const int half = p->rope[a] / 2;
+      for (int pos = 0; pos < max_pos[a]; ++pos)
+        for (int j = 0; j < half; ++j) {
+          const double omega = std::exp(-(2.0 * j / p->rope[a]) * std::log(p->theta));
+          const double phi = pos * omega;
+          p->tables[(size_t)p->tab_off[a] + (size_t)pos * half + j] = make_float2((float)std::cos(phi), (float)std::sin(phi));
+        }
+    }
+
+    // workspace layout
+    size_t off = 0;
+    p->off_status = off;  off = align_up(off + 256);
+    p->off_tables = off;  off = align_up(off + p->tables.size() * sizeof(float2));
+    p->off_seqs = off;    off = align_up(off + p->sched.size() * sizeof(SeqDev));
+    p->off_keybits = off; off = align_up(off + (size_t)p->total_ktiles * 16);
+    p->off_list = off;    off = align_up(off + (size_t)p->total_ktiles * sizeof(int));
+    p->off_count = off;   off = align_up(off + (size_t)p->n_seqs * sizeof(int));
+    const size_t rot = (size_t)p->total_tokens * p->heads * p->head_dim * 2;
+    p->off_qrot = off;    off = align_up(off + rot);
+    p->off_krot = off;    off = align_up(off + rot);
+    p->ws_bytes = off;
+
+    if (const char* e = std::getenv("SOL_ATTN3D_WAIT_LIMIT_MS")) {
+      const long v = std::atol(e);
+      if (v > 0) p->wait_limit_ns = (unsigned long long)v * 1000000ull;
+    }
+    p->v_lbo = p->head_dim == 128 ? 16384u : 16u;
+    p->v_sbo = 1024u;
+    if (const char* e = std::getenv("SOL_ATTN3D_DEBUG_V_LBO")) p->v_lbo = (unsigned)std::atol(e);
+    if (const char* e = std::getenv("SOL_ATTN3D_DEBUG_V_SBO")) p->v_sbo = (unsigned)std::atol(e);
+  } catch (const std::bad_alloc&) {
+    delete p;
+    return SOL_ATTN3D_ERR_NO_MEMORY;
+  }
+  *out = p;
+  return SOL_ATTN3D_OK;
+}
+
+// [tokens][heads][D] bf16 tensor as a 3-D TMA map with 128 x 64-element boxes, 128-byte swizzle.
+int encode_map(sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides st) {
+  const cuuint64_t dims[3] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->heads, (cuuint64_t)p->total_tokens};
+  const cuuint64_t strides[2] = {(cuuint64_t)st.head * 2, (cuuint64_t)st.tok * 2};
+  const cuuint32_t box[3] = {64, 1, 128};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = p->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    p->last_cuda = (int)r;
+    return SOL_ATTN3D_ERR_CUDA;
+  }
+  return SOL_ATTN3D_OK;
+}
+
+bool aligned16(const void* x) { return (reinterpret_cast<uintptr_t>(x) & 15u) == 0; }
+
+int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, void* kr, cudaStream_t st) {
+  sol::RopeArgs a{};
+  a.x[0] = static_cast<const __nv_bfloat16*>(q);
+  a.x[1] = static_cast<const __nv_bfloat16*>(k);
+  a.y[0] = static_cast<__nv_bfloat16*>(qr);
+  a.y[1] = static_cast<__nv_bfloat16*>(kr);
+  a.x_tok_stride[0] = p->sq.tok; a.x_head_stride[0] = p->sq.head;
+  a.x_tok_stride[1] = p->sk.tok; a.x_head_stride[1] = p->sk.head;
+  a.seqs = reinterpret_cast<const SeqDev*>(p->ws + p->off_seqs);
+  a.n_seqs = p->n_seqs;
+  a.total_tokens = p->total_tokens;
+  a.tables = reinterpret_cast<const float2*>(p->ws + p->off_tables);
+  for (int i = 0; i < 3; ++i) { a.g.rope[i] = p->rope[i]; a.g.tab_off[i] = p->tab_off[i]; }
+  a.g.head_dim = p->head_dim;
+  a.g.heads = p->heads;
+  const int chunks = p->head_dim / 8;
+  const int hpp = std::max(1, std::min(p->heads, 256 / chunks));
+  const int threads = chunks * hpp;
+  const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
+  sol::rope_qk_kernel<<<(unsigned)blocks, threads, 0, st>>>(a);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? SOL_ATTN3D_OK : fail_cuda(p, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int sol_attn3d_plan(sol_attn3d_plan_t* plan, int B, int heads, int head_dim, int T, int H, int W, int text_len,
+                    const int rope_dims[3]) {
+  if (plan == nullptr || rope_dims == nullptr || B < 1 || B > (1 << 20)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (T < 1) return SOL_ATTN3D_ERR_INVALID_ARG;
+  std::vector<int32_t> grids, lens;
+  try {
+    grids.resize((size_t)B * 3);
+    lens.resize((size_t)B);
+  } catch (const std::bad_alloc&) {
+    return SOL_ATTN3D_ERR_NO_MEMORY;
+  }
+  for (int b = 0; b < B; ++b) {
+    grids[3 * b] = T; grids[3 * b + 1] = H; grids[3 * b + 2] = W;
+    lens[b] = text_len;
+  }
+  sol_attn3d_desc d;
+  std::memset(&d, 0, sizeof(d));
+  d.size = sizeof(d);
+  d.n_seqs = B;
+  d.grids = grids.data();
+  d.text_lens = lens.data();
+  d.heads = heads;
+  d.head_dim = head_dim;
+  for (int a = 0; a < 3; ++a) d.rope_dims[a] = rope_dims[a];
+  d.theta = 10000.0;
+  return build_plan(plan, &d);
+}
+
+int sol_attn3d_plan_ex(sol_attn3d_plan_t* plan, const sol_attn3d_desc* desc) { return build_plan(plan, desc); }
+
+int sol_attn3d_cu_seqlens(sol_attn3d_plan_t plan, const int64_t** cu, int* n_seqs) {
+  if (plan == nullptr || cu == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  *cu = plan->cu.data();
+  if (n_seqs) *n_seqs = plan->n_seqs;
+  return SOL_ATTN3D_OK;
+}
+
+size_t sol_attn3d_workspace_bytes(sol_attn3d_plan_t plan) { return plan ? plan->ws_bytes : 0; }
+
+int sol_attn3d_set_workspace(sol_attn3d_plan_t p, void* device_ptr, size_t bytes) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (device_ptr == nullptr || bytes < p->ws_bytes || (reinterpret_cast<uintptr_t>(device_ptr) % kAlign) != 0)
+    return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  int dev = 0, n_dev = 0;
+  cudaError_t e = cudaGetDeviceCount(&n_dev);
+  if (e != cudaSuccess || n_dev == 0) {
+    (void)cudaGetLastError();
+    return SOL_ATTN3D_ERR_NO_DEVICE;
+  }
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return fail_cuda(p, e);
+  int major = 0;
+  if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess) return fail_cuda(p, e);
+  if (major != 10) return SOL_ATTN3D_ERR_UNSUPPORTED_ARCH;
+
+  if (p->encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) return fail_cuda(p, e);
+    p->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                sol::AttnSmem<128>::kDynBytes)) != cudaSuccess)
+    return fail_cuda(p, e);
+  if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                sol::AttnSmem<64>::kDynBytes)) != cudaSuccess)
+    return fail_cuda(p, e);
+
+  p->ws = static_cast<unsigned char*>(device_ptr);
+  p->keybits_state = 0;
+  p->v_cached = nullptr;
+  if ((e = cudaMemset(p->ws + p->off_status, 0, 256)) != cudaSuccess) return fail_cuda(p, e);
+  if ((e = cudaMemcpy(p->ws + p->off_tables, p->tables.data(), p->tables.size() * sizeof(float2),
+                      cudaMemcpyHostToDevice)) != cudaSuccess)
+    return fail_cuda(p, e);
+  if ((e = cudaMemcpy(p->ws + p->off_seqs, p->sched.data(), p->sched.size() * sizeof(SeqDev),
+                      cudaMemcpyHostToDevice)) != cudaSuccess)
+    return fail_cuda(p, e);
+  const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
+  int rc = encode_map(p, &p->tm_q, p->ws + p->off_qrot, dense);
+  if (rc == SOL_ATTN3D_OK) rc = encode_map(p, &p->tm_k, p->ws + p->off_krot, dense);
+  return rc;
+}
+
+int sol_attn3d_rope_qk(sol_attn3d_plan_t p, const void* q, const void* k, void* q_rot, void* k_rot,
+                       sol_attn3d_stream_t stream) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  if ((q == nullptr) != (q_rot == nullptr) || (k == nullptr) != (k_rot == nullptr)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (q == nullptr && k == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(q_rot) || !aligned16(k_rot)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  return launch_rope(p, q, k, q_rot, k_rot, static_cast<cudaStream_t>(stream));
+}
+
+int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
+                       const uint8_t* key_mask, sol_attn3d_stream_t stream) {
+  if (p == nullptr || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+
+  const SeqDev* d_seqs = reinterpret_cast<const SeqDev*>(p->ws + p->off_seqs);
+  uint32_t* d_bits = reinterpret_cast<uint32_t*>(p->ws + p->off_keybits);
+  int* d_list = reinterpret_cast<int*>(p->ws + p->off_list);
+  int* d_count = reinterpret_cast<int*>(p->ws + p->off_count);
+
+  // (1) validity bits per key tile: rebuilt whenever a mask is given (its contents may have changed)
+  if (key_mask != nullptr || p->keybits_state != 1) {
+    sol::keybits_kernel<<<p->n_seqs, 256, 0, st>>>(d_seqs, key_mask, d_bits, d_list, d_count);
+    if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+    p->keybits_state = key_mask ? 2 : 1;
+  }
+
+  // (2) rotary prologue: Q~, K~ into the workspace
+  int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, st);
+  if (rc != SOL_ATTN3D_OK) return rc;
+
+  // (3) attention
+  if (p->v_cached != v) {
+    rc = encode_map(p, &p->tm_v, v, p->sv);
+    if (rc != SOL_ATTN3D_OK) return rc;
+    p->v_cached = v;
+  }
+  sol::AttnParams ap{};
+  ap.seqs = d_seqs;
+  ap.n_seqs = p->n_seqs;
+  ap.heads = p->heads;
+  ap.keybits = reinterpret_cast<const uint4*>(d_bits);
+  ap.ktile_list = d_list;
+  ap.ktile_count = d_count;
+  ap.out = out;
+  ap.o_tok_stride = p->so.tok;
+  ap.o_head_stride = p->so.head;
+  ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));
+  ap.status = reinterpret_cast<unsigned int*>(p->ws + p->off_status);
+  ap.wait_limit_ns = p->wait_limit_ns;
+  ap.v_lbo = p->v_lbo;
+  ap.v_sbo = p->v_sbo;
+  ap.dbg_scores = p->dbg_scores;
+  if (p->head_dim == 128) {
+    sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(p->tm_q, p->tm_k,
+                                                                                                      p->tm_v, ap);
+  } else {
+    sol::attn_fwd_kernel<64><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(p->tm_q, p->tm_k,
+                                                                                                    p->tm_v, ap);
+  }
+  if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+  return SOL_ATTN3D_OK;
+}
+
+int sol_attn3d_status(sol_attn3d_plan_t p) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  unsigned int w = 0;
+  const cudaError_t e = cudaMemcpy(&w, p->ws + p->off_status, sizeof(w), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(p, e);
+  return w == 0 ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_DEVICE_TIMEOUT;
+}
+
+int sol_attn3d_launches_per_forward(sol_attn3d_plan_t p, int with_mask) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  return with_mask ? 3 : 2;
+}
+
+int sol_attn3d_last_cuda_error(sol_attn3d_plan_t p) { return p ? p->last_cuda : 0; }
+
+const char* sol_attn3d_strerror(int code) {
+  switch (code) {
+    case SOL_ATTN3D_OK: return "ok";
+    case SOL_ATTN3D_ERR_INVALID_ARG: return "invalid argument";
+    case SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE: return "unsupported shape or stride";
+    case SOL_ATTN3D_ERR_NO_WORKSPACE: return "workspace missing, too small or misaligned";
+    case SOL_ATTN3D_ERR_NO_DEVICE: return "no CUDA device";
+    case SOL_ATTN3D_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
+    case SOL_ATTN3D_ERR_CUDA: return "CUDA call failed";
+    case SOL_ATTN3D_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case SOL_ATTN3D_ERR_NO_MEMORY: return "out of host memory";
+    default: return "unknown error";
+  }
+}
+
+int sol_attn3d_destroy(sol_attn3d_plan_t p) {
+  delete p;
+  return SOL_ATTN3D_OK;
+}
+
+#ifdef SOL_ATTN3D_DEBUG_HOOKS
+// Diagnostic build only: raw QK^T of the first key tile of every CTA is written to `dev_buf`
+// ([total_work][2][128][128] floats).
+int sol_attn3d_debug_dump_scores(sol_attn3d_plan_t p, float* dev_buf) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  p->dbg_scores = dev_buf;
+  return SOL_ATTN3D_OK;
+}
+int sol_attn3d_debug_total_work(sol_attn3d_plan_t p) { return p ? p->total_work : 0; }
+#endif
+
+}  // extern "C"
