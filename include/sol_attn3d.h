@@ -144,6 +144,17 @@ int sol_attn3d_rope_qk(sol_attn3d_plan_t plan, const void* q, const void* k, voi
  */
 int sol_attn3d_status(sol_attn3d_plan_t plan);
 
+/*
+ * Per-kernel timing for roofline accounting (Section 3.2 times "SDPA" apart from the layout work
+ * around it).  enable != 0 creates four CUDA events owned by the plan; every later forward records
+ * them on its stream around its three steps.  sol_attn3d_last_forward_ms blocks on the last event
+ * (cudaEventSynchronize) and writes ms[0..2] = {key-validity bits, rotary prologue, attention kernel}
+ * of the most recent forward (0 for a step that was skipped).  Returns INVALID_ARG if profiling is
+ * off or no forward ran.  enable == 0 destroys the events.
+ */
+int sol_attn3d_set_profiling(sol_attn3d_plan_t plan, int enable);
+int sol_attn3d_last_forward_ms(sol_attn3d_plan_t plan, float ms[3]);
+
 /* Number of kernels one sol_attn3d_forward with / without a key mask enqueues (for launch accounting). */
 int sol_attn3d_launches_per_forward(sol_attn3d_plan_t plan, int with_mask);
 

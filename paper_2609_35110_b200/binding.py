@@ -82,6 +82,10 @@ def _lib():
     lib.sol_attn3d_rope_qk.restype = i32
     lib.sol_attn3d_status.argtypes = [vp]
     lib.sol_attn3d_status.restype = i32
+    lib.sol_attn3d_set_profiling.argtypes = [vp, i32]
+    lib.sol_attn3d_set_profiling.restype = i32
+    lib.sol_attn3d_last_forward_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.sol_attn3d_last_forward_ms.restype = i32
     lib.sol_attn3d_launches_per_forward.argtypes = [vp, i32]
     lib.sol_attn3d_launches_per_forward.restype = i32
     lib.sol_attn3d_last_cuda_error.argtypes = [vp]
@@ -180,6 +184,16 @@ def sol_attn3d_rope_qk(plan, q, k, q_rot, k_rot, stream=None) -> None:
 
 def sol_attn3d_status(plan) -> int:
     return int(_lib().sol_attn3d_status(plan))
+
+
+def sol_attn3d_set_profiling(plan, enable: bool) -> None:
+    _check(_lib().sol_attn3d_set_profiling(plan, 1 if enable else 0), "sol_attn3d_set_profiling")
+
+
+def sol_attn3d_last_forward_ms(plan) -> Tuple[float, float, float]:
+    ms = (ctypes.c_float * 3)()
+    _check(_lib().sol_attn3d_last_forward_ms(plan, ms), "sol_attn3d_last_forward_ms")
+    return float(ms[0]), float(ms[1]), float(ms[2])
 
 
 def sol_attn3d_launches_per_forward(plan, with_mask: bool) -> int:

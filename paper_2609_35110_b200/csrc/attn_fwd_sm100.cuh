@@ -25,6 +25,22 @@
 
 namespace sol {
 
+// Diagnostic builds only: per-role cycle accounting (clock64 deltas accumulated per CTA).
+#ifdef SOL_ATTN3D_DEBUG_HOOKS
+#define SOL_PROF_DECL long long prof_t = 0; long long prof_acc[4] = {0, 0, 0, 0};
+#define SOL_PROF_BEGIN() prof_t = clock64()
+#define SOL_PROF_END(slot) prof_acc[slot] += clock64() - prof_t
+#define SOL_PROF_FLUSH(base, n)                                                        \
+  if (p.dbg_prof != nullptr) {                                                         \
+    for (int pi = 0; pi < (n); ++pi) p.dbg_prof[(size_t)blockIdx.x * 16 + (base) + pi] = prof_acc[pi]; \
+  }
+#else
+#define SOL_PROF_DECL
+#define SOL_PROF_BEGIN()
+#define SOL_PROF_END(slot)
+#define SOL_PROF_FLUSH(base, n)
+#endif
+
 constexpr int kAttnThreads = 384;
 
 template <int D>
@@ -124,18 +140,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     float m_ref = -CUDART_INF_F;
     float l = 0.f;
     bool ok = true;
+    SOL_PROF_DECL
 
     for (int i = 0; i < n_proc; ++i) {
       const int jt = __ldg(&ktiles[i]);
       const uint4 kb = __ldg(&keybits[jt]);
+      SOL_PROF_BEGIN();
       ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full(t), i & 1, limit));
       if (!ok) break;
       tc_fence_after();
+      SOL_PROF_END(0);
+      SOL_PROF_BEGIN();
 
       uint32_t r[128];
 #pragma unroll
       for (int cch = 0; cch < 4; ++cch) tmem_ld32(tS + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[cch * 32]));
       tmem_wait_ld();
+      SOL_PROF_END(1);
 
       if (p.dbg_scores != nullptr && i == 0) {
         float* dst = p.dbg_scores + ((size_t)blockIdx.x * 2 + t) * 128 * 128 + (size_t)row * 128;
@@ -188,6 +209,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
 
+      SOL_PROF_BEGIN();
       const float mc = m_ref * c;
       float sum0 = 0.f, sum1 = 0.f;
       uint32_t pk[64];
@@ -200,12 +222,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         pk[cc] = pack_bf16x2(p0, p1);
       }
       l += sum0 + sum1;
+      SOL_PROF_END(2);
+      SOL_PROF_BEGIN();
       tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
       tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_p_full(t));
+      SOL_PROF_END(3);
     }
+    if (lane == 0 && wq == 0) { SOL_PROF_FLUSH(t * 4, 4) }
 
     // ---- epilogue: O / l -> bf16 -> global (rows beyond the sequence are not stored)
     if (ok && n_proc > 0) {
@@ -286,6 +312,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, true);
       bool ok = true;
+      SOL_PROF_DECL
       const uint32_t v_lbo = p.v_lbo, v_sbo = p.v_sbo;
       auto issue_qk = [&](int t, uint32_t kaddr) {
         const uint32_t qaddr = sQ + t * L::kTile;
@@ -324,17 +351,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const uint32_t it_v = it++;
           const bool more = i + 1 < n_proc;
           const uint32_t it_k = more ? it++ : 0;
-          if (!(wait_full(it_v) && mbar_wait(bar_p_full(0), i & 1, limit))) { ok = false; break; }
+          SOL_PROF_BEGIN();
+          if (!wait_full(it_v)) { ok = false; break; }
+          SOL_PROF_END(0);
+          SOL_PROF_BEGIN();
+          if (!mbar_wait(bar_p_full(0), i & 1, limit)) { ok = false; break; }
+          SOL_PROF_END(1);
           tc_fence_after();
           issue_pv(0, stage_addr(it_v), i > 0);
           tc_commit(bar_o_done(0));
           if (more) {
+            SOL_PROF_BEGIN();
             if (!wait_full(it_k)) { ok = false; break; }
+            SOL_PROF_END(2);
             tc_fence_after();
             issue_qk(0, stage_addr(it_k));
             tc_commit(bar_s_full(0));
           }
+          SOL_PROF_BEGIN();
           if (!mbar_wait(bar_p_full(1), i & 1, limit)) { ok = false; break; }
+          SOL_PROF_END(3);
           tc_fence_after();
           issue_pv(1, stage_addr(it_v), i > 0);
           tc_commit(bar_o_done(1));
@@ -346,6 +382,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
         }
       }
+      SOL_PROF_FLUSH(8, 4)
       if (!ok) {
         atomicCAS(p.status, 0u, kStatusTimeoutMma);
         // tensor-core work already issued must finish before tensor memory is released

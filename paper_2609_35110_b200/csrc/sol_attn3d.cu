@@ -58,6 +58,9 @@ struct sol_attn3d_plan_s {
   unsigned long long wait_limit_ns = 2000000000ull;
   unsigned int v_lbo = 0, v_sbo = 1024;
   float* dbg_scores = nullptr;
+  long long* dbg_prof = nullptr;
+  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool prof = false, prof_valid = false, prof_bits = false;
 };
 
 namespace {
@@ -360,16 +363,25 @@ int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const 
   int* d_list = reinterpret_cast<int*>(p->ws + p->off_list);
   int* d_count = reinterpret_cast<int*>(p->ws + p->off_count);
 
+  if (p->prof) {
+    p->prof_valid = false;
+    if ((e = cudaEventRecord(p->ev[0], st)) != cudaSuccess) return fail_cuda(p, e);
+  }
   // (1) validity bits per key tile: rebuilt whenever a mask is given (its contents may have changed)
+  p->prof_bits = false;
   if (key_mask != nullptr || p->keybits_state != 1) {
+    p->prof_bits = true;
     sol::keybits_kernel<<<p->n_seqs, 256, 0, st>>>(d_seqs, key_mask, d_bits, d_list, d_count);
     if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
     p->keybits_state = key_mask ? 2 : 1;
   }
 
+  if (p->prof && (e = cudaEventRecord(p->ev[1], st)) != cudaSuccess) return fail_cuda(p, e);
+
   // (2) rotary prologue: Q~, K~ into the workspace
   int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, st);
   if (rc != SOL_ATTN3D_OK) return rc;
+  if (p->prof && (e = cudaEventRecord(p->ev[2], st)) != cudaSuccess) return fail_cuda(p, e);
 
   // (3) attention
   if (p->v_cached != v) {
@@ -393,6 +405,7 @@ int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const 
   ap.v_lbo = p->v_lbo;
   ap.v_sbo = p->v_sbo;
   ap.dbg_scores = p->dbg_scores;
+  ap.dbg_prof = p->dbg_prof;
   if (p->head_dim == 128) {
     sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(p->tm_q, p->tm_k,
                                                                                                       p->tm_v, ap);
@@ -401,6 +414,42 @@ int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const 
                                                                                                     p->tm_v, ap);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+  if (p->prof) {
+    if ((e = cudaEventRecord(p->ev[3], st)) != cudaSuccess) return fail_cuda(p, e);
+    p->prof_valid = true;
+  }
+  return SOL_ATTN3D_OK;
+}
+
+int sol_attn3d_set_profiling(sol_attn3d_plan_t p, int enable) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if ((enable != 0) == p->prof) return SOL_ATTN3D_OK;
+  if (enable) {
+    for (int i = 0; i < 4; ++i) {
+      const cudaError_t e = cudaEventCreate(&p->ev[i]);
+      if (e != cudaSuccess) {
+        for (int j = 0; j < i; ++j) { cudaEventDestroy(p->ev[j]); p->ev[j] = nullptr; }
+        return fail_cuda(p, e);
+      }
+    }
+    p->prof = true;
+  } else {
+    for (int i = 0; i < 4; ++i) { cudaEventDestroy(p->ev[i]); p->ev[i] = nullptr; }
+    p->prof = false;
+  }
+  p->prof_valid = false;
+  return SOL_ATTN3D_OK;
+}
+
+int sol_attn3d_last_forward_ms(sol_attn3d_plan_t p, float ms[3]) {
+  if (p == nullptr || ms == nullptr || !p->prof || !p->prof_valid) return SOL_ATTN3D_ERR_INVALID_ARG;
+  cudaError_t e = cudaEventSynchronize(p->ev[3]);
+  if (e != cudaSuccess) return fail_cuda(p, e);
+  for (int i = 0; i < 3; ++i) {
+    ms[i] = 0.f;
+    if ((e = cudaEventElapsedTime(&ms[i], p->ev[i], p->ev[i + 1])) != cudaSuccess) return fail_cuda(p, e);
+  }
+  if (!p->prof_bits) ms[0] = 0.f;
   return SOL_ATTN3D_OK;
 }
 
@@ -436,6 +485,7 @@ const char* sol_attn3d_strerror(int code) {
 }
 
 int sol_attn3d_destroy(sol_attn3d_plan_t p) {
+  if (p != nullptr && p->prof) (void)sol_attn3d_set_profiling(p, 0);
   delete p;
   return SOL_ATTN3D_OK;
 }
@@ -446,6 +496,11 @@ int sol_attn3d_destroy(sol_attn3d_plan_t p) {
 int sol_attn3d_debug_dump_scores(sol_attn3d_plan_t p, float* dev_buf) {
   if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   p->dbg_scores = dev_buf;
+  return SOL_ATTN3D_OK;
+}
+int sol_attn3d_debug_prof(sol_attn3d_plan_t p, long long* dev_buf) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  p->dbg_prof = dev_buf;
   return SOL_ATTN3D_OK;
 }
 int sol_attn3d_debug_total_work(sol_attn3d_plan_t p) { return p ? p->total_work : 0; }
