@@ -43,6 +43,86 @@ namespace sol {
 
 constexpr int kAttnThreads = 384;
 
+// Fraction of exponentials evaluated on the FMA pipes instead of the special-function unit: of every
+// kEmuMod adjacent pairs the first kEmuCnt use the polynomial (the MUFU and the tensor core would
+// otherwise need the same number of cycles per tile).
+#ifndef SOL_EMU_MOD
+#define SOL_EMU_MOD 4
+#endif
+#ifndef SOL_EMU_CNT
+#define SOL_EMU_CNT 1
+#endif
+
+__device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
+  float m0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+  float m1 = max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+#pragma unroll
+  for (int cc = 6; cc + 3 < 128; cc += 4) {
+    m0 = max3(m0, __uint_as_float(r[cc]), __uint_as_float(r[cc + 1]));
+    m1 = max3(m1, __uint_as_float(r[cc + 2]), __uint_as_float(r[cc + 3]));
+  }
+  return max3(m0, m1, fmaxf(__uint_as_float(r[126]), __uint_as_float(r[127])));
+}
+
+// 2^x for a packed pair on the FMA pipes: round-to-nearest split x = j + f, f in [-0.5, 0.5], cubic
+// minimax polynomial for 2^f (relative error 7.5e-5, far below the bf16 rounding of P), exponent
+// bits added with integer arithmetic.  Inputs are clamped at -125 (results below 2^-125 are noise).
+__device__ __forceinline__ void exp2_emulated(uint64_t x2, float& p_lo, float& p_hi) {
+  float x_lo, x_hi;
+  unpack_f2(x2, x_lo, x_hi);
+  x2 = pack_f2(fmaxf(x_lo, -125.0f), fmaxf(x_hi, -125.0f));
+  const uint64_t magic = pack_f2(12582912.0f, 12582912.0f);        // 1.5 * 2^23
+  const uint64_t neg_magic = pack_f2(-12582912.0f, -12582912.0f);
+  const uint64_t neg_one = pack_f2(-1.0f, -1.0f);
+  const uint64_t xf = add_f2(x2, magic);                           // integer part lands in the low mantissa bits
+  const uint64_t ji = add_f2(xf, neg_magic);
+  const uint64_t f = fma_f2(ji, neg_one, x2);
+  uint64_t q = fma_f2(f, pack_f2(0.05517148971557617f, 0.05517148971557617f),
+                      pack_f2(0.2426111102104187f, 0.2426111102104187f));
+  q = fma_f2(q, f, pack_f2(0.6932610273361206f, 0.6932610273361206f));
+  q = fma_f2(q, f, pack_f2(0.9999280571937561f, 0.9999280571937561f));
+  float q_lo, q_hi, xf_lo, xf_hi;
+  unpack_f2(q, q_lo, q_hi);
+  unpack_f2(xf, xf_lo, xf_hi);
+  p_lo = __int_as_float(__float_as_int(q_lo) + (__float_as_int(xf_lo) << 23));
+  p_hi = __int_as_float(__float_as_int(q_hi) + (__float_as_int(xf_hi) << 23));
+}
+
+// One pass over a 128-column score row held in registers: p = 2^(s*c - mc) packed to bf16, the fp32
+// row sum of the un-rounded p, and the row maximum of s.  kEmu: evaluate a fixed share of the
+// exponentials with exp2_emulated (never on tiles with masked keys: exp2(-inf) must be exactly 0).
+template <bool kEmu>
+__device__ __forceinline__ void softmax_pass(const uint32_t (&r)[128], float c, float mc, uint32_t (&pk)[64],
+                                             float& sum, float& mx) {
+  const uint64_t c2 = pack_f2(c, c);
+  const uint64_t nmc2 = pack_f2(-mc, -mc);
+  uint64_t acc0 = pack_f2(0.f, 0.f), acc1 = pack_f2(0.f, 0.f);
+  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
+#pragma unroll
+  for (int cc = 0; cc < 64; ++cc) {
+    const float s_lo = __uint_as_float(r[2 * cc]), s_hi = __uint_as_float(r[2 * cc + 1]);
+    const uint64_t x2 = fma_f2(pack_f2(s_lo, s_hi), c2, nmc2);
+    float p_lo, p_hi;
+    if (kEmu && (cc % SOL_EMU_MOD) < SOL_EMU_CNT) {
+      exp2_emulated(x2, p_lo, p_hi);
+    } else {
+      float x_lo, x_hi;
+      unpack_f2(x2, x_lo, x_hi);
+      p_lo = ex2_approx(x_lo);
+      p_hi = ex2_approx(x_hi);
+    }
+    if (cc & 1) { acc1 = add_f2(acc1, pack_f2(p_lo, p_hi)); m1 = max3(m1, s_lo, s_hi); }
+    else        { acc0 = add_f2(acc0, pack_f2(p_lo, p_hi)); m0 = max3(m0, s_lo, s_hi); }
+    pk[cc] = pack_bf16x2(p_lo, p_hi);
+  }
+  float a, b, d, e;
+  unpack_f2(acc0, a, b);
+  unpack_f2(acc1, d, e);
+  sum = (a + b) + (d + e);
+  mx = fmaxf(m0, m1);
+}
+
+
 template <int D>
 struct AttnSmem {
   static constexpr int kTile = 128 * D * 2;               // bytes of one 128 x D bf16 tile
@@ -130,6 +210,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   if (warp < 8) {
     // =========================================================== softmax / correction / epilogue
+    setmaxnreg_inc<216>();
     const int t = warp >> 2;
     const int wq = warp & 3;
     const int row = wq * 32 + lane;
@@ -164,64 +245,46 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int cc = 0; cc < 128; ++cc) dst[cc] = __uint_as_float(r[cc]);
       }
 
-      if ((kb.x & kb.y & kb.z & kb.w) != 0xffffffffu) {
-        // mixed tile: masked or out-of-range keys get -inf
+      const bool mixed = (kb.x & kb.y & kb.z & kb.w) != 0xffffffffu;
+      if (mixed) {
+        // masked or out-of-range keys get -inf
 #pragma unroll
         for (int cc = 0; cc < 128; ++cc) {
           const uint32_t w = cc < 32 ? kb.x : cc < 64 ? kb.y : cc < 96 ? kb.z : kb.w;
           if (((w >> (cc & 31)) & 1u) == 0) r[cc] = __float_as_uint(-CUDART_INF_F);
         }
       }
-
-      float mx0 = __uint_as_float(r[0]), mx1 = __uint_as_float(r[1]);
-      float mx2 = __uint_as_float(r[2]), mx3 = __uint_as_float(r[3]);
-#pragma unroll
-      for (int cc = 4; cc < 128; cc += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(r[cc]));
-        mx1 = fmaxf(mx1, __uint_as_float(r[cc + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(r[cc + 2]));
-        mx3 = fmaxf(mx3, __uint_as_float(r[cc + 3]));
-      }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-
-      // Lazy rescale: the reference maximum only moves when the row maximum has grown by more than
-      // 2^8 in the exp2 domain, so stale-reference terms stay <= 256 and O is rarely touched.
-      if (i == 0) {
-        m_ref = mx;
-      } else {
-        const bool grow = (mx - m_ref) * c > 8.0f;
-        if (__any_sync(0xffffffffu, grow)) {
-          const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
-          if (grow) m_ref = mx;
-          l *= f;
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (i - 1) & 1, limit));
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int cch = 0; cch < D / 32; ++cch) {
-            uint32_t o[32];
-            tmem_ld32(tO + cch * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
-            tmem_st32(tO + cch * 32, o);
-          }
-        }
-      }
+      if (i == 0) m_ref = row_max128(r);
 
       SOL_PROF_BEGIN();
-      const float mc = m_ref * c;
-      float sum0 = 0.f, sum1 = 0.f;
+      // Speculative pass: exponentials against the current reference maximum while the row maximum
+      // of this tile is gathered on the side.  The reference only has to move when the maximum grew
+      // by more than 2^8 in the exp2 domain (stale-reference terms stay <= 256), which is rare.
       uint32_t pk[64];
+      float tile_sum, mx;
+      if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum, mx);
+      else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum, mx);
+      const bool grow = (mx - m_ref) * c > 8.0f;
+      if (__any_sync(0xffffffffu, grow)) {
+        // slow path: move the reference, rescale l and O (complete up to PV(i-1)), redo the tile
+        const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
+        if (grow) m_ref = mx;
+        l *= f;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (i - 1) & 1, limit));
+        if (!ok) break;
+        tc_fence_after();
 #pragma unroll
-      for (int cc = 0; cc < 64; ++cc) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(r[2 * cc]), c, -mc));
-        const float p1 = ex2_approx(fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc));
-        sum0 += p0;
-        sum1 += p1;
-        pk[cc] = pack_bf16x2(p0, p1);
+        for (int cch = 0; cch < D / 32; ++cch) {
+          uint32_t o[32];
+          tmem_ld32(tO + cch * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
+          tmem_st32(tO + cch * 32, o);
+        }
+        softmax_pass<false>(r, c, m_ref * c, pk, tile_sum, mx);
       }
-      l += sum0 + sum1;
+      l += tile_sum;
       SOL_PROF_END(2);
       SOL_PROF_BEGIN();
       tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
@@ -269,7 +332,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     } else if (lane == 0) {
       atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);
     }
-  } else if (warp == 8) {
+  } else {
+    setmaxnreg_dec<64>();
+  }
+  if (warp == 8) {
     // =========================================================== TMA producer
     if (lane == 0) {
       bool ok = true;
@@ -280,13 +346,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int hf = 0; hf < L::kHalves; ++hf)
           tma_load_3d(sQ + t * L::kTile + hf * L::kHalfBytes, &tm_q, bar_q_full, hf * 64, head,
                       tok0 + q_row0 + t * 128);
-      uint32_t it = 0;
+      uint32_t it = 0, stage = 0, par = 0;
       for (int i = 0; i < n_proc && ok; ++i) {
         const int jt = __ldg(&ktiles[i]);
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
-          const uint32_t stage = it % L::kStages;
-          const uint32_t par = (it / L::kStages) & 1u;
           if (!mbar_wait(bar_kv_empty(stage), par ^ 1u, limit)) { ok = false; break; }
           mbar_arrive_expect_tx(bar_kv_full(stage), L::kTile);
           const CUtensorMap* tm = kv ? &tm_v : &tm_k;
@@ -295,6 +359,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tma_load_3d(sKV + stage * L::kTile + hf * L::kHalfBytes, tm, bar_kv_full(stage), hf * 64, head,
                         tok0 + jt * 128);
           ++it;
+          if (++stage == (uint32_t)L::kStages) { stage = 0; par ^= 1u; }
         }
       }
       if (!ok) {
@@ -314,71 +379,81 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       bool ok = true;
       SOL_PROF_DECL
       const uint32_t v_lbo = p.v_lbo, v_sbo = p.v_sbo;
-      auto issue_qk = [&](int t, uint32_t kaddr) {
-        const uint32_t qaddr = sQ + t * L::kTile;
+      // descriptor words: only the low word (address) moves inside the loop
+      const uint32_t hi_k = smem_desc_hi_sw128(1024);
+      const uint32_t hi_v = smem_desc_hi_sw128(v_sbo);
+      const uint32_t q_lo0 = smem_desc_lo(sQ, 16), q_lo1 = smem_desc_lo(sQ + L::kTile, 16);
+      const uint32_t k_lo_base = smem_desc_lo(sKV, 16);
+      const uint32_t v_lo_base = smem_desc_lo(sKV, v_lbo);
+      constexpr uint32_t kStageStep = L::kTile >> 4;
+      const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128;
+      const uint32_t tO0 = tmem_base + 256, tO1 = tmem_base + 256 + D;
+      auto issue_qk = [&](uint32_t d_tmem, uint32_t q_lo, uint32_t stage) {
+        const uint32_t k_lo = k_lo_base + stage * kStageStep;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = (k >> 2) * L::kHalfBytes + (k & 3) * 32;
-          mma_ss(tmem_base + t * 128, smem_desc_sw128(qaddr + off, 16, 1024), smem_desc_sw128(kaddr + off, 16, 1024),
-                 idesc_qk, k > 0 ? 1u : 0u);
+          const uint32_t off = ((k >> 2) * L::kHalfBytes + (k & 3) * 32) >> 4;
+          if (k == 0) mma_ss_lohi<false>(d_tmem, q_lo + off, k_lo + off, hi_k, idesc_qk, 0u);
+          else        mma_ss_lohi<true>(d_tmem, q_lo + off, k_lo + off, hi_k, idesc_qk, 1u);
         }
       };
-      auto issue_pv = [&](int t, uint32_t vaddr, bool acc) {
+      auto issue_pv = [&](uint32_t d_tmem, uint32_t p_tmem, uint32_t stage, bool acc) {
+        const uint32_t v_lo = v_lo_base + stage * kStageStep;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          mma_ts(tmem_base + 256 + t * D, tmem_base + t * 128 + k * 8, smem_desc_sw128(vaddr + k * 2048, v_lbo, v_sbo),
-                 idesc_pv, (acc || k > 0) ? 1u : 0u);
+          if (k == 0) mma_ts_lohi<false>(d_tmem, p_tmem, v_lo, hi_v, idesc_pv, acc ? 1u : 0u);
+          else        mma_ts_lohi<true>(d_tmem, p_tmem + k * 8, v_lo + k * (2048 >> 4), hi_v, idesc_pv, 1u);
         }
       };
-      auto stage_addr = [&](uint32_t it) { return sKV + (it % L::kStages) * L::kTile; };
-      auto wait_full = [&](uint32_t it) {
-        return mbar_wait(bar_kv_full(it % L::kStages), (it / L::kStages) & 1u, limit);
-      };
+      // consumer position in the K/V ring
+      uint32_t st = 0, ph = 0;
+      auto advance = [&]() { if (++st == (uint32_t)L::kStages) { st = 0; ph ^= 1u; } };
 
       if (n_proc > 0) {
-        uint32_t it = 0;
-        ok = mbar_wait(bar_q_full, 0, limit) && wait_full(it);
+        ok = mbar_wait(bar_q_full, 0, limit) && mbar_wait(bar_kv_full(st), ph, limit);
         if (ok) {
           tc_fence_after();
-          issue_qk(0, stage_addr(it));
+          issue_qk(tS0, q_lo0, st);
           tc_commit(bar_s_full(0));
-          issue_qk(1, stage_addr(it));
+          issue_qk(tS1, q_lo1, st);
           tc_commit(bar_s_full(1));
-          tc_commit(bar_kv_empty(it % L::kStages));
-          ++it;
+          tc_commit(bar_kv_empty(st));
+          advance();
         }
         for (int i = 0; i < n_proc && ok; ++i) {
-          const uint32_t it_v = it++;
+          const uint32_t v_st = st, v_ph = ph;
+          advance();
           const bool more = i + 1 < n_proc;
-          const uint32_t it_k = more ? it++ : 0;
+          const uint32_t k_st = st, k_ph = ph;
+          if (more) advance();
           SOL_PROF_BEGIN();
-          if (!wait_full(it_v)) { ok = false; break; }
+          if (!mbar_wait(bar_kv_full(v_st), v_ph, limit)) { ok = false; break; }
           SOL_PROF_END(0);
           SOL_PROF_BEGIN();
           if (!mbar_wait(bar_p_full(0), i & 1, limit)) { ok = false; break; }
           SOL_PROF_END(1);
           tc_fence_after();
-          issue_pv(0, stage_addr(it_v), i > 0);
+          issue_pv(tO0, tS0, v_st, i > 0);
           tc_commit(bar_o_done(0));
           if (more) {
             SOL_PROF_BEGIN();
-            if (!wait_full(it_k)) { ok = false; break; }
+            if (!mbar_wait(bar_kv_full(k_st), k_ph, limit)) { ok = false; break; }
             SOL_PROF_END(2);
             tc_fence_after();
-            issue_qk(0, stage_addr(it_k));
+            issue_qk(tS0, q_lo0, k_st);
             tc_commit(bar_s_full(0));
           }
           SOL_PROF_BEGIN();
           if (!mbar_wait(bar_p_full(1), i & 1, limit)) { ok = false; break; }
           SOL_PROF_END(3);
           tc_fence_after();
-          issue_pv(1, stage_addr(it_v), i > 0);
+          issue_pv(tO1, tS1, v_st, i > 0);
           tc_commit(bar_o_done(1));
-          tc_commit(bar_kv_empty(it_v % L::kStages));
+          tc_commit(bar_kv_empty(v_st));
           if (more) {
-            issue_qk(1, stage_addr(it_k));
+            issue_qk(tS1, q_lo1, k_st);
             tc_commit(bar_s_full(1));
-            tc_commit(bar_kv_empty(it_k % L::kStages));
+            tc_commit(bar_kv_empty(k_st));
           }
         }
       }
