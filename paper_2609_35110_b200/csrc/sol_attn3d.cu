@@ -406,6 +406,10 @@ int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const 
   ap.v_sbo = p->v_sbo;
   ap.dbg_scores = p->dbg_scores;
   ap.dbg_prof = p->dbg_prof;
+  ap.dbg_flags = 0;
+#ifdef SOL_ATTN3D_DEBUG_HOOKS
+  if (const char* e = std::getenv("SOL_ATTN3D_DEBUG_FLAGS")) ap.dbg_flags = (unsigned)std::atol(e);
+#endif
   if (p->head_dim == 128) {
     sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(p->tm_q, p->tm_k,
                                                                                                       p->tm_v, ap);
