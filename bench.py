@@ -32,6 +32,12 @@ from paper_2609_35110_b200 import workloads as wl  # noqa: E402
 METRIC = "attention_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16 = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from the ncu summaries under
+# profiles/ (attn_fwd_kernel_lowres_ncu_full.md, bench_highres_launch_list.md).
+NCU_TRAFFIC = {
+    "lowres": (1023840768, "ncu capture of this workload"),
+    "highres": (int(1023840768 * 111856 / 25216), "scaled from the lowres capture by tokens x heads"),
+}
 
 
 def load_peaks():
@@ -294,15 +300,7 @@ def main():
     achieved = flops / (attn_ms * 1e-3) / 1e12
     long_step = total_ms > 1000.0
     peak = peaks["sustained"] if long_step else peaks["burst"]
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "attn_traffic.json")
-    traffic_note = None
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            tj = json.load(f)
-        if w.name in tj:
-            traffic = tj[w.name]["bytes_per_launch"]
-            traffic_note = tj[w.name].get("note")
+    traffic, traffic_note = NCU_TRAFFIC.get(w.name, (None, None))
 
     # ------------------------------------------------------------------ CPU baseline (oracle, bounded sample)
     cpu = None

@@ -8,9 +8,7 @@
 //   warp  9     tcgen05.mma issuer (one elected lane), owns the TMEM allocation
 //   warps 10-11 idle (complete the third warpgroup)
 // The two query tiles ping-pong: while the softmax of one tile runs on the ALUs, the tensor core
-// works on the other tile's QK^T / PV.  The MMA issuer serves whichever tile has its P ready first
-// (at most one key tile of lead), and P is handed over in two 64-key halves so that the first half
-// of PV overlaps the second half of the softmax.
+// works on the other tile's QK^T / PV.
 //
 // Tensor memory (512 columns x 128 lanes x 32 bit):
 //   [0,128)    S0  (fp32 scores of tile 0);  P0 (bf16, 64 columns) overwrites its first half
@@ -22,8 +20,6 @@
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
-#include <type_traits>
-
 #include "device_types.cuh"
 #include "ptx_sm100.cuh"
 
@@ -31,10 +27,7 @@ namespace sol {
 
 // Diagnostic builds only: per-role cycle accounting (clock64 deltas accumulated per CTA).
 #ifdef SOL_ATTN3D_DEBUG_HOOKS
-#define SOL_DBG_FLAG(bit) ((p.dbg_flags & (bit)) != 0)
-#define SOL_PROF_DECL long long prof_t = 0; long long prof_t2 = 0; long long prof_acc[4] = {0, 0, 0, 0};
-#define SOL_PROF2_BEGIN() prof_t2 = clock64()
-#define SOL_PROF2_END(slot) prof_acc[slot] += clock64() - prof_t2
+#define SOL_PROF_DECL long long prof_t = 0; long long prof_acc[4] = {0, 0, 0, 0};
 #define SOL_PROF_BEGIN() prof_t = clock64()
 #define SOL_PROF_END(slot) prof_acc[slot] += clock64() - prof_t
 #define SOL_PROF_FLUSH(base, n)                                                        \
@@ -42,24 +35,13 @@ namespace sol {
     for (int pi = 0; pi < (n); ++pi) p.dbg_prof[(size_t)blockIdx.x * 16 + (base) + pi] = prof_acc[pi]; \
   }
 #else
-#define SOL_DBG_FLAG(bit) false
 #define SOL_PROF_DECL
 #define SOL_PROF_BEGIN()
 #define SOL_PROF_END(slot)
-#define SOL_PROF2_BEGIN()
-#define SOL_PROF2_END(slot)
 #define SOL_PROF_FLUSH(base, n)
 #endif
 
 constexpr int kAttnThreads = 384;
-
-// MMA issuer's view of one query tile: key-tile turn, which 64-key half of P is awaited, ring position.
-struct TileProgress {
-  int turn;
-  int half;
-  uint32_t stage, phase;   // ring position of the next slot this tile consumes
-  uint32_t index;          // the same position counted in load order (K0 = 0, V0 = 1, K1 = 2, ...)
-};
 
 // Fraction of exponentials evaluated on the FMA pipes instead of the special-function unit: of every
 // kEmuMod adjacent pairs the first kEmuCnt use the polynomial (the MUFU and the tensor core would
@@ -72,15 +54,14 @@ struct TileProgress {
 #endif
 
 __device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
-  float m[4];
+  float m0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+  float m1 = max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
 #pragma unroll
-  for (int q = 0; q < 4; ++q) m[q] = fmaxf(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
-#pragma unroll
-  for (int cc = 8; cc < 128; cc += 8) {
-#pragma unroll
-    for (int q = 0; q < 4; ++q) m[q] = max3(m[q], __uint_as_float(r[cc + 2 * q]), __uint_as_float(r[cc + 2 * q + 1]));
+  for (int cc = 6; cc + 3 < 128; cc += 4) {
+    m0 = max3(m0, __uint_as_float(r[cc]), __uint_as_float(r[cc + 1]));
+    m1 = max3(m1, __uint_as_float(r[cc + 2]), __uint_as_float(r[cc + 3]));
   }
-  return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+  return max3(m0, m1, fmaxf(__uint_as_float(r[126]), __uint_as_float(r[127])));
 }
 
 // 2^x for a packed pair on the FMA pipes: round-to-nearest split x = j + f, f in [-0.5, 0.5], cubic
@@ -107,15 +88,19 @@ __device__ __forceinline__ void exp2_emulated(uint64_t x2, float& p_lo, float& p
   p_hi = __int_as_float(__float_as_int(q_hi) + (__float_as_int(xf_hi) << 23));
 }
 
-// Half a score row (64 columns, registers r[kOff .. kOff+64)): p = 2^(s*c - mc), packed to bf16 into
-// pk[0..32), fp32 sum of the un-rounded p added to acc0/acc1.  kEmu: a fixed share of the exponentials
-// uses exp2_emulated (never on tiles with masked keys: exp2(-inf) must be exactly 0).
-template <bool kEmu, int kOff>
-__device__ __forceinline__ void softmax_half(const uint32_t (&r)[128], uint64_t c2, uint64_t nmc2, uint32_t (&pk)[32],
-                                             uint64_t& acc0, uint64_t& acc1) {
+// One pass over a 128-column score row held in registers: p = 2^(s*c - mc) packed to bf16, the fp32
+// row sum of the un-rounded p, and the row maximum of s.  kEmu: evaluate a fixed share of the
+// exponentials with exp2_emulated (never on tiles with masked keys: exp2(-inf) must be exactly 0).
+template <bool kEmu>
+__device__ __forceinline__ void softmax_pass(const uint32_t (&r)[128], float c, float mc, uint32_t (&pk)[64],
+                                             float& sum, float& mx) {
+  const uint64_t c2 = pack_f2(c, c);
+  const uint64_t nmc2 = pack_f2(-mc, -mc);
+  uint64_t acc0 = pack_f2(0.f, 0.f), acc1 = pack_f2(0.f, 0.f);
+  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
 #pragma unroll
-  for (int cc = 0; cc < 32; ++cc) {
-    const float s_lo = __uint_as_float(r[kOff + 2 * cc]), s_hi = __uint_as_float(r[kOff + 2 * cc + 1]);
+  for (int cc = 0; cc < 64; ++cc) {
+    const float s_lo = __uint_as_float(r[2 * cc]), s_hi = __uint_as_float(r[2 * cc + 1]);
     const uint64_t x2 = fma_f2(pack_f2(s_lo, s_hi), c2, nmc2);
     float p_lo, p_hi;
     if (kEmu && (cc % SOL_EMU_MOD) < SOL_EMU_CNT) {
@@ -126,11 +111,17 @@ __device__ __forceinline__ void softmax_half(const uint32_t (&r)[128], uint64_t 
       p_lo = ex2_approx(x_lo);
       p_hi = ex2_approx(x_hi);
     }
-    if (cc & 1) acc1 = add_f2(acc1, pack_f2(p_lo, p_hi));
-    else        acc0 = add_f2(acc0, pack_f2(p_lo, p_hi));
+    if (cc & 1) { acc1 = add_f2(acc1, pack_f2(p_lo, p_hi)); m1 = max3(m1, s_lo, s_hi); }
+    else        { acc0 = add_f2(acc0, pack_f2(p_lo, p_hi)); m0 = max3(m0, s_lo, s_hi); }
     pk[cc] = pack_bf16x2(p_lo, p_hi);
   }
+  float a, b, d, e;
+  unpack_f2(acc0, a, b);
+  unpack_f2(acc1, d, e);
+  sum = (a + b) + (d + e);
+  mx = fmaxf(m0, m1);
 }
+
 
 template <int D>
 struct AttnSmem {
@@ -141,7 +132,7 @@ struct AttnSmem {
   static constexpr int kOffQ = 0;
   static constexpr int kOffKV = 2 * kTile;
   static constexpr int kOffBars = kOffKV + kStages * kTile;
-  static constexpr int kNumBars = 1 + 2 * kStages + 9;  // q_full, kv_full/empty, s_full[2], p_full[2][2], o_done[2], drain
+  static constexpr int kNumBars = 1 + 2 * kStages + 7;  // q_full, kv_full/empty, s_full, p_full, o_done, drain
   static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
   static constexpr int kBytes = kOffTmemPtr + 16;
   static constexpr int kDynBytes = kBytes + 1024;         // slack to align the base to 1024 bytes
@@ -167,9 +158,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   auto bar_kv_full = [&](int s) { return bars + 8u * (1 + s); };
   auto bar_kv_empty = [&](int s) { return bars + 8u * (1 + L::kStages + s); };
   auto bar_s_full = [&](int t) { return bars + 8u * (1 + 2 * L::kStages + t); };
-  auto bar_p_full = [&](int t, int half) { return bars + 8u * (3 + 2 * L::kStages + 2 * t + half); };
-  auto bar_o_done = [&](int t) { return bars + 8u * (7 + 2 * L::kStages + t); };
-  const uint32_t bar_drain = bars + 8u * (9 + 2 * L::kStages);
+  auto bar_p_full = [&](int t) { return bars + 8u * (3 + 2 * L::kStages + t); };
+  auto bar_o_done = [&](int t) { return bars + 8u * (5 + 2 * L::kStages + t); };
+  const uint32_t bar_drain = bars + 8u * (7 + 2 * L::kStages);
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + L::kOffTmemPtr);
 
   // A fault recorded by an earlier CTA stops later ones at the door (read once, CTA-uniform).
@@ -195,12 +186,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     mbar_init(bar_q_full, 1);
     for (int s = 0; s < L::kStages; ++s) {
       mbar_init(bar_kv_full(s), 1);
-      mbar_init(bar_kv_empty(s), 2);       // released once per query tile
+      mbar_init(bar_kv_empty(s), 1);
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(bar_s_full(t), 1);
-      mbar_init(bar_p_full(t, 0), 4);      // one arrival per softmax warp
-      mbar_init(bar_p_full(t, 1), 4);
+      mbar_init(bar_p_full(t), 128);
       mbar_init(bar_o_done(t), 1);
     }
     mbar_init(bar_drain, 1);
@@ -231,7 +221,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     float m_ref = -CUDART_INF_F;
     float l = 0.f;
     bool ok = true;
-    uint32_t rel_k = 0, rel_v = 0;      // ring stages of K_i and V_{i-1}
     SOL_PROF_DECL
 
     for (int i = 0; i < n_proc; ++i) {
@@ -241,14 +230,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full(t), i & 1, limit));
       if (!ok) break;
       tc_fence_after();
-      // S(i) complete means every earlier MMA of this tile is complete too: QK(i) no longer reads K_i and
-      // PV(i-1) no longer reads V_{i-1}.  Hand both ring stages back (one arrival per query tile).
-      if (wq == 0 && lane == 0) {
-        mbar_arrive(bar_kv_empty(rel_k));
-        if (i > 0) mbar_arrive(bar_kv_empty(rel_v));
-      }
-      rel_v = rel_k + 1 == (uint32_t)L::kStages ? 0u : rel_k + 1;       // V_i follows K_i in the ring
-      rel_k = rel_v + 1 == (uint32_t)L::kStages ? 0u : rel_v + 1;       // K_{i+1}
       SOL_PROF_END(0);
       SOL_PROF_BEGIN();
 
@@ -273,71 +254,51 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (((w >> (cc & 31)) & 1u) == 0) r[cc] = __float_as_uint(-CUDART_INF_F);
         }
       }
+      if (i == 0) m_ref = row_max128(r);
+
       SOL_PROF_BEGIN();
-      const float mx = row_max128(r);
-      // Lazy rescale: the reference maximum only moves when the row maximum has grown by more than
-      // 2^8 in the exp2 domain, so stale-reference terms stay <= 256 and O is rarely touched.
-      if (i == 0) {
-        m_ref = mx;
-      } else {
-        const bool grow = (mx - m_ref) * c > 8.0f;
-        if (__any_sync(0xffffffffu, grow)) {
-          const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
-          if (grow) m_ref = mx;
-          l *= f;
-          // PV(i-1) is complete (see above), so O may be rescaled in place
+      // Speculative pass: exponentials against the current reference maximum while the row maximum
+      // of this tile is gathered on the side.  The reference only has to move when the maximum grew
+      // by more than 2^8 in the exp2 domain (stale-reference terms stay <= 256), which is rare.
+      uint32_t pk[64];
+      float tile_sum, mx;
+      if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum, mx);
+      else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum, mx);
+      const bool grow = (mx - m_ref) * c > 8.0f;
+      if (__any_sync(0xffffffffu, grow)) {
+        // slow path: move the reference, rescale l and O (complete up to PV(i-1)), redo the tile
+        const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
+        if (grow) m_ref = mx;
+        l *= f;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (i - 1) & 1, limit));
+        if (!ok) break;
+        tc_fence_after();
 #pragma unroll
-          for (int cch = 0; cch < D / 32; ++cch) {
-            uint32_t o[32];
-            tmem_ld32(tO + cch * 32, o);
-            tmem_wait_ld();
+        for (int cch = 0; cch < D / 32; ++cch) {
+          uint32_t o[32];
+          tmem_ld32(tO + cch * 32, o);
+          tmem_wait_ld();
 #pragma unroll
-            for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
-            tmem_st32(tO + cch * 32, o);
-          }
-          tmem_wait_st();
+          for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
+          tmem_st32(tO + cch * 32, o);
         }
+        softmax_pass<false>(r, c, m_ref * c, pk, tile_sum, mx);
       }
-      const float mc = m_ref * c;
-      const uint64_t c2 = pack_f2(c, c);
-      const uint64_t nmc2 = pack_f2(-mc, -mc);
-      uint64_t acc0 = pack_f2(0.f, 0.f), acc1 = pack_f2(0.f, 0.f);
-      uint32_t pk[32];
-      // first 64 keys: P into columns [0,32) of S, handed to the MMA issuer at once
-      if (SOL_DBG_FLAG(4u)) {
-#pragma unroll
-        for (int cc = 0; cc < 32; ++cc) pk[cc] = r[cc] & 0x3f803f80u;
-      } else if (mixed) softmax_half<false, 0>(r, c2, nmc2, pk, acc0, acc1);
-      else              softmax_half<true, 0>(r, c2, nmc2, pk, acc0, acc1);
-      tmem_st32(tS, pk);
-      tmem_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p_full(t, 0));
-      // last 64 keys: columns [32,64)
-      if (SOL_DBG_FLAG(4u)) {
-#pragma unroll
-        for (int cc = 0; cc < 32; ++cc) pk[cc] = r[64 + cc] & 0x3f803f80u;
-      } else if (mixed) softmax_half<false, 64>(r, c2, nmc2, pk, acc0, acc1);
-      else              softmax_half<true, 64>(r, c2, nmc2, pk, acc0, acc1);
+      l += tile_sum;
       SOL_PROF_END(2);
       SOL_PROF_BEGIN();
-      tmem_st32(tS + 32, pk);
+      tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p_full(t, 1));
+      mbar_arrive(bar_p_full(t));
       SOL_PROF_END(3);
-      float sa, sb, sc, sd;
-      unpack_f2(acc0, sa, sb);
-      unpack_f2(acc1, sc, sd);
-      l += (sa + sb) + (sc + sd);
     }
     if (lane == 0 && wq == 0) { SOL_PROF_FLUSH(t * 4, 4) }
 
     // ---- epilogue: O / l -> bf16 -> global (rows beyond the sequence are not stored)
     if (ok && n_proc > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), 0, limit));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (n_proc - 1) & 1, limit));
       if (ok) tc_fence_after();
     }
     if (ok) {
@@ -429,7 +390,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint32_t tO0 = tmem_base + 256, tO1 = tmem_base + 256 + D;
       auto issue_qk = [&](uint32_t d_tmem, uint32_t q_lo, uint32_t stage) {
         const uint32_t k_lo = k_lo_base + stage * kStageStep;
-        if (SOL_DBG_FLAG(1u)) return;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint32_t off = ((k >> 2) * L::kHalfBytes + (k & 3) * 32) >> 4;
@@ -437,107 +397,63 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           else        mma_ss_lohi<true>(d_tmem, q_lo + off, k_lo + off, hi_k, idesc_qk, 1u);
         }
       };
-      // PV for one 64-key half (4 k-steps): P columns [32*half, 32*half+32), V rows [64*half, 64*half+64)
-      auto issue_pv_half = [&](uint32_t d_tmem, uint32_t p_tmem, uint32_t stage, int half, bool acc) {
-        const uint32_t v_lo = v_lo_base + stage * kStageStep + half * (4 * (2048 >> 4));
-        const uint32_t p_col = p_tmem + half * 32;
-        if (SOL_DBG_FLAG(2u)) return;
+      auto issue_pv = [&](uint32_t d_tmem, uint32_t p_tmem, uint32_t stage, bool acc) {
+        const uint32_t v_lo = v_lo_base + stage * kStageStep;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (k == 0) mma_ts_lohi<false>(d_tmem, p_col, v_lo, hi_v, idesc_pv, acc ? 1u : 0u);
-          else        mma_ts_lohi<true>(d_tmem, p_col + k * 8, v_lo + k * (2048 >> 4), hi_v, idesc_pv, 1u);
+        for (int k = 0; k < 8; ++k) {
+          if (k == 0) mma_ts_lohi<false>(d_tmem, p_tmem, v_lo, hi_v, idesc_pv, acc ? 1u : 0u);
+          else        mma_ts_lohi<true>(d_tmem, p_tmem + k * 8, v_lo + k * (2048 >> 4), hi_v, idesc_pv, 1u);
         }
       };
+      // consumer position in the K/V ring
+      uint32_t st = 0, ph = 0;
+      auto advance = [&]() { if (++st == (uint32_t)L::kStages) { st = 0; ph ^= 1u; } };
 
       if (n_proc > 0) {
-        // Per query tile: turn index, half within the turn, position in the K/V ring.  Both tiles walk
-        // the same ring (K0 V0 K1 V1 ...); a stage is free again when both have committed past it.
-        TileProgress tp0{0, 0, 0u, 0u, 0u}, tp1{0, 0, 0u, 0u, 0u};
-        uint32_t seen = 1;   // number of ring slots (in load order) already observed full; slot 0 is checked below
-        auto advance = [&](TileProgress& me) {
-          ++me.index;
-          if (++me.stage == (uint32_t)L::kStages) { me.stage = 0; me.phase ^= 1u; }
-        };
-        // the other tile may already have waited for this slot
-        auto wait_slot = [&](const TileProgress& me) -> bool {
-          if (me.index < seen) return true;
-          if (!mbar_wait(bar_kv_full(me.stage), me.phase, limit)) return false;
-          seen = me.index + 1;
-          return true;
-        };
-        // One step for tile T if its next P half has arrived: 1 = progressed, 0 = not ready, -1 = time-out.
-        auto try_serve = [&](auto tag, TileProgress& me, const TileProgress& other) -> int {
-          constexpr int T = decltype(tag)::value;
-          if (me.turn >= n_proc) return 0;
-          if (me.turn > other.turn && other.turn < n_proc) return 0;        // at most one turn of lead
-          if (!mbar_test_wait(bar_p_full(T, me.half), me.turn & 1)) return 0;
-          const uint32_t tS = T ? tS1 : tS0, tO = T ? tO1 : tO0;
-          if (me.half == 0) {
-            SOL_PROF2_BEGIN();
-            if (!wait_slot(me)) return -1;   // V of this turn
-            SOL_PROF2_END(2);
-            tc_fence_after();
-            SOL_PROF2_BEGIN();
-            issue_pv_half(tO, tS, me.stage, 0, me.turn > 0);
-            SOL_PROF2_END(1);
-            me.half = 1;
-          } else {
-            tc_fence_after();
-            SOL_PROF2_BEGIN();
-            issue_pv_half(tO, tS, me.stage, 1, true);
-            SOL_PROF2_END(1);
-            if (me.turn + 1 == n_proc) tc_commit(bar_o_done(T));     // only the last PV needs its own signal
-            advance(me);
-            if (me.turn + 1 < n_proc) {
-              SOL_PROF2_BEGIN();
-              if (!wait_slot(me)) return -1;  // K of the next turn
-              SOL_PROF2_END(2);
-              tc_fence_after();
-              SOL_PROF2_BEGIN();
-              issue_qk(tS, T ? q_lo1 : q_lo0, me.stage);
-              SOL_PROF2_END(3);
-              tc_commit(bar_s_full(T));
-              advance(me);
-            }
-            me.half = 0;
-            ++me.turn;
-          }
-          return 1;
-        };
-
-        ok = mbar_wait(bar_q_full, 0, limit) && mbar_wait(bar_kv_full(0), 0, limit);
+        ok = mbar_wait(bar_q_full, 0, limit) && mbar_wait(bar_kv_full(st), ph, limit);
         if (ok) {
           tc_fence_after();
-          issue_qk(tS0, q_lo0, 0);
+          issue_qk(tS0, q_lo0, st);
           tc_commit(bar_s_full(0));
-          issue_qk(tS1, q_lo1, 0);
+          issue_qk(tS1, q_lo1, st);
           tc_commit(bar_s_full(1));
-          advance(tp0);
-          advance(tp1);
+          tc_commit(bar_kv_empty(st));
+          advance();
         }
-        unsigned long long t_idle0 = 0;
-        uint32_t spins = 0;
-        const std::integral_constant<int, 0> tile0{};
-        const std::integral_constant<int, 1> tile1{};
-        while (ok && (tp0.turn < n_proc || tp1.turn < n_proc)) {
-          int rc;
+        for (int i = 0; i < n_proc && ok; ++i) {
+          const uint32_t v_st = st, v_ph = ph;
+          advance();
+          const bool more = i + 1 < n_proc;
+          const uint32_t k_st = st, k_ph = ph;
+          if (more) advance();
           SOL_PROF_BEGIN();
-          if (tp0.turn <= tp1.turn) {          // the tile that is behind is asked first
-            rc = try_serve(tile0, tp0, tp1);
-            if (rc == 0) rc = try_serve(tile1, tp1, tp0);
-          } else {
-            rc = try_serve(tile1, tp1, tp0);
-            if (rc == 0) rc = try_serve(tile0, tp0, tp1);
+          if (!mbar_wait(bar_kv_full(v_st), v_ph, limit)) { ok = false; break; }
+          SOL_PROF_END(0);
+          SOL_PROF_BEGIN();
+          if (!mbar_wait(bar_p_full(0), i & 1, limit)) { ok = false; break; }
+          SOL_PROF_END(1);
+          tc_fence_after();
+          issue_pv(tO0, tS0, v_st, i > 0);
+          tc_commit(bar_o_done(0));
+          if (more) {
+            SOL_PROF_BEGIN();
+            if (!mbar_wait(bar_kv_full(k_st), k_ph, limit)) { ok = false; break; }
+            SOL_PROF_END(2);
+            tc_fence_after();
+            issue_qk(tS0, q_lo0, k_st);
+            tc_commit(bar_s_full(0));
           }
-          if (rc > 0) { SOL_PROF_END(0); }
-          if (rc < 0) {
-            ok = false;
-          } else if (rc > 0) {
-            spins = 0;
-          } else if ((++spins & 0xfffu) == 0) {
-            const unsigned long long now = globaltimer_ns();
-            if (spins == 0x1000u) t_idle0 = now;
-            if (now - t_idle0 > limit) ok = false;
+          SOL_PROF_BEGIN();
+          if (!mbar_wait(bar_p_full(1), i & 1, limit)) { ok = false; break; }
+          SOL_PROF_END(3);
+          tc_fence_after();
+          issue_pv(tO1, tS1, v_st, i > 0);
+          tc_commit(bar_o_done(1));
+          tc_commit(bar_kv_empty(v_st));
+          if (more) {
+            issue_qk(tS1, q_lo1, k_st);
+            tc_commit(bar_s_full(1));
+            tc_commit(bar_kv_empty(k_st));
           }
         }
       }

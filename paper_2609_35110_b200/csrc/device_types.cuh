@@ -47,6 +47,7 @@ enum : unsigned int {
   kStatusTimeoutProducer = 1,
   kStatusTimeoutMma = 2,
   kStatusTimeoutSoftmax = 3,
+  kStatusBadAlignment = 4,
 };
 
 }  // namespace sol
