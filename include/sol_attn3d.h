@@ -52,7 +52,8 @@ typedef enum {
   SOL_ATTN3D_ERR_UNSUPPORTED_ARCH = -5, /* current device is not compute capability 10.x */
   SOL_ATTN3D_ERR_CUDA = -6,             /* a CUDA call failed; sol_attn3d_last_cuda_error() has the code */
   SOL_ATTN3D_ERR_DEVICE_TIMEOUT = -7,   /* a bounded wait inside a kernel ran out (status word) */
-  SOL_ATTN3D_ERR_NO_MEMORY = -8         /* host allocation failed */
+  SOL_ATTN3D_ERR_NO_MEMORY = -8,        /* host allocation failed */
+  SOL_ATTN3D_ERR_SCRATCH_LIMIT = -9     /* sol_attn3d_forward_noalloc: the plan needs more than the built-in scratch */
 } sol_attn3d_error;
 
 /*
@@ -128,6 +129,45 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t plan, void* device_ptr, size_t by
  */
 int sol_attn3d_forward(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out,
                        const uint8_t* key_mask, sol_attn3d_stream_t stream);
+
+/*
+ * sol_attn3d_forward for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a deployment variant of the call above, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- an inference plugin whose host
+ * framework owns all device memory and forbids allocation inside its enqueue hook, a real-time loop
+ * that may not touch the allocator after start-up, a process whose memory has been handed over
+ * completely to another pool.  Such a caller cannot provide the workspace that sol_attn3d_forward wants.
+ * Here the scratch (rotated Q and K, rotary tables, sequence table, key-validity bits) is a 32 MiB
+ * array built into the library image, so the caller passes only inputs and outputs.  Every GPU context
+ * that loads the library holds those 32 MiB until the process ends, whether this function is used or not.
+ *
+ *   plan           any plan with sol_attn3d_workspace_bytes(plan) <= 32 MiB (33,554,432 bytes); larger
+ *                  plans are refused with SOL_ATTN3D_ERR_SCRATCH_LIMIT before anything is enqueued.
+ *                  No workspace needs to be bound.
+ *   q, k, v, out, key_mask, stream   exactly as for sol_attn3d_forward.
+ *   device_status  optional DEVICE pointer to one 4-byte word (4-byte aligned) that receives the status
+ *                  word of this call: zeroed on `stream` first, nonzero after the stream has drained if
+ *                  a bounded wait inside a kernel ran out (then `out` is undefined).  With NULL the
+ *                  word stays inside the built-in array and cannot be read; sol_attn3d_status does not
+ *                  see this path.
+ *
+ * The function calls no cudaMalloc, cudaFree or other allocating routine, neither directly nor through
+ * a library.  The first call on each device looks up the device address of the built-in array
+ * (cudaGetSymbolAddress), raises the kernels' shared-memory limit and resolves one driver entry
+ * point; do that first call with the device current and before any stream capture begins.  Later
+ * calls only enqueue work: a 4-byte memset, two small host-to-device copies of the plan's tables, and
+ * three kernels.  Nothing synchronises.
+ *
+ * All calls on a device share the one array and it keeps the previous call's contents.  Everything a
+ * call reads from it is rewritten by that call first (the status word is cleared, tables are copied
+ * in again, rotated Q/K and key bits are recomputed), so calls that follow one another on a stream,
+ * also with different plans, are independent.  Calls that OVERLAP on the GPU (different streams, or
+ * host threads racing on the same device) corrupt each other's scratch: serialise them.
+ * Errors: INVALID_ARG, SCRATCH_LIMIT, NO_DEVICE, UNSUPPORTED_ARCH, CUDA.
+ */
+int sol_attn3d_forward_noalloc(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out,
+                               const uint8_t* key_mask, unsigned int* device_status, sol_attn3d_stream_t stream);
 
 /*
  * The rotary prologue alone (Section 3.5 group (2), rotation part): q_rot / k_rot receive the rotated

@@ -52,6 +52,7 @@ ERR_UNSUPPORTED_ARCH = -5
 ERR_CUDA = -6
 ERR_DEVICE_TIMEOUT = -7
 ERR_NO_MEMORY = -8
+ERR_SCRATCH_LIMIT = -9
 
 _LIB = None
 
@@ -78,6 +79,8 @@ def _lib():
     lib.sol_attn3d_set_workspace.restype = i32
     lib.sol_attn3d_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.sol_attn3d_forward.restype = i32
+    lib.sol_attn3d_forward_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sol_attn3d_forward_noalloc.restype = i32
     lib.sol_attn3d_rope_qk.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sol_attn3d_rope_qk.restype = i32
     lib.sol_attn3d_status.argtypes = [vp]
@@ -175,6 +178,26 @@ def sol_attn3d_forward(plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, 
         raise ValueError("key_mask must be a contiguous CUDA uint8 tensor")
     _check(_lib().sol_attn3d_forward(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask), _stream(stream)),
            "sol_attn3d_forward")
+
+
+def sol_attn3d_forward_noalloc(plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                               key_mask: Optional[torch.Tensor] = None, device_status: Optional[torch.Tensor] = None,
+                               stream=None) -> None:
+    """Forward without a caller workspace: the scratch is the 32 MiB array inside the library.
+
+    For callers that may not allocate device memory (see include/sol_attn3d.h).  ``device_status`` is an
+    optional CUDA int32 tensor with one element that receives the call's status word.  Calls on one
+    device must not overlap on the GPU.
+    """
+    for t in (q, k, v, out):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v, out must be CUDA bf16 tensors")
+    if key_mask is not None and (not key_mask.is_cuda or key_mask.dtype != torch.uint8 or not key_mask.is_contiguous()):
+        raise ValueError("key_mask must be a contiguous CUDA uint8 tensor")
+    if device_status is not None and (not device_status.is_cuda or device_status.element_size() != 4):
+        raise ValueError("device_status must be a CUDA tensor of 4-byte elements")
+    _check(_lib().sol_attn3d_forward_noalloc(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask),
+                                             _ptr(device_status), _stream(stream)), "sol_attn3d_forward_noalloc")
 
 
 def sol_attn3d_rope_qk(plan, q, k, q_rot, k_rot, stream=None) -> None:

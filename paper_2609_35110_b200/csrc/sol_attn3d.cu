@@ -457,6 +457,165 @@ int sol_attn3d_last_forward_ms(sol_attn3d_plan_t p, float ms[3]) {
   return SOL_ATTN3D_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Variant of sol_attn3d_forward for callers that cannot allocate device memory at all.
+//
+// The scratch that the kernels need (rotated Q and K, rotary tables, sequence table, key-validity
+// bits) lives in one array that is part of the library image.  Its size is fixed when the library is
+// built; every GPU context that loads the library holds that much memory until the process exits.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = 32u << 20;   // 32 MiB
+static __device__ __align__(256) unsigned char sol_attn3d_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+// Device address of the array per device.  The array's name is only a host-side handle in host code;
+// the address a kernel can use comes from cudaGetSymbolAddress, asked once per device.
+unsigned char* g_static_scratch_addr[kMaxDevices] = {};
+EncodeTiledFn g_static_encode = nullptr;
+
+int static_scratch_for_current_device(sol_attn3d_plan_t p, unsigned char** out) {
+  int dev = 0, n_dev = 0;
+  cudaError_t e = cudaGetDeviceCount(&n_dev);
+  if (e != cudaSuccess || n_dev == 0) {
+    (void)cudaGetLastError();
+    return SOL_ATTN3D_ERR_NO_DEVICE;
+  }
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return fail_cuda(p, e);
+  if (dev < 0 || dev >= kMaxDevices) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;
+  if (g_static_scratch_addr[dev] == nullptr) {
+    int major = 0;
+    if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
+      return fail_cuda(p, e);
+    if (major != 10) return SOL_ATTN3D_ERR_UNSUPPORTED_ARCH;
+    unsigned char* addr = nullptr;
+    if ((e = cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), sol_attn3d_static_scratch)) != cudaSuccess)
+      return fail_cuda(p, e);
+    if (addr == nullptr || (reinterpret_cast<uintptr_t>(addr) % kAlign) != 0) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+    if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  sol::AttnSmem<128>::kDynBytes)) != cudaSuccess)
+      return fail_cuda(p, e);
+    if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  sol::AttnSmem<64>::kDynBytes)) != cudaSuccess)
+      return fail_cuda(p, e);
+    if (g_static_encode == nullptr) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+      if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) return fail_cuda(p, e);
+      g_static_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    g_static_scratch_addr[dev] = addr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return SOL_ATTN3D_OK;
+}
+
+int encode_map_with(EncodeTiledFn fn, sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides st) {
+  const cuuint64_t dims[3] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->heads, (cuuint64_t)p->total_tokens};
+  const cuuint64_t strides[2] = {(cuuint64_t)st.head * 2, (cuuint64_t)st.tok * 2};
+  const cuuint32_t box[3] = {64, 1, 128};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    p->last_cuda = (int)r;
+    return SOL_ATTN3D_ERR_CUDA;
+  }
+  return SOL_ATTN3D_OK;
+}
+}  // namespace
+
+int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
+                               const uint8_t* key_mask, unsigned int* device_status, sol_attn3d_stream_t stream) {
+  if (p == nullptr || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(device_status) & 3u) != 0) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws_bytes > kStaticScratchBytes) return SOL_ATTN3D_ERR_SCRATCH_LIMIT;
+  unsigned char* ws = nullptr;
+  int rc = static_scratch_for_current_device(p, &ws);
+  if (rc != SOL_ATTN3D_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+
+  // The array still holds whatever the previous call (of any plan) left there.  What this call reads
+  // before writing is rewritten here: the status word starts at zero, tables and sequence table are
+  // copied in again; Q~, K~ and the key bits are produced by this call's own kernels.
+  unsigned int* status = device_status ? device_status : reinterpret_cast<unsigned int*>(ws + p->off_status);
+  if ((e = cudaMemsetAsync(status, 0, sizeof(unsigned int), st)) != cudaSuccess) return fail_cuda(p, e);
+  if ((e = cudaMemcpyAsync(ws + p->off_tables, p->tables.data(), p->tables.size() * sizeof(float2),
+                           cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return fail_cuda(p, e);
+  if ((e = cudaMemcpyAsync(ws + p->off_seqs, p->sched.data(), p->sched.size() * sizeof(SeqDev),
+                           cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return fail_cuda(p, e);
+
+  const SeqDev* d_seqs = reinterpret_cast<const SeqDev*>(ws + p->off_seqs);
+  uint32_t* d_bits = reinterpret_cast<uint32_t*>(ws + p->off_keybits);
+  int* d_list = reinterpret_cast<int*>(ws + p->off_list);
+  int* d_count = reinterpret_cast<int*>(ws + p->off_count);
+  sol::keybits_kernel<<<p->n_seqs, 256, 0, st>>>(d_seqs, key_mask, d_bits, d_list, d_count);
+  if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+
+  {
+    sol::RopeArgs a{};
+    a.x[0] = static_cast<const __nv_bfloat16*>(q);
+    a.x[1] = static_cast<const __nv_bfloat16*>(k);
+    a.y[0] = reinterpret_cast<__nv_bfloat16*>(ws + p->off_qrot);
+    a.y[1] = reinterpret_cast<__nv_bfloat16*>(ws + p->off_krot);
+    a.x_tok_stride[0] = p->sq.tok; a.x_head_stride[0] = p->sq.head;
+    a.x_tok_stride[1] = p->sk.tok; a.x_head_stride[1] = p->sk.head;
+    a.seqs = d_seqs;
+    a.n_seqs = p->n_seqs;
+    a.total_tokens = p->total_tokens;
+    a.tables = reinterpret_cast<const float2*>(ws + p->off_tables);
+    for (int i = 0; i < 3; ++i) { a.g.rope[i] = p->rope[i]; a.g.tab_off[i] = p->tab_off[i]; }
+    a.g.head_dim = p->head_dim;
+    a.g.heads = p->heads;
+    const int chunks = p->head_dim / 8;
+    const int hpp = std::max(1, std::min(p->heads, 256 / chunks));
+    const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
+    sol::rope_qk_kernel<<<(unsigned)blocks, chunks * hpp, 0, st>>>(a);
+    if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+  }
+
+  CUtensorMap tm_q, tm_k, tm_v;
+  const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
+  if ((rc = encode_map_with(g_static_encode, p, &tm_q, ws + p->off_qrot, dense)) != SOL_ATTN3D_OK) return rc;
+  if ((rc = encode_map_with(g_static_encode, p, &tm_k, ws + p->off_krot, dense)) != SOL_ATTN3D_OK) return rc;
+  if ((rc = encode_map_with(g_static_encode, p, &tm_v, v, p->sv)) != SOL_ATTN3D_OK) return rc;
+
+  sol::AttnParams ap{};
+  ap.seqs = d_seqs;
+  ap.n_seqs = p->n_seqs;
+  ap.heads = p->heads;
+  ap.keybits = reinterpret_cast<const uint4*>(d_bits);
+  ap.ktile_list = d_list;
+  ap.ktile_count = d_count;
+  ap.out = out;
+  ap.o_tok_stride = p->so.tok;
+  ap.o_head_stride = p->so.head;
+  ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));
+  ap.status = status;
+  ap.wait_limit_ns = p->wait_limit_ns;
+  ap.v_lbo = p->v_lbo;
+  ap.v_sbo = p->v_sbo;
+  ap.dbg_scores = nullptr;
+  ap.dbg_prof = nullptr;
+  ap.dbg_flags = 0;
+  if (p->head_dim == 128) {
+    sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(tm_q, tm_k, tm_v,
+                                                                                                      ap);
+  } else {
+    sol::attn_fwd_kernel<64><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(tm_q, tm_k, tm_v,
+                                                                                                    ap);
+  }
+  if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+  return SOL_ATTN3D_OK;
+}
+
 int sol_attn3d_status(sol_attn3d_plan_t p) {
   if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
@@ -484,6 +643,7 @@ const char* sol_attn3d_strerror(int code) {
     case SOL_ATTN3D_ERR_CUDA: return "CUDA call failed";
     case SOL_ATTN3D_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case SOL_ATTN3D_ERR_NO_MEMORY: return "out of host memory";
+    case SOL_ATTN3D_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the built-in 32 MiB array holds";
     default: return "unknown error";
   }
 }
