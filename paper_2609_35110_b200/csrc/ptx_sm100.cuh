@@ -56,7 +56,21 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   return t;
 }
 // Bounded wait: returns false if `limit_ns` of wall time passed without the phase completing.
+// SOL_SPIN_TEST_WAIT: poll with the non-blocking test_wait instead of try_wait (which may park the
+// thread for a hardware time slice and wake it late).
+#ifndef SOL_SPIN_TEST_WAIT
+#define SOL_SPIN_TEST_WAIT 1
+#endif
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
+#if SOL_SPIN_TEST_WAIT
+  if (mbar_test_wait(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (!mbar_test_wait(bar, parity)) {
+    if ((++spins & 0x3ffu) == 0 && globaltimer_ns() - t0 > limit_ns) return false;
+  }
+  return true;
+#else
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
@@ -64,6 +78,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_
     if ((++spins & 0x3ffu) == 0 && globaltimer_ns() - t0 > limit_ns) return false;
   }
   return true;
+#endif
+}
+
+// The same for a whole converged warp: every lane polls, the verdict is made uniform.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, limit_ns));
 }
 
 // ------------------------------------------------------------------ TMA
@@ -169,6 +189,64 @@ __device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, ui
         : "memory");
   }
 }
+// Warp-uniform variants: every lane of the (converged) warp executes the call, one elected lane issues
+// the instruction.  Keeping the issuing warp convergent lets the compiler hold descriptors and addresses
+// in uniform registers instead of moving them over from per-thread registers for every instruction.
+template <bool kAcc>
+__device__ __forceinline__ void mma_ss_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                             uint32_t accumulate) {
+  if (kAcc) {
+    asm volatile(
+        "{\n\t.reg .pred p, pe;\n\t.reg .b32 re;\n\t.reg .b64 da, db;\n\t"
+        "elect.sync re|pe, 0xffffffff;\n\t"
+        "setp.eq.u32 p, 0, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p, pe;\n\t.reg .b32 re;\n\t.reg .b64 da, db;\n\t"
+        "elect.sync re|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+template <bool kAcc>
+__device__ __forceinline__ void mma_ts_elect(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc, uint32_t accumulate) {
+  if (kAcc) {
+    asm volatile(
+        "{\n\t.reg .pred p, pe;\n\t.reg .b32 re;\n\t.reg .b64 db;\n\t"
+        "elect.sync re|pe, 0xffffffff;\n\t"
+        "setp.eq.u32 p, 0, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p, pe;\n\t.reg .b32 re;\n\t.reg .b64 db;\n\t"
+        "elect.sync re|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+__device__ __forceinline__ void tc_commit_elect(uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\t.reg .b32 re;\n\t"
+      "elect.sync re|pe, 0xffffffff;\n\t"
+      "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar)
+      : "memory");
+}
+
 // Low / high words of a 128-byte-swizzle shared-memory descriptor (see smem_desc_sw128 below).
 __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
   return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
