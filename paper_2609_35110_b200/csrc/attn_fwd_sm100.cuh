@@ -49,13 +49,13 @@ constexpr int kAttnThreads = 384;
 // kEmuMod adjacent pairs the first kEmuCnt use the polynomial (the MUFU and the tensor core would
 // otherwise need the same number of cycles per tile).
 #ifndef SOL_TURNS
-#define SOL_TURNS 1
+#define SOL_TURNS 0
 #endif
 #ifndef SOL_EMU_MOD
 #define SOL_EMU_MOD 4
 #endif
 #ifndef SOL_EMU_CNT
-#define SOL_EMU_CNT 1
+#define SOL_EMU_CNT 0
 #endif
 
 __device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
@@ -69,28 +69,19 @@ __device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
   return max3(m0, m1, fmaxf(__uint_as_float(r[126]), __uint_as_float(r[127])));
 }
 
-// 2^x for a packed pair on the FMA pipes: round-to-nearest split x = j + f, f in [-0.5, 0.5], cubic
-// minimax polynomial for 2^f (relative error 7.5e-5, far below the bf16 rounding of P), exponent
-// bits added with integer arithmetic.  Inputs are clamped at -125 (results below 2^-125 are noise).
-__device__ __forceinline__ void exp2_emulated(uint64_t x2, float& p_lo, float& p_hi) {
-  float x_lo, x_hi;
-  unpack_f2(x2, x_lo, x_hi);
-  x2 = pack_f2(fmaxf(x_lo, -125.0f), fmaxf(x_hi, -125.0f));
-  const uint64_t magic = pack_f2(12582912.0f, 12582912.0f);        // 1.5 * 2^23
-  const uint64_t neg_magic = pack_f2(-12582912.0f, -12582912.0f);
-  const uint64_t neg_one = pack_f2(-1.0f, -1.0f);
-  const uint64_t xf = add_f2(x2, magic);                           // integer part lands in the low mantissa bits
-  const uint64_t ji = add_f2(xf, neg_magic);
-  const uint64_t f = fma_f2(ji, neg_one, x2);
-  uint64_t q = fma_f2(f, pack_f2(0.05517148971557617f, 0.05517148971557617f),
-                      pack_f2(0.2426111102104187f, 0.2426111102104187f));
-  q = fma_f2(q, f, pack_f2(0.6932610273361206f, 0.6932610273361206f));
-  q = fma_f2(q, f, pack_f2(0.9999280571937561f, 0.9999280571937561f));
-  float q_lo, q_hi, xf_lo, xf_hi;
-  unpack_f2(q, q_lo, q_hi);
-  unpack_f2(xf, xf_lo, xf_hi);
-  p_lo = __int_as_float(__float_as_int(q_lo) + (__float_as_int(xf_lo) << 23));
-  p_hi = __int_as_float(__float_as_int(q_hi) + (__float_as_int(xf_hi) << 23));
+// 2^x on the FMA / integer pipes: round-to-nearest split x = j + f, f in [-0.5, 0.5], cubic minimax
+// polynomial for 2^f (relative error 7.5e-5, far below the bf16 rounding of P), exponent bits added with
+// integer arithmetic.  Inputs are clamped at -125 (results below 2^-125 are noise).
+// Scalar fp32 on purpose: on this part a packed fma.f32x2 occupies the FMA pipe about four times as long
+// as one scalar FFMA (measured), so packing saves issue slots but costs pipe time.
+__device__ __forceinline__ float exp2_emulated(float x) {
+  x = fmaxf(x, -125.0f);
+  const float xf = x + 12582912.0f;                 // 1.5 * 2^23: integer part lands in the low mantissa bits
+  const float f = x - (xf - 12582912.0f);
+  float q = fmaf(f, 0.05517148971557617f, 0.2426111102104187f);
+  q = fmaf(q, f, 0.6932610273361206f);
+  q = fmaf(q, f, 0.9999280571937561f);
+  return __int_as_float(__float_as_int(q) + (__float_as_int(xf) << 23));
 }
 
 // One pass over a 128-column score row held in registers: p = 2^(s*c - mc) packed to bf16, the fp32
@@ -99,34 +90,29 @@ __device__ __forceinline__ void exp2_emulated(uint64_t x2, float& p_lo, float& p
 template <bool kEmu>
 __device__ __forceinline__ void softmax_pass(const uint32_t (&r)[128], float c, float mc, uint32_t (&pk)[64],
                                              float& sum, float& mx) {
-  const uint64_t c2 = pack_f2(c, c);
-  const uint64_t nmc2 = pack_f2(-mc, -mc);
-  uint64_t acc0 = pack_f2(0.f, 0.f), acc1 = pack_f2(0.f, 0.f);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
   float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
 #pragma unroll
   for (int cc = 0; cc < 64; ++cc) {
     const float s_lo = __uint_as_float(r[2 * cc]), s_hi = __uint_as_float(r[2 * cc + 1]);
-    const uint64_t x2 = fma_f2(pack_f2(s_lo, s_hi), c2, nmc2);
+    const float x_lo = fmaf(s_lo, c, -mc), x_hi = fmaf(s_hi, c, -mc);
     float p_lo, p_hi;
     if (kEmu && (cc % SOL_EMU_MOD) < SOL_EMU_CNT) {
-      exp2_emulated(x2, p_lo, p_hi);
+      p_lo = exp2_emulated(x_lo);
+      p_hi = exp2_emulated(x_hi);
     } else {
-      float x_lo, x_hi;
-      unpack_f2(x2, x_lo, x_hi);
       p_lo = ex2_approx(x_lo);
       p_hi = ex2_approx(x_hi);
     }
-    if (cc & 1) { acc1 = add_f2(acc1, pack_f2(p_lo, p_hi)); m1 = max3(m1, s_lo, s_hi); }
-    else        { acc0 = add_f2(acc0, pack_f2(p_lo, p_hi)); m0 = max3(m0, s_lo, s_hi); }
+    acc[(2 * cc) & 3] += p_lo;
+    acc[(2 * cc + 1) & 3] += p_hi;
+    if (cc & 1) m1 = max3(m1, s_lo, s_hi);
+    else        m0 = max3(m0, s_lo, s_hi);
     pk[cc] = pack_bf16x2(p_lo, p_hi);
   }
-  float a, b, d, e;
-  unpack_f2(acc0, a, b);
-  unpack_f2(acc1, d, e);
-  sum = (a + b) + (d + e);
+  sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
   mx = fmaxf(m0, m1);
 }
-
 
 template <int D>
 struct AttnSmem {

@@ -59,7 +59,7 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 // SOL_SPIN_TEST_WAIT: poll with the non-blocking test_wait instead of try_wait (which may park the
 // thread for a hardware time slice and wake it late).
 #ifndef SOL_SPIN_TEST_WAIT
-#define SOL_SPIN_TEST_WAIT 1
+#define SOL_SPIN_TEST_WAIT 0
 #endif
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
 #if SOL_SPIN_TEST_WAIT
