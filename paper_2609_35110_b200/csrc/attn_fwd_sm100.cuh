@@ -43,7 +43,18 @@ namespace sol {
 #define SOL_PROF_FLUSH(base, n)
 #endif
 
-constexpr int kAttnThreads = 384;
+// Register split after launch (384 threads x 168): the softmax warpgroups take what the third
+// warpgroup (producer, MMA issuer, two idle warps) gives back: (168 - other) * 128 >= (softmax - 168) * 256.
+#ifndef SOL_REGS_SOFTMAX
+#define SOL_REGS_SOFTMAX 216
+#endif
+#ifndef SOL_REGS_OTHER
+#define SOL_REGS_OTHER 64
+#endif
+#ifndef SOL_ATTN_THREADS
+#define SOL_ATTN_THREADS 384
+#endif
+constexpr int kAttnThreads = SOL_ATTN_THREADS;   // 8 softmax warps + producer + MMA issuer (+ 2 idle warps if 384)
 
 // Fraction of exponentials evaluated on the FMA pipes instead of the special-function unit: of every
 // kEmuMod adjacent pairs the first kEmuCnt use the polynomial (the MUFU and the tensor core would
@@ -204,7 +215,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   if (warp < 8) {
     // =========================================================== softmax / correction / epilogue
-    setmaxnreg_inc<216>();
+#if SOL_ATTN_THREADS == 384
+    setmaxnreg_inc<SOL_REGS_SOFTMAX>();
+#endif
     const int t = warp >> 2;
     const int wq = warp & 3;
     const int row = wq * 32 + lane;
@@ -346,7 +359,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);
     }
   } else {
-    setmaxnreg_dec<64>();
+#if SOL_ATTN_THREADS == 384
+    setmaxnreg_dec<SOL_REGS_OTHER>();
+#endif
   }
   if (warp == 8) {
     // =========================================================== TMA producer
