@@ -95,18 +95,17 @@ __device__ __forceinline__ float exp2_emulated(float x) {
   return __int_as_float(__float_as_int(q) + (__float_as_int(xf) << 23));
 }
 
-// One pass over a 128-column score row held in registers: p = 2^(s*c - mc) packed to bf16, the fp32
-// row sum of the un-rounded p, and the row maximum of s.  kEmu: evaluate a fixed share of the
-// exponentials with exp2_emulated (never on tiles with masked keys: exp2(-inf) must be exactly 0).
+// One pass over a 128-column score row held in registers: p = 2^(s*c - mc) packed to bf16 and the fp32
+// row sum of the un-rounded p.  kEmu: evaluate a fixed share of the exponentials with exp2_emulated
+// (never on tiles with masked keys: exp2(-inf) must be exactly 0).
 template <bool kEmu>
 __device__ __forceinline__ void softmax_pass(const uint32_t (&r)[128], float c, float mc, uint32_t (&pk)[64],
-                                             float& sum, float& mx) {
+                                             float& sum) {
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;
 #pragma unroll
   for (int cc = 0; cc < 64; ++cc) {
-    const float s_lo = __uint_as_float(r[2 * cc]), s_hi = __uint_as_float(r[2 * cc + 1]);
-    const float x_lo = fmaf(s_lo, c, -mc), x_hi = fmaf(s_hi, c, -mc);
+    const float x_lo = fmaf(__uint_as_float(r[2 * cc]), c, -mc);
+    const float x_hi = fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc);
     float p_lo, p_hi;
     if (kEmu && (cc % SOL_EMU_MOD) < SOL_EMU_CNT) {
       p_lo = exp2_emulated(x_lo);
@@ -117,12 +116,9 @@ __device__ __forceinline__ void softmax_pass(const uint32_t (&r)[128], float c, 
     }
     acc[(2 * cc) & 3] += p_lo;
     acc[(2 * cc + 1) & 3] += p_hi;
-    if (cc & 1) m1 = max3(m1, s_lo, s_hi);
-    else        m0 = max3(m0, s_lo, s_hi);
     pk[cc] = pack_bf16x2(p_lo, p_hi);
   }
   sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-  mx = fmaxf(m0, m1);
 }
 
 template <int D>
@@ -277,32 +273,37 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (i == 0) m_ref = row_max128(r);
 
       SOL_PROF_BEGIN();
-      // Speculative pass: exponentials against the current reference maximum while the row maximum
-      // of this tile is gathered on the side.  The reference only has to move when the maximum grew
-      // by more than 2^8 in the exp2 domain (stale-reference terms stay <= 256), which is rare.
+      // Speculative pass: exponentials against the current reference maximum, no row maximum taken.
+      // All terms are positive, so a row sum <= 2^8 proves that every term is <= 2^8: the reference
+      // is still good enough (the result does not depend on which reference is used, only overflow
+      // does).  Only when the sum is larger (or not finite) is the row maximum computed; if it has grown
+      // by more than 2^8 in the exp2 domain the reference moves, l and O are rescaled and the tile is
+      // redone from the scores still held in registers, before any of its P is released.  Rare.
       uint32_t pk[64];
-      float tile_sum, mx;
-      if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum, mx);
-      else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum, mx);
-      const bool grow = (mx - m_ref) * c > 8.0f;
-      if (__any_sync(0xffffffffu, grow)) {
-        // slow path: move the reference, rescale l and O (complete up to PV(i-1)), redo the tile
-        const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
-        if (grow) m_ref = mx;
-        l *= f;
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (i - 1) & 1, limit));
-        if (!ok) break;
-        tc_fence_after();
+      float tile_sum;
+      if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
+      else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum);
+      if (__any_sync(0xffffffffu, !(tile_sum <= 256.0f))) {
+        const float mx = row_max128(r);
+        const bool grow = (mx - m_ref) * c > 8.0f;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
+          if (grow) m_ref = mx;
+          l *= f;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (i - 1) & 1, limit));
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
-        for (int cch = 0; cch < D / 32; ++cch) {
-          uint32_t o[32];
-          tmem_ld32(tO + cch * 32, o);
-          tmem_wait_ld();
+          for (int cch = 0; cch < D / 32; ++cch) {
+            uint32_t o[32];
+            tmem_ld32(tO + cch * 32, o);
+            tmem_wait_ld();
 #pragma unroll
-          for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
-          tmem_st32(tO + cch * 32, o);
+            for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
+            tmem_st32(tO + cch * 32, o);
+          }
+          softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
         }
-        softmax_pass<false>(r, c, m_ref * c, pk, tile_sum, mx);
       }
       l += tile_sum;
 #if SOL_TURNS
