@@ -104,6 +104,20 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of per-rank times over all ranks (identity without a process group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_tflops(flops_per_replica, world, ms_per_step):
+    """Replicas only: every rank runs the same workload, the job's rate is world x one replica's work over the slowest time."""
+    return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
 def oracle_sample(w, inp_cpu, heads_sample, rows_per_head):
     """(seq, head, rows) selection used by the CPU baseline: the parity rows of a few heads."""
     sel = []
@@ -281,11 +295,9 @@ def main():
     # ------------------------------------------------------------------ max over ranks
     ms_per_step = total_ms / args.steps
     if dist is not None:
-        t = torch.tensor([ms_per_step, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t[0])
+        ms_per_step, e_max = max_over_ranks([ms_per_step, e2e["ms"] if e2e else 0.0], dist, dev)
         if e2e:
-            e2e["ms"] = float(t[1])
+            e2e["ms"] = e_max
     if rank != 0:
         if dist is not None:
             dist.barrier()
@@ -293,7 +305,7 @@ def main():
         return 0
 
     flops = w.flops()                       # valid keys only: no credit for skipped work
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(flops, world, ms_per_step)
     attn_ms = statistics.mean(k[2] for k in kernel_ms)
     rope_ms = statistics.mean(k[1] for k in kernel_ms)
     bits_ms = statistics.mean(k[0] for k in kernel_ms)
@@ -339,7 +351,7 @@ def main():
         "gpu_launches": launches * args.steps,
     }
     if e2e:
-        line["e2e"] = {"value": world * flops / (e2e["ms"] * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e["ms"],
+        line["e2e"] = {"value": whole_job_tflops(flops, world, e2e["ms"]), "unit": UNIT, "ms_per_step": e2e["ms"],
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"]}
     if cpu:
         line["cpu_baseline"] = cpu

@@ -503,7 +503,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           issue_qk(tS0, q_lo0, st);
           tc_commit_elect(bar_s_full(0));
           issue_qk(tS1, q_lo1, st);
-          tc_commit_elect(bar_s_full(1));
+          // (test hook: CTA 0 withholds this signal so that the waits downstream run into their limit)
+          if (!(p.fault_inject == 1u && blockIdx.x == 0)) tc_commit_elect(bar_s_full(1));
           tc_commit_elect(bar_kv_empty(st));
           advance();
         }

@@ -37,6 +37,7 @@ struct AttnParams {
   float scale_log2;         // log2(e) / sqrt(head_dim)
   unsigned int* status;     // 0 = fine; written once on a wait time-out
   unsigned long long wait_limit_ns;
+  unsigned int fault_inject;  // test hook: 1 = CTA 0 never publishes S of query tile 1 (exercises the bounded waits)
   unsigned int v_lbo, v_sbo;  // byte offsets of the V (MN-major) shared-memory descriptor
   float* dbg_scores;        // optional: raw QK^T of the first processed key tile, [cta][2][128][128]
   unsigned int dbg_flags;   // diagnostic builds: ablation switches (1 skip QK, 2 skip PV, 4 skip softmax math)

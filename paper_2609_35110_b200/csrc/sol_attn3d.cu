@@ -57,6 +57,7 @@ struct sol_attn3d_plan_s {
   int last_cuda = 0;
   unsigned long long wait_limit_ns = 2000000000ull;
   unsigned int v_lbo = 0, v_sbo = 1024;
+  unsigned int fault_inject = 0;
   float* dbg_scores = nullptr;
   long long* dbg_prof = nullptr;
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -197,6 +198,8 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
       const long v = std::atol(e);
       if (v > 0) p->wait_limit_ns = (unsigned long long)v * 1000000ull;
     }
+    // Test hook for the failure-detection path: a wait inside the kernel is made to run out on purpose.
+    if (const char* e = std::getenv("SOL_ATTN3D_FAULT_INJECT")) p->fault_inject = (unsigned)std::atol(e);
     p->v_lbo = p->head_dim == 128 ? 16384u : 16u;
     p->v_sbo = 1024u;
     if (const char* e = std::getenv("SOL_ATTN3D_DEBUG_V_LBO")) p->v_lbo = (unsigned)std::atol(e);
@@ -404,6 +407,7 @@ int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const 
   ap.wait_limit_ns = p->wait_limit_ns;
   ap.v_lbo = p->v_lbo;
   ap.v_sbo = p->v_sbo;
+  ap.fault_inject = p->fault_inject;
   ap.dbg_scores = p->dbg_scores;
   ap.dbg_prof = p->dbg_prof;
   ap.dbg_flags = 0;
@@ -602,6 +606,7 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
   ap.wait_limit_ns = p->wait_limit_ns;
   ap.v_lbo = p->v_lbo;
   ap.v_sbo = p->v_sbo;
+  ap.fault_inject = 0;
   ap.dbg_scores = nullptr;
   ap.dbg_prof = nullptr;
   ap.dbg_flags = 0;
