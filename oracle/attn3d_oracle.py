@@ -21,6 +21,8 @@ Section 3.4):
       omega = theta ** (-2j/d_a), phi = pos_a * omega and the ADJACENT pair
       (x[o_a+2j], x[o_a+2j+1]) is rotated by phi.  Head dims beyond
       d_T+d_H+d_W pass through.  Prefix tokens and V are never rotated;
+  O3' optional QK normalisation before O3 (fusion group (2) of Section 3.5): RMS norm over head_dim
+      per (token, head) with a learned gain vector, see qk_rms_norm;
   O4  s_ij = <q~_i, k~_j> / sqrt(head_dim) for keys j of the same sequence
       whose key-padding mask is nonzero;
   O5  two-pass softmax in fp64: m_i = max_j s_ij, e_ij = exp(s_ij - m_i),
@@ -115,6 +117,20 @@ def rope_rotate(x: torch.Tensor, pos: torch.Tensor, has_pos: torch.Tensor,
     return out
 
 
+def qk_rms_norm(x: torch.Tensor, gain: torch.Tensor, eps: float) -> torch.Tensor:
+    """QK normalisation, the first half of fusion group (2) in Section 3.5 ("QK normalization with partial
+    RoPE"): RMS norm over head_dim of every (token, head) row, times a learned gain of length head_dim.
+
+        y = x / sqrt(mean_d(x_d^2) + eps) * gain            (fp64, nothing rounded)
+
+    The paper prints no formula; per-head normalisation over head_dim with a gain shared by all heads is
+    the reading taken here (it is the common "QK-norm" of video DiTs).  x: [..., D] fp64, gain: [D].
+    """
+    assert x.dtype == F64
+    ms = (x * x).mean(dim=-1, keepdim=True)
+    return x / torch.sqrt(ms + eps) * gain.to(F64)
+
+
 def attention_rows(q_rot: torch.Tensor, k_rot: torch.Tensor, v: torch.Tensor,
                    valid: Optional[torch.Tensor], head_dim: int,
                    row_chunk: Optional[int] = None) -> torch.Tensor:
@@ -152,7 +168,9 @@ def attn3d_oracle_pos(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
                       rope_dims: Sequence[int], theta: float,
                       key_mask: Optional[torch.Tensor] = None,
                       select: Optional[List[Tuple[int, int, torch.Tensor]]] = None,
-                      origin: Sequence[int] = (0, 0, 0), pairing: str = "adjacent"):
+                      origin: Sequence[int] = (0, 0, 0), pairing: str = "adjacent",
+                      q_gain: Optional[torch.Tensor] = None, k_gain: Optional[torch.Tensor] = None,
+                      norm_eps: float = 1e-6):
     """Internal entry with explicit per-token positions.
 
     q, k, v: [total, heads, D]; pos [total, 3] int64; has_pos [total] bool;
@@ -173,12 +191,16 @@ def attn3d_oracle_pos(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
         a, b = int(cu_seqlens[s]), int(cu_seqlens[s + 1])
         kh = widen(k[a:b, h, :])
         vh = widen(v[a:b, h, :])
+        if k_gain is not None:
+            kh = qk_rms_norm(kh, widen(k_gain), norm_eps)          # normalise, then rotate (Section 3.5 (2))
         k_rot = rope_rotate(kh, pos[a:b], has_pos[a:b], rope_dims, theta, origin, pairing)
         if rows is None:
             rows_t = torch.arange(b - a, dtype=torch.int64)
         else:
             rows_t = torch.as_tensor(rows, dtype=torch.int64)
         qh = widen(q[a:b, h, :][rows_t])
+        if q_gain is not None:
+            qh = qk_rms_norm(qh, widen(q_gain), norm_eps)
         q_rot = rope_rotate(qh, pos[a:b][rows_t], has_pos[a:b][rows_t], rope_dims, theta, origin, pairing)
         valid = None if key_mask is None else (key_mask[a:b].to("cpu") != 0)
         o = attention_rows(q_rot, k_rot, vh, valid, D)
@@ -205,22 +227,29 @@ def layout_positions(seqs: Sequence[Tuple[int, int, int, int]]):
 def attn3d_oracle(q, k, v, seqs: Sequence[Tuple[int, int, int, int]],
                   rope_dims: Sequence[int], theta: float = 10000.0,
                   key_mask: Optional[torch.Tensor] = None,
-                  select: Optional[List[Tuple[int, int, torch.Tensor]]] = None):
+                  select: Optional[List[Tuple[int, int, torch.Tensor]]] = None,
+                  q_gain: Optional[torch.Tensor] = None, k_gain: Optional[torch.Tensor] = None,
+                  norm_eps: float = 1e-6):
     """Public entry: q, k, v [total, heads, D] packed prefix-first per sequence.
 
     A batch of B equal sequences is the packed case with B identical entries
-    in ``seqs`` (batch b starts at token b*N).
+    in ``seqs`` (batch b starts at token b*N).  With q_gain / k_gain given, Q and K are RMS-normalised
+    over head_dim (qk_rms_norm) before the rotary embedding.
     """
     cu, pos, has = layout_positions(seqs)
     assert cu[-1] == q.shape[0], "token count does not match the sequence list"
-    return attn3d_oracle_pos(q, k, v, cu, pos, has, rope_dims, theta, key_mask, select)
+    return attn3d_oracle_pos(q, k, v, cu, pos, has, rope_dims, theta, key_mask, select,
+                             q_gain=q_gain, k_gain=k_gain, norm_eps=norm_eps)
 
 
 def rope_oracle(x, seqs: Sequence[Tuple[int, int, int, int]], rope_dims: Sequence[int],
-                theta: float = 10000.0) -> torch.Tensor:
-    """O0-O3 only: the rotated tensor in fp64, [total, heads, D]."""
+                theta: float = 10000.0, gain: Optional[torch.Tensor] = None, norm_eps: float = 1e-6) -> torch.Tensor:
+    """O0-O3 only: the (optionally RMS-normalised, then) rotated tensor in fp64, [total, heads, D]."""
     _, pos, has = layout_positions(seqs)
-    return rope_rotate(widen(x), pos, has, rope_dims, theta)
+    xw = widen(x)
+    if gain is not None:
+        xw = qk_rms_norm(xw, widen(gain), norm_eps)
+    return rope_rotate(xw, pos, has, rope_dims, theta)
 
 
 def compare(gpu_rows: torch.Tensor, ref_rows: torch.Tensor) -> Tuple[float, float]:

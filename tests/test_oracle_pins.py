@@ -413,3 +413,62 @@ def test_widen_is_exact_and_compare_metrics():
     got = torch.tensor([[3.0, 4.5]], dtype=torch.float32)
     ma, rl = orc.compare(got, ref)
     assert ma == 0.5 and abs(rl - 0.1) < 1e-15
+
+
+# ---------------------------------------------------------------- QK normalisation (Section 3.5, group (2))
+def test_qk_rms_norm_closed_form_and_invariants():
+    # closed form: x = (3, 4): mean square 12.5
+    x = torch.tensor([[3.0, 4.0]], dtype=F64)
+    g = torch.tensor([2.0, -1.0], dtype=F64)
+    y = orc.qk_rms_norm(x, g, 0.0)
+    assert torch.allclose(y, torch.tensor([[6.0 / math.sqrt(12.5), -4.0 / math.sqrt(12.5)]], dtype=F64), atol=1e-15)
+    y = orc.qk_rms_norm(x, g, 3.5)                       # eps sits inside the square root, next to the mean square
+    assert torch.allclose(y, torch.tensor([[6.0 / 4.0, -4.0 / 4.0]], dtype=F64), atol=1e-15)
+    # invariants: unit gain gives unit RMS; positive rescaling of a row changes nothing; rows are independent
+    x = rnd(7, 3, 16, seed=200).to(F64)
+    one = torch.ones(16, dtype=F64)
+    y = orc.qk_rms_norm(x, one, 0.0)
+    assert torch.allclose((y * y).mean(-1), torch.ones(7, 3, dtype=F64), atol=1e-14)
+    assert torch.allclose(orc.qk_rms_norm(x * 37.5, one, 0.0), y, atol=1e-14)
+    x2 = x.clone()
+    x2[2, 1] *= -3.0
+    y2 = orc.qk_rms_norm(x2, one, 0.0)
+    assert torch.equal(y2[:2], y[:2]) and torch.allclose(y2[2, 1], -y[2, 1], atol=1e-15) and torch.equal(y2[2, 0], y[2, 0])
+    # the gain multiplies element-wise after the normalisation
+    g = rnd(16, seed=201).to(F64)
+    assert torch.allclose(orc.qk_rms_norm(x, g, 1e-6), orc.qk_rms_norm(x, one, 1e-6) * g, atol=1e-15)
+
+
+def test_qk_norm_inside_attention_matches_brute_force_and_order():
+    seqs = [(2, 1, 2, 3), (0, 2, 1, 2)]
+    total, heads, D = 8 + 4, 2, 8
+    q, k, v = (rnd(total, heads, D, seed=210 + i) for i in range(3))
+    gq, gk = rnd(D, seed=213).float(), rnd(D, seed=214).float()
+    eps = 1e-3
+    got = orc.attn3d_oracle(q, k, v, seqs, (2, 2, 4), 100.0, None, None, q_gain=gq, k_gain=gk, norm_eps=eps)
+
+    def norm_loops(x, g):
+        x = x.to(F64).tolist()
+        g = g.to(F64).tolist()
+        out = [[[0.0] * D for _ in range(heads)] for _ in range(total)]
+        for t in range(total):
+            for h in range(heads):
+                ms = sum(e * e for e in x[t][h]) / D
+                for d in range(D):
+                    out[t][h][d] = x[t][h][d] / math.sqrt(ms + eps) * g[d]
+        return torch.tensor(out, dtype=F64)
+
+    ref = brute_force(norm_loops(q, gq), norm_loops(k, gk), v, seqs, (2, 2, 4), 100.0)
+    assert torch.allclose(got, ref, atol=1e-12)
+    # normalise-then-rotate, not the other way round: with a non-constant gain the two differ ...
+    rot_then_norm = orc.qk_rms_norm(orc.rope_oracle(k, seqs, (2, 2, 4), 100.0), gk, eps)
+    norm_then_rot = orc.rope_oracle(k, seqs, (2, 2, 4), 100.0, gain=gk, norm_eps=eps)
+    assert not torch.allclose(rot_then_norm, norm_then_rot, atol=1e-3)
+    # ... and with a constant gain they coincide (rotations preserve the mean square)
+    c = torch.full((D,), 1.5)
+    a = orc.qk_rms_norm(orc.rope_oracle(k, seqs, (2, 2, 4), 100.0), c, eps)
+    b = orc.rope_oracle(k, seqs, (2, 2, 4), 100.0, gain=c, norm_eps=eps)
+    assert torch.allclose(a, b, atol=1e-14)
+    # no gains given: the plain path, bit for bit
+    assert torch.equal(orc.attn3d_oracle(q, k, v, seqs, (2, 2, 4), 100.0),
+                       orc.attn3d_oracle(q, k, v, seqs, (2, 2, 4), 100.0, q_gain=None, k_gain=None))
