@@ -138,11 +138,12 @@ def sample_flops(w, sel):
     return fl
 
 
-def run_oracle(w, inp_cpu, sel):
+def run_oracle(w, inp_cpu, sel, q_gain=None, k_gain=None):
     from oracle import attn3d_oracle as orc   # CPU-baseline leg: the one place bench.py runs the oracle
     seqs = [(s.text_len, s.T, s.H, s.W) for s in w.seqs]
     t0 = time.perf_counter()
-    ref = orc.attn3d_oracle(inp_cpu.q, inp_cpu.k, inp_cpu.v, seqs, w.rope_dims, w.theta, inp_cpu.key_mask, sel)
+    ref = orc.attn3d_oracle(inp_cpu.q, inp_cpu.k, inp_cpu.v, seqs, w.rope_dims, w.theta, inp_cpu.key_mask, sel,
+                            q_gain=q_gain, k_gain=k_gain)
     return ref, time.perf_counter() - t0
 
 
@@ -165,6 +166,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--qknorm", action="store_true",
+                    help="time sol_attn3d_forward_qknorm (QK RMS-norm fused into the rotary producer) instead")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -223,6 +226,20 @@ def main():
     out = torch.empty((w.total_tokens, w.heads, w.head_dim), dtype=torch.bfloat16, device=dev)
     B.sol_attn3d_set_profiling(attn.plan, True)
     stream = torch.cuda.current_stream()
+    if args.qknorm:
+        # synthetic learned gains (the paper's checkpoints are not available)
+        gg = torch.Generator(device=dev).manual_seed(w.seed + 77)
+        q_gain = 1.0 + 0.1 * torch.randn(w.head_dim, generator=gg, device=dev, dtype=torch.float32)
+        k_gain = 1.0 + 0.1 * torch.randn(w.head_dim, generator=gg, device=dev, dtype=torch.float32)
+        config["qknorm"] = "RMS-norm over head_dim with synthetic gains, eps 1e-6, fused into the rotary producer"
+
+        def forward(q, k, v, mask, out):
+            B.sol_attn3d_forward_qknorm(attn.plan, q, k, v, out, mask, q_gain, k_gain, 1e-6)
+    else:
+        q_gain = k_gain = None
+
+        def forward(q, k, v, mask, out):
+            attn.forward(q, k, v, mask, out=out)
 
     def barrier():
         if dist is not None:
@@ -230,7 +247,7 @@ def main():
         torch.cuda.synchronize()
 
     for _ in range(warmup):
-        attn.forward(inp.q, inp.k, inp.v, inp.key_mask, out=out)
+        forward(inp.q, inp.k, inp.v, inp.key_mask, out)
     torch.cuda.synchronize()
     if attn.status() != 0:
         raise SystemExit("device reported a wait time-out during warm-up")
@@ -245,7 +262,7 @@ def main():
     barrier()
     ev0.record(stream)
     for _ in range(args.steps):
-        attn.forward(inp.q, inp.k, inp.v, inp.key_mask, out=out)
+        forward(inp.q, inp.k, inp.v, inp.key_mask, out)
     ev1.record(stream)
     barrier()
     total_ms = ev0.elapsed_time(ev1)
@@ -254,7 +271,7 @@ def main():
     # per-kernel durations (CUDA events recorded by the library on the launching stream): a second
     # short loop so that the blocking event read never sits inside the timed region above
     for _ in range(min(args.steps, 5)):
-        attn.forward(inp.q, inp.k, inp.v, inp.key_mask, out=out)
+        forward(inp.q, inp.k, inp.v, inp.key_mask, out)
         kernel_ms.append(B.sol_attn3d_last_forward_ms(attn.plan))
     torch.cuda.synchronize()
     if attn.status() != 0:
@@ -277,7 +294,7 @@ def main():
             dv.copy_(hv, non_blocking=True)
             if dmask is not None:
                 dmask.copy_(hmask, non_blocking=True)
-            attn.forward(dq, dk, dv, dmask, out=out)
+            forward(dq, dk, dv, dmask, out)
             hout.copy_(out, non_blocking=True)
 
         e2e_step()
@@ -322,7 +339,8 @@ def main():
         inp_cpu = wl.Inputs(inp.q.cpu(), inp.k.cpu(), inp.v.cpu(), None if inp.key_mask is None else inp.key_mask.cpu())
         heads_s, rows = cpu_sample_spec(w)
         sel = oracle_sample(w, inp_cpu, heads_s, rows)
-        ref, dt = run_oracle(w, inp_cpu, sel)
+        ref, dt = run_oracle(w, inp_cpu, sel, None if q_gain is None else q_gain.cpu(),
+                             None if k_gain is None else k_gain.cpu())
         cpu = {"value": sample_flops(w, sel) / dt / 1e12, "unit": UNIT, "cores": torch.get_num_threads(),
                "kind": "oracle", "seconds": dt,
                "sample": f"{len(sel)} (seq, head) groups x {len(sel[0][2])} query rows against all keys (fp64)"}

@@ -131,6 +131,29 @@ int sol_attn3d_forward(sol_attn3d_plan_t plan, const void* q, const void* k, con
                        const uint8_t* key_mask, sol_attn3d_stream_t stream);
 
 /*
+ * sol_attn3d_forward with the QK normalisation of the paper's fusion group (2) ("QK normalization with
+ * partial RoPE", Section 3.5) done by the library's producer kernel: every (token, head) row of q and k is
+ * RMS-normalised over head_dim in fp32,  y = x / sqrt(mean(x^2) + eps) * gain,  then rotated, and rounded
+ * to bf16 once.  The paper prints no formula; per-head normalisation with one gain vector per tensor is
+ * the reading taken.  V is not normalised.
+ *   q_gain, k_gain  DEVICE pointers to head_dim fp32 values each (4-byte aligned), both required.
+ *   eps             >= 0.
+ * Everything else as for sol_attn3d_forward.  Errors: as sol_attn3d_forward, plus INVALID_ARG for a NULL gain.
+ */
+int sol_attn3d_forward_qknorm(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out,
+                              const uint8_t* key_mask, const float* q_gain, const float* k_gain, float eps,
+                              sol_attn3d_stream_t stream);
+
+/*
+ * The producer alone (fusion group (2) of Section 3.5: QK normalisation + partial RoPE): q_out / k_out
+ * receive the normalised, rotated bf16 tensors, contiguous [total_tokens, heads, head_dim].  Either tensor
+ * may be NULL together with its output; a tensor that is given needs its gain.  Needs a bound workspace
+ * (tables).  Asynchronous on `stream`.
+ */
+int sol_attn3d_qknorm_rope(sol_attn3d_plan_t plan, const void* q, const void* k, const float* q_gain,
+                           const float* k_gain, float eps, void* q_out, void* k_out, sol_attn3d_stream_t stream);
+
+/*
  * sol_attn3d_forward for callers that must not allocate device memory.  (The paper has no counterpart:
  * this is a deployment variant of the call above, not a step of the method.)
  *

@@ -81,6 +81,10 @@ def _lib():
     lib.sol_attn3d_forward.restype = i32
     lib.sol_attn3d_forward_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sol_attn3d_forward_noalloc.restype = i32
+    lib.sol_attn3d_forward_qknorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp]
+    lib.sol_attn3d_forward_qknorm.restype = i32
+    lib.sol_attn3d_qknorm_rope.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
+    lib.sol_attn3d_qknorm_rope.restype = i32
     lib.sol_attn3d_rope_qk.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sol_attn3d_rope_qk.restype = i32
     lib.sol_attn3d_status.argtypes = [vp]
@@ -198,6 +202,29 @@ def sol_attn3d_forward_noalloc(plan, q: torch.Tensor, k: torch.Tensor, v: torch.
         raise ValueError("device_status must be a CUDA tensor of 4-byte elements")
     _check(_lib().sol_attn3d_forward_noalloc(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask),
                                              _ptr(device_status), _stream(stream)), "sol_attn3d_forward_noalloc")
+
+
+def _check_gain(g: torch.Tensor, head_dim_hint=None):
+    if g is None or not g.is_cuda or g.dtype != torch.float32 or not g.is_contiguous():
+        raise ValueError("gains must be contiguous CUDA float32 tensors of head_dim elements")
+
+
+def sol_attn3d_forward_qknorm(plan, q, k, v, out, key_mask, q_gain: torch.Tensor, k_gain: torch.Tensor, eps: float,
+                              stream=None) -> None:
+    """Forward with QK RMS-norm (gain vectors of head_dim fp32 values) applied before the rotary embedding."""
+    for t in (q, k, v, out):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v, out must be CUDA bf16 tensors")
+    _check_gain(q_gain)
+    _check_gain(k_gain)
+    _check(_lib().sol_attn3d_forward_qknorm(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask), _ptr(q_gain),
+                                            _ptr(k_gain), ctypes.c_float(eps), _stream(stream)),
+           "sol_attn3d_forward_qknorm")
+
+
+def sol_attn3d_qknorm_rope(plan, q, k, q_gain, k_gain, eps: float, q_out, k_out, stream=None) -> None:
+    _check(_lib().sol_attn3d_qknorm_rope(plan, _ptr(q), _ptr(k), _ptr(q_gain), _ptr(k_gain), ctypes.c_float(eps),
+                                         _ptr(q_out), _ptr(k_out), _stream(stream)), "sol_attn3d_qknorm_rope")
 
 
 def sol_attn3d_rope_qk(plan, q, k, q_rot, k_rot, stream=None) -> None:

@@ -50,9 +50,13 @@ __global__ void __launch_bounds__(256) keybits_kernel(const SeqDev* __restrict__
 }
 
 // ---------------------------------------------------------------------------------------------
-// 3D rotary embedding of Q and K.  A thread owns one 16-byte chunk (8 head dims = 4 adjacent
-// pairs) of a token, fetches the four (cos, sin) once and walks over the heads, so the angle
-// lookups are amortised over all heads.  Prefix tokens are copied.  fp32 math, bf16 RNE out.
+// Producer of the attention operands: optional QK RMS-norm (over head_dim, learned gain) followed by
+// the 3D rotary embedding of Q and K -- the paper's fusion group (2), "QK normalization with partial
+// RoPE" (Section 3.5) -- written once as bf16.  A thread owns one 16-byte chunk (8 head dims = 4
+// adjacent pairs) of a token, fetches the four (cos, sin) once and walks over the heads, so the angle
+// lookups are amortised over all heads.  The chunks of one (token, head) row sit in adjacent lanes; the
+// sum of squares is a shuffle reduction over them.  fp32 math throughout, one rounding to bf16 at the
+// end.  Prefix tokens are normalised but not rotated.
 // Layout in: [token][head][D] with element strides (tok, head); out: contiguous.
 // Block: (D/8) x HEADS_PER_PASS threads handle one token per iteration.
 // ---------------------------------------------------------------------------------------------
@@ -60,6 +64,8 @@ struct RopeArgs {
   const __nv_bfloat16* x[2];
   __nv_bfloat16* y[2];
   long long x_tok_stride[2], x_head_stride[2];
+  const float* gain[2];       // [head_dim] each, or nullptr: no normalisation for that tensor
+  float eps;
   const SeqDev* seqs;
   int n_seqs;
   long long total_tokens;
@@ -67,21 +73,18 @@ struct RopeArgs {
   RopeGeom g;
 };
 
-__device__ __forceinline__ uint32_t rotate_pair(uint32_t xy, float2 cs) {
-  const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(&xy);
-  const float xe = __low2float(v), xo = __high2float(v);
-  const float re = xe * cs.x - xo * cs.y;
-  const float ro = xe * cs.y + xo * cs.x;
-  const __nv_bfloat162 r = __floats2bfloat162_rn(re, ro);
-  return *reinterpret_cast<const uint32_t*>(&r);
-}
-
 __global__ void __launch_bounds__(256) rope_qk_kernel(const RopeArgs a) {
-  const int chunks = a.g.head_dim >> 3;          // 16-byte chunks per head row
+  const int chunks = a.g.head_dim >> 3;          // 16-byte chunks per head row (8 or 16: divides the warp)
   const int heads_per_pass = blockDim.x / chunks;
   const int chunk = threadIdx.x % chunks;
   const int hsub = threadIdx.x / chunks;
   const int d1 = a.g.rope[0], d2 = d1 + a.g.rope[1], d3 = d2 + a.g.rope[2];
+  const float inv_d = 1.0f / (float)a.g.head_dim;
+  float gn[2][8];
+#pragma unroll
+  for (int which = 0; which < 2; ++which)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) gn[which][e] = a.gain[which] ? __ldg(a.gain[which] + chunk * 8 + e) : 1.0f;
 
   for (long long tok = blockIdx.x; tok < a.total_tokens; tok += gridDim.x) {
     // which sequence, which grid position
@@ -110,17 +113,42 @@ __global__ void __launch_bounds__(256) rope_qk_kernel(const RopeArgs a) {
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
       if (a.x[which] == nullptr) continue;
+      const bool norm = a.gain[which] != nullptr;
       const __nv_bfloat16* src = a.x[which] + tok * a.x_tok_stride[which] + chunk * 8;
       __nv_bfloat16* dst = a.y[which] + (tok * a.g.heads) * (long long)a.g.head_dim + chunk * 8;
       for (int h = hsub; h < a.g.heads; h += heads_per_pass) {
-        uint4 v = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
-        if (rotate) {
-          v.x = rotate_pair(v.x, cs[0]);
-          v.y = rotate_pair(v.y, cs[1]);
-          v.z = rotate_pair(v.z, cs[2]);
-          v.w = rotate_pair(v.w, cs[3]);
+        // all lanes of a row enter together (the loop bound depends on hsub only)
+        const unsigned lanes = __activemask();
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float f[8];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162*>(&w[u]);
+          f[2 * u] = __low2float(b2);
+          f[2 * u + 1] = __high2float(b2);
         }
-        *reinterpret_cast<uint4*>(dst + (long long)h * a.g.head_dim) = v;
+        if (norm) {
+          float ss = 0.f;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+          for (int off = chunks >> 1; off > 0; off >>= 1) ss += __shfl_xor_sync(lanes, ss, off);
+          const float r = rsqrtf(ss * inv_d + a.eps);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) f[e] = f[e] * r * gn[which][e];
+        }
+        uint32_t o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          float re = f[2 * u], ro = f[2 * u + 1];
+          if (rotate) {
+            re = f[2 * u] * cs[u].x - f[2 * u + 1] * cs[u].y;
+            ro = f[2 * u] * cs[u].y + f[2 * u + 1] * cs[u].x;
+          }
+          const __nv_bfloat162 r2 = __floats2bfloat162_rn(re, ro);
+          o[u] = *reinterpret_cast<const uint32_t*>(&r2);
+        }
+        *reinterpret_cast<uint4*>(dst + (long long)h * a.g.head_dim) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   }

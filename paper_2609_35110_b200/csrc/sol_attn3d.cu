@@ -230,8 +230,12 @@ int encode_map(sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides s
 
 bool aligned16(const void* x) { return (reinterpret_cast<uintptr_t>(x) & 15u) == 0; }
 
-int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, void* kr, cudaStream_t st) {
+int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, void* kr, const float* q_gain,
+                const float* k_gain, float eps, cudaStream_t st) {
   sol::RopeArgs a{};
+  a.gain[0] = q_gain;
+  a.gain[1] = k_gain;
+  a.eps = eps;
   a.x[0] = static_cast<const __nv_bfloat16*>(q);
   a.x[1] = static_cast<const __nv_bfloat16*>(k);
   a.y[0] = static_cast<__nv_bfloat16*>(qr);
@@ -349,11 +353,43 @@ int sol_attn3d_rope_qk(sol_attn3d_plan_t p, const void* q, const void* k, void* 
   if ((q == nullptr) != (q_rot == nullptr) || (k == nullptr) != (k_rot == nullptr)) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (q == nullptr && k == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(q_rot) || !aligned16(k_rot)) return SOL_ATTN3D_ERR_INVALID_ARG;
-  return launch_rope(p, q, k, q_rot, k_rot, static_cast<cudaStream_t>(stream));
+  return launch_rope(p, q, k, q_rot, k_rot, nullptr, nullptr, 0.f, static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
+                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream);
 }
 
 int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
                        const uint8_t* key_mask, sol_attn3d_stream_t stream) {
+  return forward_impl(p, q, k, v, out, key_mask, nullptr, nullptr, 0.f, stream);
+}
+
+int sol_attn3d_forward_qknorm(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
+                              const uint8_t* key_mask, const float* q_gain, const float* k_gain, float eps,
+                              sol_attn3d_stream_t stream) {
+  if (q_gain == nullptr || k_gain == nullptr || !(eps >= 0.f)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q_gain) & 3u) != 0 || (reinterpret_cast<uintptr_t>(k_gain) & 3u) != 0)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  return forward_impl(p, q, k, v, out, key_mask, q_gain, k_gain, eps, stream);
+}
+
+int sol_attn3d_qknorm_rope(sol_attn3d_plan_t p, const void* q, const void* k, const float* q_gain, const float* k_gain,
+                           float eps, void* q_out, void* k_out, sol_attn3d_stream_t stream) {
+  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  if ((q == nullptr) != (q_out == nullptr) || (k == nullptr) != (k_out == nullptr)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (q == nullptr && k == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if ((q != nullptr && q_gain == nullptr) || (k != nullptr && k_gain == nullptr) || !(eps >= 0.f))
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(q_out) || !aligned16(k_out)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  return launch_rope(p, q, k, q_out, k_out, q_gain, k_gain, eps, static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
+                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream) {
   if (p == nullptr || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
@@ -382,7 +418,7 @@ int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const 
   if (p->prof && (e = cudaEventRecord(p->ev[1], st)) != cudaSuccess) return fail_cuda(p, e);
 
   // (2) rotary prologue: Q~, K~ into the workspace
-  int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, st);
+  int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, q_gain, k_gain, eps, st);
   if (rc != SOL_ATTN3D_OK) return rc;
   if (p->prof && (e = cudaEventRecord(p->ev[2], st)) != cudaSuccess) return fail_cuda(p, e);
 
@@ -428,6 +464,7 @@ int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const 
   }
   return SOL_ATTN3D_OK;
 }
+}  // namespace
 
 int sol_attn3d_set_profiling(sol_attn3d_plan_t p, int enable) {
   if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
