@@ -252,6 +252,85 @@ def rope_oracle(x, seqs: Sequence[Tuple[int, int, int, int]], rope_dims: Sequenc
     return rope_rotate(xw, pos, has, rope_dims, theta)
 
 
+# ---------------------------------------------------------------------------------------------
+# Block-sparse variant: the per-step dynamic sparsity of Section 3.4 ("Sparse Attention").
+# This is an approximation of dense attention, so the oracle follows the algorithm step by step.
+# Steps and notation (the paper gives the rule, not the block statistic; readings are marked):
+#   B1  query blocks of QBLK = 256 tokens, KV blocks of KBLK = 128 tokens, per sequence and head  [reading]
+#   B2  block-level score  b_ij = < mean of q~ over block i , mean of k~ over block j > / sqrt(D)    [reading:
+#       mean-pooled, pre-softmax logits; q~, k~ are the rotated operands AS THE KERNEL SEES THEM, i.e.
+#       rounded to bf16, so that both sides take the selection decision on the same numbers]
+#   B3  per query block: mu_i, sigma_i = mean and (population) standard deviation of b_ij over all KV
+#       blocks j; KV block j is selected iff b_ij > mu_i + tau * sigma_i                      [Section 3.4]
+#   B4  safety rails [Section 3.4]: KV blocks holding any prefix token are always selected (exact prefix
+#       sink); query blocks holding any prefix token attend densely.  The block with the largest score
+#       is always kept, so no query block is left without keys.                                [last: reading]
+#   B5  attention as O4-O5 restricted to the keys of the selected blocks (and to valid keys).
+# ---------------------------------------------------------------------------------------------
+QBLK = 256
+KBLK = 128
+
+
+def block_scores(q_rot: torch.Tensor, k_rot: torch.Tensor, head_dim: int) -> torch.Tensor:
+    """B2 for one (sequence, head): q_rot, k_rot [N, D] fp64 -> [ceil(N/256), ceil(N/128)]."""
+    n = q_rot.shape[0]
+    nq, nk = (n + QBLK - 1) // QBLK, (n + KBLK - 1) // KBLK
+    qbar = torch.stack([q_rot[i * QBLK: min(n, (i + 1) * QBLK)].mean(0) for i in range(nq)])
+    kbar = torch.stack([k_rot[j * KBLK: min(n, (j + 1) * KBLK)].mean(0) for j in range(nk)])
+    return (qbar @ kbar.t()) / math.sqrt(head_dim)
+
+
+def block_select(scores: torch.Tensor, tau: float, text_len: int) -> torch.Tensor:
+    """B3-B4: bool [n_qblocks, n_kblocks], True = KV block attended."""
+    mu = scores.mean(dim=1, keepdim=True)
+    sigma = torch.sqrt(((scores - mu) ** 2).mean(dim=1, keepdim=True))
+    sel = scores > mu + tau * sigma
+    sel[torch.arange(scores.shape[0]), scores.argmax(dim=1)] = True
+    if text_len > 0:
+        sel[:, : (text_len + KBLK - 1) // KBLK] = True           # exact prefix KV sink
+        sel[: (text_len + QBLK - 1) // QBLK, :] = True           # prefix queries stay dense
+    return sel
+
+
+def attn3d_sparse_oracle(q, k, v, seqs: Sequence[Tuple[int, int, int, int]], rope_dims: Sequence[int],
+                         theta: float, tau: float, key_mask: Optional[torch.Tensor] = None,
+                         selection: Optional[List[List[torch.Tensor]]] = None,
+                         operand_dtype: torch.dtype = torch.bfloat16):
+    """Block-sparse attention, all rows.  Returns (out fp64 [total, heads, D], selection, scores) where
+    selection[s][h] is the bool block mask used and scores[s][h] the block scores (None when a selection
+    was supplied).  ``selection`` overrides B2-B4 (used to check the attention arithmetic on a given
+    choice of blocks).  ``operand_dtype`` is the rounding applied to q~, k~ before the block statistic.
+    """
+    cu, pos, has = layout_positions(seqs)
+    total, heads, D = q.shape
+    out = torch.zeros(total, heads, v.shape[2], dtype=F64)
+    used, scs = [], []
+    for s, (L, T, H, W) in enumerate(seqs):
+        a, b = cu[s], cu[s + 1]
+        n = b - a
+        used.append([])
+        scs.append([])
+        valid = None if key_mask is None else (key_mask[a:b].to("cpu") != 0)
+        for h in range(heads):
+            q_rot = rope_rotate(widen(q[a:b, h]), pos[a:b], has[a:b], rope_dims, theta)
+            k_rot = rope_rotate(widen(k[a:b, h]), pos[a:b], has[a:b], rope_dims, theta)
+            if selection is None:
+                sc = block_scores(q_rot.to(operand_dtype).to(F64), k_rot.to(operand_dtype).to(F64), D)
+                sel = block_select(sc, tau, L)
+            else:
+                sc, sel = None, selection[s][h]
+            used[-1].append(sel)
+            scs[-1].append(sc)
+            vh = widen(v[a:b, h])
+            for i in range(sel.shape[0]):
+                keys = sel[i].repeat_interleave(KBLK)[:n]
+                if valid is not None:
+                    keys = keys & valid
+                r0, r1 = i * QBLK, min(n, (i + 1) * QBLK)
+                out[a + r0: a + r1, h] = attention_rows(q_rot[r0:r1], k_rot, vh, keys, D)
+    return out, used, scs
+
+
 def compare(gpu_rows: torch.Tensor, ref_rows: torch.Tensor) -> Tuple[float, float]:
     """O6: (max-abs error, relative L2 error) of widened GPU rows against fp64 rows."""
     g = widen(gpu_rows)

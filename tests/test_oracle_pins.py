@@ -472,3 +472,64 @@ def test_qk_norm_inside_attention_matches_brute_force_and_order():
     # no gains given: the plain path, bit for bit
     assert torch.equal(orc.attn3d_oracle(q, k, v, seqs, (2, 2, 4), 100.0),
                        orc.attn3d_oracle(q, k, v, seqs, (2, 2, 4), 100.0, q_gain=None, k_gain=None))
+
+
+# ---------------------------------------------------------------- block-sparse variant (Section 3.4)
+def test_block_select_rule_on_hand_made_scores():
+    # one query block, scores 0..7: mu = 3.5, sigma = sqrt(5.25) = 2.2913
+    sc = torch.arange(8, dtype=F64)[None]
+    assert orc.block_select(sc, 1.0, 0).tolist() == [[False] * 6 + [True, True]]       # > 5.79
+    assert orc.block_select(sc, 1.5, 0).tolist() == [[False] * 7 + [True]]             # > 6.94
+    assert orc.block_select(sc, 0.0, 0).tolist() == [[False] * 4 + [True] * 4]         # > mean
+    # constant scores: sigma = 0, nothing is strictly above the mean; the arg-max block is kept
+    assert int(orc.block_select(torch.ones(1, 5, dtype=F64), 1.0, 0).sum()) == 1
+    # rails: prefix of 130 tokens = KV blocks 0 and 1 always on; query block 0 (holds prefix rows) dense
+    sc = torch.tensor([[0.0, 0, 0, 0, 9.0], [0.0, 0, 0, 0, 9.0]], dtype=F64)
+    sel = orc.block_select(sc, 1.0, 130)
+    assert sel.tolist() == [[True] * 5, [True, True, False, False, True]]
+    # a larger tau never selects more
+    g = torch.Generator().manual_seed(5)
+    sc = torch.randn(6, 40, generator=g, dtype=F64)
+    a, b, c = (orc.block_select(sc, t, 0) for t in (1.0, 1.25, 1.5))
+    assert bool((b <= a).all()) and bool((c <= b).all()) and int(c.sum()) < int(a.sum())
+
+
+def test_block_scores_are_pooled_logits():
+    n, D = 300, 8
+    q, k = rnd(n, D, seed=300).to(F64), rnd(n, D, seed=301).to(F64)
+    sc = orc.block_scores(q, k, D)
+    assert sc.shape == (2, 3)
+    # block (1, 2): query rows 256..299, keys 256..299 (ragged tails average over what is there)
+    want = float(q[256:].mean(0) @ k[256:].mean(0)) / math.sqrt(D)
+    assert abs(float(sc[1, 2]) - want) < 1e-14
+    # pooled logits = mean of the full logit block (bilinearity)
+    full = (q[:256] @ k[128:256].t()) / math.sqrt(D)
+    assert abs(float(sc[0, 1]) - float(full.mean())) < 1e-13
+
+
+def test_sparse_oracle_reduces_to_dense_and_respects_selection():
+    seqs = [(130, 2, 10, 26)]                       # 130 + 520 = 650 tokens: 3 query blocks, 6 KV blocks
+    n = 650
+    q, k, v = (rnd(n, 2, 16, seed=310 + i) for i in range(3))
+    dense = orc.attn3d_oracle(q, k, v, seqs, (4, 6, 6), 10000.0)
+    # everything selected = dense attention
+    full = [[torch.ones(3, 6, dtype=torch.bool) for _ in range(2)]]
+    out, _, _ = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 1.0, selection=full)
+    assert torch.allclose(out, dense, atol=1e-13)
+    # tau = -inf selects everything as well
+    out, used, sc = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, -1e30)
+    assert torch.allclose(out, dense, atol=1e-13) and all(bool(u.all()) for u in used[0])
+    # a real tau: prefix rails hold, prefix query block equals dense, a dropped block's V does not matter
+    out, used, sc = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 0.5)
+    sel = used[0][1]
+    assert bool(sel[:, :2].all()) and bool(sel[0].all()) and not bool(sel.all())
+    assert torch.allclose(out[:256], dense[:256], atol=1e-13)
+    i, j = [(int(a), int(b)) for a, b in zip(*torch.nonzero(~sel, as_tuple=True))][0]
+    v2 = v.clone()
+    v2[j * 128: (j + 1) * 128, 1] = 50.0
+    out2, _, _ = orc.attn3d_sparse_oracle(q, k, v2, seqs, (4, 6, 6), 10000.0, 0.5, selection=used)
+    assert torch.equal(out2[i * 256: (i + 1) * 256, 1], out[i * 256: (i + 1) * 256, 1])
+    # the block statistic is taken on bf16-rounded rotated operands
+    qr = orc.rope_oracle(q, seqs, (4, 6, 6), 10000.0)[:, 1].to(torch.bfloat16).to(F64)
+    kr = orc.rope_oracle(k, seqs, (4, 6, 6), 10000.0)[:, 1].to(torch.bfloat16).to(F64)
+    assert torch.equal(sc[0][1], orc.block_scores(qr, kr, 16))
