@@ -166,6 +166,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sparse-tau", type=float, default=None,
+                    help="time sol_attn3d_forward_sparse with this tau (block-sparse variant of Section 3.4)")
     ap.add_argument("--qknorm", action="store_true",
                     help="time sol_attn3d_forward_qknorm (QK RMS-norm fused into the rotary producer) instead")
     args = ap.parse_args()
@@ -235,6 +237,13 @@ def main():
 
         def forward(q, k, v, mask, out):
             B.sol_attn3d_forward_qknorm(attn.plan, q, k, v, out, mask, q_gain, k_gain, 1e-6)
+    elif args.sparse_tau is not None:
+        q_gain = k_gain = None
+        sparse_ws = torch.empty(B.sol_attn3d_sparse_workspace_bytes(attn.plan), dtype=torch.uint8, device=dev)
+        config["sparse"] = f"block-sparse, tau={args.sparse_tau}, query blocks 256 x KV blocks 128"
+
+        def forward(q, k, v, mask, out):
+            B.sol_attn3d_forward_sparse(attn.plan, q, k, v, out, mask, args.sparse_tau, sparse_ws)
     else:
         q_gain = k_gain = None
 
@@ -322,6 +331,11 @@ def main():
         return 0
 
     flops = w.flops()                       # valid keys only: no credit for skipped work
+    if args.sparse_tau is not None:
+        sel_tiles, all_tiles = B.sol_attn3d_sparse_stats(attn.plan, sparse_ws)
+        config["sparse_density"] = sel_tiles / max(all_tiles, 1)
+        config["dense_equivalent_tflops"] = whole_job_tflops(flops, world, ms_per_step)
+        flops *= sel_tiles / max(all_tiles, 1)          # executed (query block, key tile) pairs only
     value = whole_job_tflops(flops, world, ms_per_step)
     attn_ms = statistics.mean(k[2] for k in kernel_ms)
     rope_ms = statistics.mean(k[1] for k in kernel_ms)
@@ -334,7 +348,7 @@ def main():
     # ------------------------------------------------------------------ CPU baseline (oracle, bounded sample)
     cpu = None
     parity = None
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and world == 1 and args.sparse_tau is None:
         from oracle import attn3d_oracle as orc
         inp_cpu = wl.Inputs(inp.q.cpu(), inp.k.cpu(), inp.v.cpu(), None if inp.key_mask is None else inp.key_mask.cpu())
         heads_s, rows = cpu_sample_spec(w)

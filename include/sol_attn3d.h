@@ -154,6 +154,36 @@ int sol_attn3d_qknorm_rope(sol_attn3d_plan_t plan, const void* q, const void* k,
                            const float* k_gain, float eps, void* q_out, void* k_out, sol_attn3d_stream_t stream);
 
 /*
+ * Block-sparse variant of sol_attn3d_forward: the per-step dynamic sparsity of Section 3.4 ("Sparse
+ * Attention") with its safety rails.  An approximation of dense attention.
+ *   Query blocks of 256 tokens, KV blocks of 128 tokens, per sequence and head.  Block-level score =
+ *   <mean of rotated q over the query block, mean of rotated k over the KV block> / sqrt(head_dim) (the
+ *   paper does not print the block statistic: mean-pooled logits of the bf16 operands are the reading
+ *   taken).  Per query block, mu and sigma are the mean and (population) standard deviation of its scores
+ *   over all KV blocks; a KV block is attended iff score > mu + tau * sigma.  Rails: KV blocks holding a
+ *   prefix token are always attended (exact prefix sink); query blocks holding a prefix token attend
+ *   densely; the best-scoring block is always kept.  The softmax runs over the valid keys of the
+ *   attended blocks only.  The paper's schedule uses tau = 1.0, 1.25, 1.5 for its three refinement steps
+ *   and keeps the first two layers dense (call sol_attn3d_forward for those).
+ *   sparse_ws  caller-owned DEVICE scratch of sol_attn3d_sparse_workspace_bytes(plan) bytes, 256-byte
+ *              aligned (pooled operands, per-CTA key-tile lists, counters); one forward in flight per buffer.
+ * Everything else as for sol_attn3d_forward (the plan's workspace must be bound).  Extra kernels per call:
+ * two pooling kernels and one selection kernel per sequence.
+ */
+size_t sol_attn3d_sparse_workspace_bytes(sol_attn3d_plan_t plan);
+int sol_attn3d_forward_sparse(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out,
+                              const uint8_t* key_mask, float tau, void* sparse_ws, size_t sparse_ws_bytes,
+                              sol_attn3d_stream_t stream);
+/* After the stream has drained: attended / total (query block, KV block) pairs of the last sparse forward
+ * on this scratch (synchronous 16-byte copy). */
+int sol_attn3d_sparse_stats(sol_attn3d_plan_t plan, const void* sparse_ws, long long* selected_tiles,
+                            long long* all_tiles);
+/* After the stream has drained: the ascending KV-block list of one (sequence, head, query block) of the last
+ * sparse forward (synchronous copies; for inspection and tests).  *count receives the full length. */
+int sol_attn3d_sparse_selection(sol_attn3d_plan_t plan, const void* sparse_ws, int seq, int head, int query_block,
+                                int* kv_blocks, int capacity, int* count);
+
+/*
  * sol_attn3d_forward for callers that must not allocate device memory.  (The paper has no counterpart:
  * this is a deployment variant of the call above, not a step of the method.)
  *

@@ -85,6 +85,14 @@ def _lib():
     lib.sol_attn3d_forward_qknorm.restype = i32
     lib.sol_attn3d_qknorm_rope.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
     lib.sol_attn3d_qknorm_rope.restype = i32
+    lib.sol_attn3d_sparse_workspace_bytes.argtypes = [vp]
+    lib.sol_attn3d_sparse_workspace_bytes.restype = ctypes.c_size_t
+    lib.sol_attn3d_forward_sparse.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp]
+    lib.sol_attn3d_forward_sparse.restype = i32
+    lib.sol_attn3d_sparse_stats.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_longlong)]
+    lib.sol_attn3d_sparse_stats.restype = i32
+    lib.sol_attn3d_sparse_selection.argtypes = [vp, vp, i32, i32, i32, ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
+    lib.sol_attn3d_sparse_selection.restype = i32
     lib.sol_attn3d_rope_qk.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sol_attn3d_rope_qk.restype = i32
     lib.sol_attn3d_status.argtypes = [vp]
@@ -202,6 +210,35 @@ def sol_attn3d_forward_noalloc(plan, q: torch.Tensor, k: torch.Tensor, v: torch.
         raise ValueError("device_status must be a CUDA tensor of 4-byte elements")
     _check(_lib().sol_attn3d_forward_noalloc(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask),
                                              _ptr(device_status), _stream(stream)), "sol_attn3d_forward_noalloc")
+
+
+def sol_attn3d_sparse_workspace_bytes(plan) -> int:
+    return int(_lib().sol_attn3d_sparse_workspace_bytes(plan))
+
+
+def sol_attn3d_forward_sparse(plan, q, k, v, out, key_mask, tau: float, sparse_ws: torch.Tensor, stream=None) -> None:
+    """Block-sparse forward (mu + tau*sigma selection of 128-key blocks per 256-row query block)."""
+    for t in (q, k, v, out):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v, out must be CUDA bf16 tensors")
+    _check(_lib().sol_attn3d_forward_sparse(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask),
+                                            ctypes.c_float(tau), _ptr(sparse_ws),
+                                            sparse_ws.numel() * sparse_ws.element_size(), _stream(stream)),
+           "sol_attn3d_forward_sparse")
+
+
+def sol_attn3d_sparse_stats(plan, sparse_ws: torch.Tensor) -> Tuple[int, int]:
+    a, b = ctypes.c_longlong(), ctypes.c_longlong()
+    _check(_lib().sol_attn3d_sparse_stats(plan, _ptr(sparse_ws), ctypes.byref(a), ctypes.byref(b)), "sol_attn3d_sparse_stats")
+    return int(a.value), int(b.value)
+
+
+def sol_attn3d_sparse_selection(plan, sparse_ws: torch.Tensor, seq: int, head: int, query_block: int, capacity: int) -> list:
+    buf = (ctypes.c_int * max(capacity, 1))()
+    n = ctypes.c_int()
+    _check(_lib().sol_attn3d_sparse_selection(plan, _ptr(sparse_ws), seq, head, query_block, buf, capacity,
+                                              ctypes.byref(n)), "sol_attn3d_sparse_selection")
+    return [int(buf[i]) for i in range(min(n.value, capacity))]
 
 
 def _check_gain(g: torch.Tensor, head_dim_hint=None):

@@ -174,8 +174,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int local = (int)blockIdx.x - sq.work_start;
   const int head = local / sq.n_qpairs;
   const int pair = local - head * sq.n_qpairs;
-  const int n_proc = p.ktile_count[si];
-  const int* __restrict__ ktiles = p.ktile_list + sq.ktile_start;
+  // dense: every CTA of a sequence walks the same list of key tiles; block-sparse: each CTA has its own
+  const bool sparse = p.cta_list != nullptr;
+  const int n_proc = sparse ? p.cta_count[blockIdx.x] : p.ktile_count[si];
+  const int* __restrict__ ktiles =
+      sparse ? p.cta_list + sq.sparse_list_start + (long long)local * sq.n_ktiles : p.ktile_list + sq.ktile_start;
   const uint4* __restrict__ keybits = p.keybits + sq.ktile_start;
   const int q_row0 = pair * 256;                       // first local query row of the CTA
   const int tok0 = (int)sq.tok_start;                  // TMA token coordinate of the sequence start

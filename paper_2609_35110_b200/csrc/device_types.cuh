@@ -15,6 +15,7 @@ struct SeqDev {
   int work_start;       // first CTA index of this sequence (CTAs: head-major, query pair fastest)
   int ktile_start;      // offset of this sequence in keybits / ktile_list
   int seq_id;           // index in the caller's order
+  long long sparse_list_start;  // block-sparse mode: offset of this sequence's per-CTA key-tile lists
 };
 
 // Rotary tables: for axis a, entry [tab_off[a] + pos * (rope[a]/2) + j] = (cos, sin)(pos * theta^(-2j/rope[a])).
@@ -32,6 +33,8 @@ struct AttnParams {
   const uint4* keybits;     // [ktile] 128 validity bits (bit b of word w = key 32*w + b of the tile)
   const int* ktile_list;    // per sequence, tiles that hold at least one valid key, ascending
   const int* ktile_count;   // per sequence (schedule order)
+  const int* cta_list;      // block-sparse mode: per CTA, the key tiles it attends (n_ktiles slots each); else nullptr
+  const int* cta_count;     // block-sparse mode: per CTA, how many
   void* out;
   long long o_tok_stride, o_head_stride;  // in elements
   float scale_log2;         // log2(e) / sqrt(head_dim)

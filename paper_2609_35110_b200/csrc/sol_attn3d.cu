@@ -14,6 +14,7 @@
 #include "attn_fwd_sm100.cuh"
 #include "device_types.cuh"
 #include "prologue_kernels.cuh"
+#include "sparse_kernels.cuh"
 
 namespace {
 
@@ -49,6 +50,9 @@ struct sol_attn3d_plan_s {
   size_t off_status = 0, off_tables = 0, off_seqs = 0, off_keybits = 0, off_list = 0, off_count = 0, off_qrot = 0,
          off_krot = 0, ws_bytes = 0;
   unsigned char* ws = nullptr;
+  // block-sparse scratch (passed per call): byte offsets
+  size_t sp_off_stats = 0, sp_off_count = 0, sp_off_qbar = 0, sp_off_kbar = 0, sp_off_list = 0, sp_bytes = 0;
+  std::vector<size_t> sp_qbar_seq, sp_kbar_seq;   // per sequence (schedule order), in floats
 
   EncodeTiledFn encode = nullptr;
   CUtensorMap tm_q{}, tm_k{}, tm_v{};
@@ -159,6 +163,26 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     if (work > 0x7fffffffll) {
       delete p;
       return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;
+    }
+    {
+      // block-sparse mode: per-CTA key-tile lists (n_ktiles slots each), pooled operands per sequence
+      long long list_slots = 0;
+      size_t qbar = 0, kbar = 0;
+      for (SeqDev& q : seqs) {
+        q.sparse_list_start = list_slots;
+        list_slots += (long long)q.n_qpairs * d->heads * q.n_ktiles;
+        p->sp_qbar_seq.push_back(qbar);
+        p->sp_kbar_seq.push_back(kbar);
+        qbar += (size_t)d->heads * q.n_qpairs * d->head_dim;
+        kbar += (size_t)d->heads * q.n_ktiles * d->head_dim;
+      }
+      size_t o = 0;
+      p->sp_off_stats = o; o = align_up(o + 256);
+      p->sp_off_count = o; o = align_up(o + (size_t)work * sizeof(int));
+      p->sp_off_qbar = o;  o = align_up(o + qbar * sizeof(float));
+      p->sp_off_kbar = o;  o = align_up(o + kbar * sizeof(float));
+      p->sp_off_list = o;  o = align_up(o + (size_t)list_slots * sizeof(int));
+      p->sp_bytes = o;
     }
     p->sched = seqs;
     p->total_work = (int)work;
@@ -358,7 +382,8 @@ int sol_attn3d_rope_qk(sol_attn3d_plan_t p, const void* q, const void* k, void* 
 
 namespace {
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
-                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream);
+                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream,
+                 unsigned char* sparse_ws = nullptr, float tau = 0.f);
 }
 
 int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
@@ -375,6 +400,54 @@ int sol_attn3d_forward_qknorm(sol_attn3d_plan_t p, const void* q, const void* k,
   return forward_impl(p, q, k, v, out, key_mask, q_gain, k_gain, eps, stream);
 }
 
+size_t sol_attn3d_sparse_workspace_bytes(sol_attn3d_plan_t p) { return p ? p->sp_bytes : 0; }
+
+int sol_attn3d_forward_sparse(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
+                              const uint8_t* key_mask, float tau, void* sparse_ws, size_t sparse_ws_bytes,
+                              sol_attn3d_stream_t stream) {
+  if (p == nullptr || !(tau == tau)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (sparse_ws == nullptr || sparse_ws_bytes < p->sp_bytes || (reinterpret_cast<uintptr_t>(sparse_ws) % kAlign) != 0)
+    return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  return forward_impl(p, q, k, v, out, key_mask, nullptr, nullptr, 0.f, stream, static_cast<unsigned char*>(sparse_ws), tau);
+}
+
+int sol_attn3d_sparse_stats(sol_attn3d_plan_t p, const void* sparse_ws, long long* selected_tiles, long long* all_tiles) {
+  if (p == nullptr || sparse_ws == nullptr || selected_tiles == nullptr || all_tiles == nullptr)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  unsigned long long h[2] = {0, 0};
+  const cudaError_t e = cudaMemcpy(h, static_cast<const unsigned char*>(sparse_ws) + p->sp_off_stats, sizeof(h),
+                                   cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(p, e);
+  *selected_tiles = (long long)h[0];
+  *all_tiles = (long long)h[1];
+  return SOL_ATTN3D_OK;
+}
+
+int sol_attn3d_sparse_selection(sol_attn3d_plan_t p, const void* sparse_ws, int seq, int head, int query_block,
+                                int* kv_blocks, int capacity, int* count) {
+  if (p == nullptr || sparse_ws == nullptr || count == nullptr || seq < 0 || seq >= p->n_seqs || head < 0 ||
+      head >= p->heads || query_block < 0 || (kv_blocks == nullptr && capacity > 0))
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  const SeqDev* sq = nullptr;
+  for (const SeqDev& c : p->sched)
+    if (c.seq_id == seq) sq = &c;
+  if (sq == nullptr || query_block >= sq->n_qpairs) return SOL_ATTN3D_ERR_INVALID_ARG;
+  const long long local = (long long)head * sq->n_qpairs + query_block;
+  const unsigned char* base = static_cast<const unsigned char*>(sparse_ws);
+  int n = 0;
+  cudaError_t e = cudaMemcpy(&n, base + p->sp_off_count + (size_t)(sq->work_start + local) * sizeof(int), sizeof(int),
+                             cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(p, e);
+  *count = n;
+  const int take = std::min(n, capacity);
+  if (take > 0) {
+    e = cudaMemcpy(kv_blocks, base + p->sp_off_list + (size_t)(sq->sparse_list_start + local * sq->n_ktiles) * sizeof(int),
+                   (size_t)take * sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_cuda(p, e);
+  }
+  return SOL_ATTN3D_OK;
+}
+
 int sol_attn3d_qknorm_rope(sol_attn3d_plan_t p, const void* q, const void* k, const float* q_gain, const float* k_gain,
                            float eps, void* q_out, void* k_out, sol_attn3d_stream_t stream) {
   if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
@@ -389,7 +462,8 @@ int sol_attn3d_qknorm_rope(sol_attn3d_plan_t p, const void* q, const void* k, co
 
 namespace {
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
-                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream) {
+                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream,
+                 unsigned char* sparse_ws, float tau) {
   if (p == nullptr || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
@@ -422,6 +496,35 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   if (rc != SOL_ATTN3D_OK) return rc;
   if (p->prof && (e = cudaEventRecord(p->ev[2], st)) != cudaSuccess) return fail_cuda(p, e);
 
+  // (2b) block-sparse mode: pooled operands, block logits, selection -> per-CTA key-tile lists
+  const int* d_cta_list = nullptr;
+  const int* d_cta_count = nullptr;
+  if (sparse_ws != nullptr) {
+    if ((e = cudaMemsetAsync(sparse_ws + p->sp_off_stats, 0, 256, st)) != cudaSuccess) return fail_cuda(p, e);
+    const __nv_bfloat16* q_rot = reinterpret_cast<const __nv_bfloat16*>(p->ws + p->off_qrot);
+    const __nv_bfloat16* k_rot = reinterpret_cast<const __nv_bfloat16*>(p->ws + p->off_krot);
+    float* qbar = reinterpret_cast<float*>(sparse_ws + p->sp_off_qbar);
+    float* kbar = reinterpret_cast<float*>(sparse_ws + p->sp_off_kbar);
+    int* lists = reinterpret_cast<int*>(sparse_ws + p->sp_off_list);
+    int* counts = reinterpret_cast<int*>(sparse_ws + p->sp_off_count);
+    unsigned long long* stats = reinterpret_cast<unsigned long long*>(sparse_ws + p->sp_off_stats);
+    for (int s = 0; s < p->n_seqs; ++s) {
+      const SeqDev& sq = p->sched[(size_t)s];
+      sol::pool_blocks_kernel<<<sq.n_qpairs * p->heads, p->head_dim, 0, st>>>(q_rot, d_seqs, p->heads, p->head_dim, 256, s,
+                                                                             sq.n_qpairs, qbar + p->sp_qbar_seq[(size_t)s]);
+      sol::pool_blocks_kernel<<<sq.n_ktiles * p->heads, p->head_dim, 0, st>>>(k_rot, d_seqs, p->heads, p->head_dim, 128, s,
+                                                                             sq.n_ktiles, kbar + p->sp_kbar_seq[(size_t)s]);
+      const size_t smem = ((size_t)p->head_dim + (size_t)sq.n_ktiles + 32) * sizeof(float);
+      if (smem > 48 * 1024) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;      // > ~12k key tiles per sequence
+      sol::select_blocks_kernel<<<sq.n_qpairs * p->heads, 256, smem, st>>>(
+          d_seqs, s, p->heads, p->head_dim, tau, qbar + p->sp_qbar_seq[(size_t)s], kbar + p->sp_kbar_seq[(size_t)s],
+          reinterpret_cast<const uint4*>(d_bits), lists, counts, stats);
+      if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+    }
+    d_cta_list = lists;
+    d_cta_count = counts;
+  }
+
   // (3) attention
   if (p->v_cached != v) {
     rc = encode_map(p, &p->tm_v, v, p->sv);
@@ -435,6 +538,8 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.keybits = reinterpret_cast<const uint4*>(d_bits);
   ap.ktile_list = d_list;
   ap.ktile_count = d_count;
+  ap.cta_list = d_cta_list;
+  ap.cta_count = d_cta_count;
   ap.out = out;
   ap.o_tok_stride = p->so.tok;
   ap.o_head_stride = p->so.head;
