@@ -154,6 +154,19 @@ int sol_attn3d_qknorm_rope(sol_attn3d_plan_t plan, const void* q, const void* k,
                            const float* k_gain, float eps, void* q_out, void* k_out, sol_attn3d_stream_t stream);
 
 /*
+ * Rectangular attention: fewer queries than keys.  Serves the reference-KV caching of the paper (section
+ * "Caching Reference Tokens for Reference to Video Generation", paragraph "Reference KV caching mechanism":
+ * after the first step the reference query rows are skipped, text and generated tokens attend to the cached
+ * reference K/V and to each other): every token of the sequence is a key, but only the rows with
+ * query_mask != 0 are computed and written.
+ *   query_mask  DEVICE pointer, uint8 [total_tokens], nonzero = compute this query row.  Rows with 0 are
+ *               not written (`out` keeps what it held); 256-row query blocks without any wanted row cost nothing.
+ * Everything else as for sol_attn3d_forward; wanted rows get bit-identical results.  One extra tiny kernel per call.
+ */
+int sol_attn3d_forward_rect(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out,
+                            const uint8_t* key_mask, const uint8_t* query_mask, sol_attn3d_stream_t stream);
+
+/*
  * Block-sparse variant of sol_attn3d_forward: the per-step dynamic sparsity of Section 3.4 ("Sparse
  * Attention") with its safety rails.  An approximation of dense attention.
  *   Query blocks of 256 tokens, KV blocks of 128 tokens, per sequence and head.  Block-level score =

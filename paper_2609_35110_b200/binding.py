@@ -85,6 +85,8 @@ def _lib():
     lib.sol_attn3d_forward_qknorm.restype = i32
     lib.sol_attn3d_qknorm_rope.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
     lib.sol_attn3d_qknorm_rope.restype = i32
+    lib.sol_attn3d_forward_rect.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sol_attn3d_forward_rect.restype = i32
     lib.sol_attn3d_sparse_workspace_bytes.argtypes = [vp]
     lib.sol_attn3d_sparse_workspace_bytes.restype = ctypes.c_size_t
     lib.sol_attn3d_forward_sparse.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp]
@@ -210,6 +212,17 @@ def sol_attn3d_forward_noalloc(plan, q: torch.Tensor, k: torch.Tensor, v: torch.
         raise ValueError("device_status must be a CUDA tensor of 4-byte elements")
     _check(_lib().sol_attn3d_forward_noalloc(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask),
                                              _ptr(device_status), _stream(stream)), "sol_attn3d_forward_noalloc")
+
+
+def sol_attn3d_forward_rect(plan, q, k, v, out, key_mask, query_mask: torch.Tensor, stream=None) -> None:
+    """Rectangular forward: only rows with query_mask != 0 are computed and written; all tokens are keys."""
+    for t in (q, k, v, out):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v, out must be CUDA bf16 tensors")
+    if not query_mask.is_cuda or query_mask.dtype != torch.uint8 or not query_mask.is_contiguous():
+        raise ValueError("query_mask must be a contiguous CUDA uint8 tensor")
+    _check(_lib().sol_attn3d_forward_rect(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask), _ptr(query_mask),
+                                          _stream(stream)), "sol_attn3d_forward_rect")
 
 
 def sol_attn3d_sparse_workspace_bytes(plan) -> int:

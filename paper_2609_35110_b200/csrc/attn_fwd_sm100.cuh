@@ -174,6 +174,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int local = (int)blockIdx.x - sq.work_start;
   const int head = local / sq.n_qpairs;
   const int pair = local - head * sq.n_qpairs;
+  // rectangular mode: a query pair without a wanted row has nothing to do (CTA-uniform, before any set-up)
+  if (p.pair_needed != nullptr && p.pair_needed[sq.pair_start + pair] == 0) return;
   // dense: every CTA of a sequence walks the same list of key tiles; block-sparse: each CTA has its own
   const bool sparse = p.cta_list != nullptr;
   const int n_proc = sparse ? p.cta_count[blockIdx.x] : p.ktile_count[si];
@@ -333,7 +335,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     if (ok) {
       const int qrow = q_row0 + t * 128 + row;
-      const bool store = qrow < sq.n_tokens;
+      bool store = qrow < sq.n_tokens;
+      if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
       const float inv = (n_proc > 0) ? 1.0f / l : 0.f;
       __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
                            (sq.tok_start + qrow) * p.o_tok_stride + (long long)head * p.o_head_stride;

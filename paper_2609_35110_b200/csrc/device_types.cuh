@@ -15,6 +15,8 @@ struct SeqDev {
   int work_start;       // first CTA index of this sequence (CTAs: head-major, query pair fastest)
   int ktile_start;      // offset of this sequence in keybits / ktile_list
   int seq_id;           // index in the caller's order
+  int pair_start;       // index of this sequence's first query pair in per-pair arrays
+  int pad1;
   long long sparse_list_start;  // block-sparse mode: offset of this sequence's per-CTA key-tile lists
 };
 
@@ -33,6 +35,8 @@ struct AttnParams {
   const uint4* keybits;     // [ktile] 128 validity bits (bit b of word w = key 32*w + b of the tile)
   const int* ktile_list;    // per sequence, tiles that hold at least one valid key, ascending
   const int* ktile_count;   // per sequence (schedule order)
+  const uint8_t* query_mask;   // rectangular mode: uint8 [total_tokens], nonzero = this query row is wanted; else nullptr
+  const uint8_t* pair_needed;  // rectangular mode: per (sequence, query pair), nonzero = at least one wanted row
   const int* cta_list;      // block-sparse mode: per CTA, the key tiles it attends (n_ktiles slots each); else nullptr
   const int* cta_count;     // block-sparse mode: per CTA, how many
   void* out;

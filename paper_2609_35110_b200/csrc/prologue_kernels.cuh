@@ -50,6 +50,26 @@ __global__ void __launch_bounds__(256) keybits_kernel(const SeqDev* __restrict__
 }
 
 // ---------------------------------------------------------------------------------------------
+// Rectangular attention (fewer queries than keys): which 256-row query pairs hold at least one wanted
+// query row.  One warp per (sequence, pair); grid = total pairs.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) pair_needed_kernel(const SeqDev* __restrict__ seqs, int n_seqs,
+                                                         const uint8_t* __restrict__ query_mask,
+                                                         uint8_t* __restrict__ pair_needed) {
+  int s = 0;
+  while (s + 1 < n_seqs && !((int)blockIdx.x >= seqs[s].pair_start && (int)blockIdx.x < seqs[s].pair_start + seqs[s].n_qpairs)) ++s;
+  const SeqDev sq = seqs[s];
+  const int pair = (int)blockIdx.x - sq.pair_start;
+  bool any = false;
+  for (int r = threadIdx.x; r < 256; r += 32) {
+    const int row = pair * 256 + r;
+    if (row < sq.n_tokens && query_mask[sq.tok_start + row] != 0) any = true;
+  }
+  any = __any_sync(0xffffffffu, any);
+  if (threadIdx.x == 0) pair_needed[blockIdx.x] = any ? 1 : 0;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Producer of the attention operands: optional QK RMS-norm (over head_dim, learned gain) followed by
 // the 3D rotary embedding of Q and K -- the paper's fusion group (2), "QK normalization with partial
 // RoPE" (Section 3.5) -- written once as bf16.  A thread owns one 16-byte chunk (8 head dims = 4

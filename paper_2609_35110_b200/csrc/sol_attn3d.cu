@@ -47,8 +47,9 @@ struct sol_attn3d_plan_s {
   int tab_off[3] = {0, 0, 0};
 
   // workspace layout (byte offsets)
-  size_t off_status = 0, off_tables = 0, off_seqs = 0, off_keybits = 0, off_list = 0, off_count = 0, off_qrot = 0,
-         off_krot = 0, ws_bytes = 0;
+  size_t off_status = 0, off_tables = 0, off_seqs = 0, off_keybits = 0, off_list = 0, off_count = 0, off_pairs = 0,
+         off_qrot = 0, off_krot = 0, ws_bytes = 0;
+  int total_pairs = 0;
   unsigned char* ws = nullptr;
   // block-sparse scratch (passed per call): byte offsets
   size_t sp_off_stats = 0, sp_off_count = 0, sp_off_qbar = 0, sp_off_kbar = 0, sp_off_list = 0, sp_bytes = 0;
@@ -153,9 +154,12 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     std::stable_sort(seqs.begin(), seqs.end(), [](const SeqDev& a, const SeqDev& b) { return a.n_tokens > b.n_tokens; });
     long long work = 0;
     long long ktiles = 0;
+    long long pairs = 0;
     for (SeqDev& q : seqs) {
       q.work_start = (int)work;
       q.ktile_start = (int)ktiles;
+      q.pair_start = (int)pairs;
+      pairs += q.n_qpairs;
       work += (long long)q.n_qpairs * d->heads;
       ktiles += q.n_ktiles;
       if (work > 0x7fffffffll) break;
@@ -187,6 +191,7 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     p->sched = seqs;
     p->total_work = (int)work;
     p->total_ktiles = (int)ktiles;
+    p->total_pairs = (int)pairs;
 
     // cos/sin tables, built in fp64 and rounded once to fp32
     size_t n_entries = 0;
@@ -213,6 +218,7 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     p->off_keybits = off; off = align_up(off + (size_t)p->total_ktiles * 16);
     p->off_list = off;    off = align_up(off + (size_t)p->total_ktiles * sizeof(int));
     p->off_count = off;   off = align_up(off + (size_t)p->n_seqs * sizeof(int));
+    p->off_pairs = off;   off = align_up(off + (size_t)p->total_pairs);
     const size_t rot = (size_t)p->total_tokens * p->heads * p->head_dim * 2;
     p->off_qrot = off;    off = align_up(off + rot);
     p->off_krot = off;    off = align_up(off + rot);
@@ -383,7 +389,7 @@ int sol_attn3d_rope_qk(sol_attn3d_plan_t p, const void* q, const void* k, void* 
 namespace {
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
                  const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream,
-                 unsigned char* sparse_ws = nullptr, float tau = 0.f);
+                 unsigned char* sparse_ws = nullptr, float tau = 0.f, const uint8_t* query_mask = nullptr);
 }
 
 int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
@@ -398,6 +404,12 @@ int sol_attn3d_forward_qknorm(sol_attn3d_plan_t p, const void* q, const void* k,
   if ((reinterpret_cast<uintptr_t>(q_gain) & 3u) != 0 || (reinterpret_cast<uintptr_t>(k_gain) & 3u) != 0)
     return SOL_ATTN3D_ERR_INVALID_ARG;
   return forward_impl(p, q, k, v, out, key_mask, q_gain, k_gain, eps, stream);
+}
+
+int sol_attn3d_forward_rect(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
+                            const uint8_t* key_mask, const uint8_t* query_mask, sol_attn3d_stream_t stream) {
+  if (query_mask == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  return forward_impl(p, q, k, v, out, key_mask, nullptr, nullptr, 0.f, stream, nullptr, 0.f, query_mask);
 }
 
 size_t sol_attn3d_sparse_workspace_bytes(sol_attn3d_plan_t p) { return p ? p->sp_bytes : 0; }
@@ -463,7 +475,7 @@ int sol_attn3d_qknorm_rope(sol_attn3d_plan_t p, const void* q, const void* k, co
 namespace {
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
                  const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream,
-                 unsigned char* sparse_ws, float tau) {
+                 unsigned char* sparse_ws, float tau, const uint8_t* query_mask) {
   if (p == nullptr || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
@@ -495,6 +507,15 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, q_gain, k_gain, eps, st);
   if (rc != SOL_ATTN3D_OK) return rc;
   if (p->prof && (e = cudaEventRecord(p->ev[2], st)) != cudaSuccess) return fail_cuda(p, e);
+
+  // (2a) rectangular mode: which query pairs hold a wanted row
+  const uint8_t* d_pair_needed = nullptr;
+  if (query_mask != nullptr) {
+    uint8_t* flags = p->ws + p->off_pairs;
+    sol::pair_needed_kernel<<<p->total_pairs, 32, 0, st>>>(d_seqs, p->n_seqs, query_mask, flags);
+    if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+    d_pair_needed = flags;
+  }
 
   // (2b) block-sparse mode: pooled operands, block logits, selection -> per-CTA key-tile lists
   const int* d_cta_list = nullptr;
@@ -538,6 +559,8 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.keybits = reinterpret_cast<const uint4*>(d_bits);
   ap.ktile_list = d_list;
   ap.ktile_count = d_count;
+  ap.query_mask = query_mask;
+  ap.pair_needed = d_pair_needed;
   ap.cta_list = d_cta_list;
   ap.cta_count = d_cta_count;
   ap.out = out;
