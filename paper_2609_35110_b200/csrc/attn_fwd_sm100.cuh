@@ -4,8 +4,9 @@
 // One CTA = one (sequence, head, pair of 128-row query tiles).  Warp roles:
 //   warps 0-3   softmax / correction / epilogue of query tile 0 (thread = one query row)
 //   warps 4-7   the same for query tile 1
-//   warp  8     TMA producer (one elected lane)
-//   warp  9     tcgen05.mma issuer (one elected lane), owns the TMEM allocation
+//   warp  8     TMA producer (lane 0)
+//   warp  9     tcgen05.mma issuer: the whole warp runs the loop convergently, one elected lane issues each
+//               instruction (descriptors then stay in uniform registers); owns the TMEM allocation
 //   warps 10-11 idle (complete the third warpgroup)
 // The two query tiles ping-pong: while the softmax of one tile runs on the ALUs, the tensor core
 // works on the other tile's QK^T / PV.
@@ -25,24 +26,6 @@
 
 namespace sol {
 
-// Diagnostic builds only: per-role cycle accounting (clock64 deltas accumulated per CTA).
-#ifdef SOL_ATTN3D_DEBUG_HOOKS
-#define SOL_PROF_DECL long long prof_t = 0; long long prof_acc[4] = {0, 0, 0, 0};
-#define SOL_PROF_BEGIN() prof_t = clock64()
-#define SOL_PROF_END(slot) prof_acc[slot] += clock64() - prof_t
-#define SOL_STAMP(slot, cond) if ((cond) && p.dbg_prof != nullptr) p.dbg_prof[(size_t)blockIdx.x * 16 + 16 * gridDim.x + (slot)] = clock64()
-#define SOL_PROF_FLUSH(base, n)                                                        \
-  if (p.dbg_prof != nullptr) {                                                         \
-    for (int pi = 0; pi < (n); ++pi) p.dbg_prof[(size_t)blockIdx.x * 16 + (base) + pi] = prof_acc[pi]; \
-  }
-#else
-#define SOL_STAMP(slot, cond)
-#define SOL_PROF_DECL
-#define SOL_PROF_BEGIN()
-#define SOL_PROF_END(slot)
-#define SOL_PROF_FLUSH(base, n)
-#endif
-
 // Register split after launch (384 threads x 168): the softmax warpgroups take what the third
 // warpgroup (producer, MMA issuer, two idle warps) gives back: (168 - other) * 128 >= (softmax - 168) * 256.
 #ifndef SOL_REGS_SOFTMAX
@@ -51,17 +34,11 @@ namespace sol {
 #ifndef SOL_REGS_OTHER
 #define SOL_REGS_OTHER 64
 #endif
-#ifndef SOL_ATTN_THREADS
-#define SOL_ATTN_THREADS 384
-#endif
-constexpr int kAttnThreads = SOL_ATTN_THREADS;   // 8 softmax warps + producer + MMA issuer (+ 2 idle warps if 384)
+constexpr int kAttnThreads = 384;   // 8 softmax warps + producer + MMA issuer + 2 idle warps (a full third warpgroup)
 
 // Fraction of exponentials evaluated on the FMA pipes instead of the special-function unit: of every
 // kEmuMod adjacent pairs the first kEmuCnt use the polynomial (the MUFU and the tensor core would
 // otherwise need the same number of cycles per tile).
-#ifndef SOL_TURNS
-#define SOL_TURNS 0
-#endif
 #ifndef SOL_EMU_MOD
 #define SOL_EMU_MOD 4
 #endif
@@ -130,7 +107,7 @@ struct AttnSmem {
   static constexpr int kOffQ = 0;
   static constexpr int kOffKV = 2 * kTile;
   static constexpr int kOffBars = kOffKV + kStages * kTile;
-  static constexpr int kNumBars = 1 + 2 * kStages + 9;  // q_full, kv_full/empty, s_full, p_full, o_done, drain, turn[2]
+  static constexpr int kNumBars = 1 + 2 * kStages + 7;  // q_full, kv_full/empty, s_full[2], p_full[2], o_done[2], drain
   static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
   static constexpr int kBytes = kOffTmemPtr + 16;
   static constexpr int kDynBytes = kBytes + 1024;         // slack to align the base to 1024 bytes
@@ -159,7 +136,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   auto bar_p_full = [&](int t) { return bars + 8u * (3 + 2 * L::kStages + t); };
   auto bar_o_done = [&](int t) { return bars + 8u * (5 + 2 * L::kStages + t); };
   const uint32_t bar_drain = bars + 8u * (7 + 2 * L::kStages);
-  auto bar_turn = [&](int t) { return bars + 8u * (8 + 2 * L::kStages + t); };
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + L::kOffTmemPtr);
 
   // A fault recorded by an earlier CTA stops later ones at the door (read once, CTA-uniform).
@@ -198,8 +174,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(bar_o_done(t), 1);
     }
     mbar_init(bar_drain, 1);
-    mbar_init(bar_turn(0), 4);
-    mbar_init(bar_turn(1), 4);
     fence_mbar_init();
     prefetch_tensormap(&tm_q);
     prefetch_tensormap(&tm_k);
@@ -216,9 +190,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   if (warp < 8) {
     // =========================================================== softmax / correction / epilogue
-#if SOL_ATTN_THREADS == 384
     setmaxnreg_inc<SOL_REGS_SOFTMAX>();
-#endif
     const int t = warp >> 2;
     const int wq = warp & 3;
     const int row = wq * 32 + lane;
@@ -229,31 +201,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     float m_ref = -CUDART_INF_F;
     float l = 0.f;
     bool ok = true;
-    SOL_PROF_DECL
 
     for (int i = 0; i < n_proc; ++i) {
       const int jt = __ldg(&ktiles[i]);
       const uint4 kb = __ldg(&keybits[jt]);
-      SOL_PROF_BEGIN();
       ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full(t), i & 1, limit));
       if (!ok) break;
       tc_fence_after();
-      SOL_PROF_END(0);
-      SOL_STAMP(1, t == 0 && warp == 0 && lane == 0 && i == 10);
-      SOL_PROF_BEGIN();
 
       uint32_t r[128];
 #pragma unroll
       for (int cch = 0; cch < 4; ++cch) tmem_ld32(tS + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[cch * 32]));
       tmem_wait_ld();
-      SOL_PROF_END(1);
-      SOL_STAMP(2, t == 0 && warp == 0 && lane == 0 && i == 10);
 
-      if (p.dbg_scores != nullptr && i == 0) {
-        float* dst = p.dbg_scores + ((size_t)blockIdx.x * 2 + t) * 128 * 128 + (size_t)row * 128;
-#pragma unroll
-        for (int cc = 0; cc < 128; ++cc) dst[cc] = __uint_as_float(r[cc]);
-      }
 
       const bool mixed = (kb.x & kb.y & kb.z & kb.w) != 0xffffffffu;
       if (mixed) {
@@ -264,20 +224,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (((w >> (cc & 31)) & 1u) == 0) r[cc] = __float_as_uint(-CUDART_INF_F);
         }
       }
-#if SOL_TURNS
-      // The two softmax warpgroups take turns in the arithmetic section: a tile's softmax then has the
-      // issue slots and the special-function unit to itself and finishes sooner, which shortens the
-      // S -> P -> PV -> QK chain of that tile; the other tile's MMAs run meanwhile.
-      if (t == 0) {
-        if (i > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_turn(1), (i - 1) & 1, limit));
-      } else {
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_turn(0), i & 1, limit));
-      }
-      if (!ok) break;
-#endif
       if (i == 0) m_ref = row_max128(r);
-
-      SOL_PROF_BEGIN();
       // Speculative pass: exponentials against the current reference maximum, no row maximum taken.
       // All terms are positive, so a row sum <= 2^8 proves that every term is <= 2^8: the reference
       // is still good enough (the result does not depend on which reference is used, only overflow
@@ -311,22 +258,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       l += tile_sum;
-#if SOL_TURNS
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_turn(t));
-#endif
-      SOL_PROF_END(2);
-      SOL_STAMP(3, t == 0 && warp == 0 && lane == 0 && i == 10);
-      SOL_PROF_BEGIN();
       tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
       tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_p_full(t));
-      SOL_PROF_END(3);
-      SOL_STAMP(4, t == 0 && warp == 0 && lane == 0 && i == 10);
     }
-    if (lane == 0 && wq == 0) { SOL_PROF_FLUSH(t * 4, 4) }
 
     // ---- epilogue: O / l -> bf16 -> global (rows beyond the sequence are not stored)
     if (ok && n_proc > 0) {
@@ -366,9 +303,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);
     }
   } else {
-#if SOL_ATTN_THREADS == 384
     setmaxnreg_dec<SOL_REGS_OTHER>();
-#endif
   }
   if (warp == 8) {
     // =========================================================== TMA producer
@@ -387,14 +322,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
           if (!mbar_wait(bar_kv_empty(stage), par ^ 1u, limit)) { ok = false; break; }
-#ifdef SOL_ATTN3D_DEBUG_HOOKS
-          if ((p.dbg_flags & 8u) != 0 && i >= 3) {       // ablation: no K/V traffic after the ring is primed
-            mbar_arrive(bar_kv_full(stage));
-            ++it;
-            if (++stage == (uint32_t)L::kStages) { stage = 0; par ^= 1u; }
-            continue;
-          }
-#endif
           mbar_arrive_expect_tx(bar_kv_full(stage), L::kTile);
           const CUtensorMap* tm = kv ? &tm_v : &tm_k;
 #pragma unroll
@@ -421,7 +348,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, true);
       bool ok = true;
-      SOL_PROF_DECL
       const uint32_t v_lbo = p.v_lbo, v_sbo = p.v_sbo;
       // descriptor words: only the low word (address) moves inside the loop
       const uint32_t hi_k = smem_desc_hi_sw128(1024);
@@ -455,55 +381,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
       if (n_proc > 0) {
         ok = mbar_wait_warp(bar_q_full, 0, limit) && mbar_wait_warp(bar_kv_full(st), ph, limit);
-#if defined(SOL_ATTN3D_DEBUG_HOOKS) && !defined(SOL_NO_PROF)
-        if (ok && p.dbg_prof != nullptr && mbar_wait_warp(bar_kv_full(1), 0, limit)) {
-          // latency probes on the drain barrier: 32 QK-type MMAs, then 32 PV-type MMAs, each + commit
-          tc_fence_after();
-          long long t0 = clock64();
-          issue_qk(tS0, q_lo0, 0); issue_qk(tS1, q_lo1, 0); issue_qk(tS0, q_lo0, 0); issue_qk(tS1, q_lo1, 0);
-          tc_commit_elect(bar_drain);
-          while (!mbar_test_wait(bar_drain, 0)) {}
-          long long t1 = clock64();
-          p.dbg_prof[(size_t)blockIdx.x * 16 + 12] = t1 - t0;
-          t0 = clock64();
-          issue_pv(tO0, tS0, 1, false); issue_pv(tO1, tS1, 1, false); issue_pv(tO0, tS0, 1, true); issue_pv(tO1, tS1, 1, true);
-          tc_commit_elect(bar_drain);
-          while (!mbar_test_wait(bar_drain, 1)) {}
-          t1 = clock64();
-          p.dbg_prof[(size_t)blockIdx.x * 16 + 13] = t1 - t0;
-          {
-            // primitive costs with an idle pipe
-            t0 = clock64();
-#pragma unroll
-            for (int q = 0; q < 16; ++q) tc_fence_after();
-            t1 = clock64();
-            p.dbg_prof[(size_t)blockIdx.x * 16 + 14] = t1 - t0;
-            t0 = clock64();
-            bool any = false;
-#pragma unroll
-            for (int q = 0; q < 16; ++q) any |= mbar_try_wait(bar_q_full, 0);
-            t1 = clock64();
-            p.dbg_prof[(size_t)blockIdx.x * 16 + 15] = (t1 - t0) + (any ? 0 : 1);
-            // fence cost with a busy pipe: 16 MMAs queued, then 16 fences
-            issue_qk(tS0, q_lo0, 0); issue_qk(tS1, q_lo1, 0);
-            t0 = clock64();
-#pragma unroll
-            for (int q = 0; q < 16; ++q) tc_fence_after();
-            t1 = clock64();
-            p.dbg_prof[(size_t)blockIdx.x * 16 + 8] = t1 - t0;     // overwritten later by the loop stats unless kept
-            t0 = clock64();
-#pragma unroll
-            for (int q = 0; q < 8; ++q) tc_commit_elect(bar_turn(0));     // spare barrier (count 4): arrivals only
-            t1 = clock64();
-            p.dbg_prof[(size_t)blockIdx.x * 16 + 9] = t1 - t0;
-          }
-          // leave the drain barrier in phase 0 for the error path
-          tc_commit_elect(bar_drain);
-          while (!mbar_test_wait(bar_drain, 0)) {}
-          tc_commit_elect(bar_drain);
-          while (!mbar_test_wait(bar_drain, 1)) {}
-        }
-#endif
         if (ok) {
           tc_fence_after();
           issue_qk(tS0, q_lo0, st);
@@ -520,32 +397,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const bool more = i + 1 < n_proc;
           const uint32_t k_st = st, k_ph = ph;
           if (more) advance();
-          SOL_PROF_BEGIN();
           if (!mbar_wait_warp(bar_kv_full(v_st), v_ph, limit)) { ok = false; break; }
-          SOL_PROF_END(0);
-          SOL_PROF_BEGIN();
-          SOL_STAMP(9, i == 10);
           if (!mbar_wait_warp(bar_p_full(0), i & 1, limit)) { ok = false; break; }
-          SOL_PROF_END(1);
-          SOL_STAMP(5, i == 10);
           tc_fence_after();
           issue_pv(tO0, tS0, v_st, i > 0);
           tc_commit_elect(bar_o_done(0));
-          SOL_STAMP(6, i == 10);
           if (more) {
-            SOL_PROF_BEGIN();
             if (!mbar_wait_warp(bar_kv_full(k_st), k_ph, limit)) { ok = false; break; }
-            SOL_PROF_END(2);
             tc_fence_after();
             issue_qk(tS0, q_lo0, k_st);
             tc_commit_elect(bar_s_full(0));
-            SOL_STAMP(0, i == 9);      // S0(10) requested
-            SOL_STAMP(7, i == 10);     // S0(11) requested
           }
-          SOL_PROF_BEGIN();
           if (!mbar_wait_warp(bar_p_full(1), i & 1, limit)) { ok = false; break; }
-          SOL_STAMP(8, i == 10);
-          SOL_PROF_END(3);
           tc_fence_after();
           issue_pv(tO1, tS1, v_st, i > 0);
           tc_commit_elect(bar_o_done(1));
@@ -557,9 +420,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
         }
       }
-#if defined(SOL_ATTN3D_DEBUG_HOOKS) && !defined(SOL_NO_PROF)
-      if (p.dbg_prof != nullptr) { p.dbg_prof[(size_t)blockIdx.x * 16 + 10] = prof_acc[1]; p.dbg_prof[(size_t)blockIdx.x * 16 + 11] = prof_acc[3]; }
-#endif
       if (!ok) {
         if (lane == 0) atomicCAS(p.status, 0u, kStatusTimeoutMma);
         // tensor-core work already issued must finish before tensor memory is released

@@ -46,9 +46,6 @@ struct AttnParams {
   unsigned long long wait_limit_ns;
   unsigned int fault_inject;  // test hook: 1 = CTA 0 never publishes S of query tile 1 (exercises the bounded waits)
   unsigned int v_lbo, v_sbo;  // byte offsets of the V (MN-major) shared-memory descriptor
-  float* dbg_scores;        // optional: raw QK^T of the first processed key tile, [cta][2][128][128]
-  unsigned int dbg_flags;   // diagnostic builds: ablation switches (1 skip QK, 2 skip PV, 4 skip softmax math)
-  long long* dbg_prof;      // optional (diagnostic builds): per-CTA cycle counters, [cta][16]
 };
 
 enum : unsigned int {

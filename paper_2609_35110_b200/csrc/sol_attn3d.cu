@@ -63,8 +63,6 @@ struct sol_attn3d_plan_s {
   unsigned long long wait_limit_ns = 2000000000ull;
   unsigned int v_lbo = 0, v_sbo = 1024;
   unsigned int fault_inject = 0;
-  float* dbg_scores = nullptr;
-  long long* dbg_prof = nullptr;
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
   bool prof = false, prof_valid = false, prof_bits = false;
 };
@@ -232,8 +230,6 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     if (const char* e = std::getenv("SOL_ATTN3D_FAULT_INJECT")) p->fault_inject = (unsigned)std::atol(e);
     p->v_lbo = p->head_dim == 128 ? 16384u : 16u;
     p->v_sbo = 1024u;
-    if (const char* e = std::getenv("SOL_ATTN3D_DEBUG_V_LBO")) p->v_lbo = (unsigned)std::atol(e);
-    if (const char* e = std::getenv("SOL_ATTN3D_DEBUG_V_SBO")) p->v_sbo = (unsigned)std::atol(e);
   } catch (const std::bad_alloc&) {
     delete p;
     return SOL_ATTN3D_ERR_NO_MEMORY;
@@ -572,12 +568,6 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.v_lbo = p->v_lbo;
   ap.v_sbo = p->v_sbo;
   ap.fault_inject = p->fault_inject;
-  ap.dbg_scores = p->dbg_scores;
-  ap.dbg_prof = p->dbg_prof;
-  ap.dbg_flags = 0;
-#ifdef SOL_ATTN3D_DEBUG_HOOKS
-  if (const char* e = std::getenv("SOL_ATTN3D_DEBUG_FLAGS")) ap.dbg_flags = (unsigned)std::atol(e);
-#endif
   if (p->head_dim == 128) {
     sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(p->tm_q, p->tm_k,
                                                                                                       p->tm_v, ap);
@@ -772,9 +762,6 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
   ap.v_lbo = p->v_lbo;
   ap.v_sbo = p->v_sbo;
   ap.fault_inject = 0;
-  ap.dbg_scores = nullptr;
-  ap.dbg_prof = nullptr;
-  ap.dbg_flags = 0;
   if (p->head_dim == 128) {
     sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(tm_q, tm_k, tm_v,
                                                                                                       ap);
@@ -824,20 +811,5 @@ int sol_attn3d_destroy(sol_attn3d_plan_t p) {
   return SOL_ATTN3D_OK;
 }
 
-#ifdef SOL_ATTN3D_DEBUG_HOOKS
-// Diagnostic build only: raw QK^T of the first key tile of every CTA is written to `dev_buf`
-// ([total_work][2][128][128] floats).
-int sol_attn3d_debug_dump_scores(sol_attn3d_plan_t p, float* dev_buf) {
-  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
-  p->dbg_scores = dev_buf;
-  return SOL_ATTN3D_OK;
-}
-int sol_attn3d_debug_prof(sol_attn3d_plan_t p, long long* dev_buf) {
-  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
-  p->dbg_prof = dev_buf;
-  return SOL_ATTN3D_OK;
-}
-int sol_attn3d_debug_total_work(sol_attn3d_plan_t p) { return p ? p->total_work : 0; }
-#endif
 
 }  // extern "C"
