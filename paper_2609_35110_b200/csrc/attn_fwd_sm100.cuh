@@ -265,39 +265,61 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_arrive(bar_p_full(t));
     }
 
-    // ---- epilogue: O / l -> bf16 -> global (rows beyond the sequence are not stored)
+    // ---- epilogue: O / l -> bf16 -> shared-memory staging -> coalesced 16-byte stores
+    //      (rows beyond the sequence, or not wanted by the query mask, are not stored)
     if (ok && n_proc > 0) {
       ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (n_proc - 1) & 1, limit));
       if (ok) tc_fence_after();
     }
-    if (ok) {
-      const int qrow = q_row0 + t * 128 + row;
-      bool store = qrow < sq.n_tokens;
-      if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
-      const float inv = (n_proc > 0) ? 1.0f / l : 0.f;
-      __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
-                           (sq.tok_start + qrow) * p.o_tok_stride + (long long)head * p.o_head_stride;
+    if (ok && n_proc > 0) {
+      // Each warp stages its 32 rows (bf16, XOR-swizzled 16-byte chunks) in the part of the query tile's
+      // shared memory that belongs to those rows -- every MMA that read it has completed -- and then writes
+      // them out with D/8 lanes per row, so every store instruction covers whole contiguous rows.
+      constexpr int kRowBytes = D * 2;
+      constexpr int kLanesPerRow = D / 8;
+      uint8_t* stage = smem + L::kOffQ + t * L::kTile + wq * 32 * kRowBytes;
+      const float inv = 1.0f / l;
 #pragma unroll
       for (int cch = 0; cch < D / 32; ++cch) {
         uint32_t o[32];
-        if (n_proc > 0) {
-          tmem_ld32(tO + cch * 32, o);
-          tmem_wait_ld();
-        } else {
+        tmem_ld32(tO + cch * 32, o);
+        tmem_wait_ld();
 #pragma unroll
-          for (int cc = 0; cc < 32; ++cc) o[cc] = 0u;
+        for (int v4 = 0; v4 < 4; ++v4) {
+          uint4 w;
+          w.x = pack_bf16x2(__uint_as_float(o[8 * v4 + 0]) * inv, __uint_as_float(o[8 * v4 + 1]) * inv);
+          w.y = pack_bf16x2(__uint_as_float(o[8 * v4 + 2]) * inv, __uint_as_float(o[8 * v4 + 3]) * inv);
+          w.z = pack_bf16x2(__uint_as_float(o[8 * v4 + 4]) * inv, __uint_as_float(o[8 * v4 + 5]) * inv);
+          w.w = pack_bf16x2(__uint_as_float(o[8 * v4 + 6]) * inv, __uint_as_float(o[8 * v4 + 7]) * inv);
+          const int ch = cch * 4 + v4;
+          *reinterpret_cast<uint4*>(stage + lane * kRowBytes + ((ch ^ (lane & (kLanesPerRow - 1))) << 4)) = w;
         }
+      }
+      __syncwarp();
+      const int ch = lane % kLanesPerRow;
+#pragma unroll 4
+      for (int r0 = 0; r0 < 32; r0 += 32 / kLanesPerRow) {
+        const int rr = r0 + lane / kLanesPerRow;
+        const int qrow = q_row0 + t * 128 + wq * 32 + rr;
+        bool store = qrow < sq.n_tokens;
+        if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
+        const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * kRowBytes + ((ch ^ (rr & (kLanesPerRow - 1))) << 4));
         if (store) {
-#pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(o[8 * v4 + 0]) * inv, __uint_as_float(o[8 * v4 + 1]) * inv);
-            w.y = pack_bf16x2(__uint_as_float(o[8 * v4 + 2]) * inv, __uint_as_float(o[8 * v4 + 3]) * inv);
-            w.z = pack_bf16x2(__uint_as_float(o[8 * v4 + 4]) * inv, __uint_as_float(o[8 * v4 + 5]) * inv);
-            w.w = pack_bf16x2(__uint_as_float(o[8 * v4 + 6]) * inv, __uint_as_float(o[8 * v4 + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + cch * 32 + v4 * 8) = w;
-          }
+          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (sq.tok_start + qrow) * p.o_tok_stride +
+                               (long long)head * p.o_head_stride + ch * 8;
+          *reinterpret_cast<uint4*>(dst) = w;
         }
+      }
+    } else if (ok) {
+      // no key tile at all (every key of the sequence masked): the row is defined as zero
+      const int qrow = q_row0 + t * 128 + row;
+      bool store = qrow < sq.n_tokens;
+      if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
+      if (store) {
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
+                             (sq.tok_start + qrow) * p.o_tok_stride + (long long)head * p.o_head_stride;
+#pragma unroll
+        for (int c16 = 0; c16 < D / 8; ++c16) *reinterpret_cast<uint4*>(dst + c16 * 8) = make_uint4(0u, 0u, 0u, 0u);
       }
     } else if (lane == 0) {
       atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);
