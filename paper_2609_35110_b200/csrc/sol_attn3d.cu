@@ -528,12 +528,13 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
     for (int s = 0; s < p->n_seqs; ++s) {
       const SeqDev& sq = p->sched[(size_t)s];
       sol::pool_blocks_kernel<<<sq.n_qpairs * p->heads, p->head_dim, 0, st>>>(q_rot, d_seqs, p->heads, p->head_dim, 256, s,
-                                                                             sq.n_qpairs, qbar + p->sp_qbar_seq[(size_t)s]);
+                                                                             sq.n_qpairs, 0, qbar + p->sp_qbar_seq[(size_t)s]);
       sol::pool_blocks_kernel<<<sq.n_ktiles * p->heads, p->head_dim, 0, st>>>(k_rot, d_seqs, p->heads, p->head_dim, 128, s,
-                                                                             sq.n_ktiles, kbar + p->sp_kbar_seq[(size_t)s]);
-      const size_t smem = ((size_t)p->head_dim + (size_t)sq.n_ktiles + 32) * sizeof(float);
-      if (smem > 48 * 1024) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;      // > ~12k key tiles per sequence
-      sol::select_blocks_kernel<<<sq.n_qpairs * p->heads, 256, smem, st>>>(
+                                                                             sq.n_ktiles, 1, kbar + p->sp_kbar_seq[(size_t)s]);
+      const size_t smem = (size_t)sol::kSelectRows * ((size_t)p->head_dim + (size_t)sq.n_ktiles) * sizeof(float);
+      if (smem > 48 * 1024) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;      // > ~1400 key tiles (180k tokens) per sequence
+      const int groups = (sq.n_qpairs + sol::kSelectRows - 1) / sol::kSelectRows;
+      sol::select_blocks_kernel<<<groups * p->heads, 256, smem, st>>>(
           d_seqs, s, p->heads, p->head_dim, tau, qbar + p->sp_qbar_seq[(size_t)s], kbar + p->sp_kbar_seq[(size_t)s],
           reinterpret_cast<const uint4*>(d_bits), lists, counts, stats);
       if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);

@@ -12,12 +12,15 @@
 namespace sol {
 
 // ---------------------------------------------------------------------------------------------
-// Mean of the rotated operand over a block of tokens, per head: out[head][block][d] (fp32).
+// Mean of the rotated operand over a block of tokens, per head (fp32).
 // x: rotated bf16 [token][head][D] contiguous.  One CTA per (sequence, head, block); thread d sums
 // column d over the block's tokens in order.  blockDim = D.
+// Output layout: out[head][block][d], or transposed out[head][d][block] (so that the selection kernel
+// reads the pooled keys with consecutive threads on consecutive blocks).
 // ---------------------------------------------------------------------------------------------
 __global__ void pool_blocks_kernel(const __nv_bfloat16* __restrict__ x, const SeqDev* __restrict__ seqs, int heads,
-                                   int head_dim, int block_tokens, int seq_index, int n_blocks, float* __restrict__ out) {
+                                   int head_dim, int block_tokens, int seq_index, int n_blocks, int transposed,
+                                   float* __restrict__ out) {
   const SeqDev sq = seqs[seq_index];
   const int blk = blockIdx.x % n_blocks;
   const int head = blockIdx.x / n_blocks;
@@ -27,101 +30,108 @@ __global__ void pool_blocks_kernel(const __nv_bfloat16* __restrict__ x, const Se
   const __nv_bfloat16* src = x + ((sq.tok_start + t0) * heads + head) * (long long)head_dim + d;
   float acc = 0.f;
   for (int t = t0; t < t1; ++t, src += (long long)heads * head_dim) acc += __bfloat162float(*src);
-  out[((long long)head * n_blocks + blk) * head_dim + d] = acc / (float)(t1 - t0);
+  const float mean = acc / (float)(t1 - t0);
+  if (transposed) out[((long long)head * head_dim + d) * n_blocks + blk] = mean;
+  else            out[((long long)head * n_blocks + blk) * head_dim + d] = mean;
 }
 
 // ---------------------------------------------------------------------------------------------
-// One CTA per attention work item (sequence, head, query block): block logits against every KV
-// block, mean and standard deviation, threshold, rails, ascending list of selected key tiles.
+// One CTA per (sequence, head, group of 8 query blocks): block logits of the 8 query blocks against
+// every KV block (the pooled keys are read once per group), then one warp per query block: mean and
+// standard deviation, threshold, rails, ascending list of selected key tiles.
 // Key tiles without any valid key (key-padding mask, see keybits) are never listed.
+// qbar: [head][query block][d]; kbar_t: [head][d][KV block].  blockDim = 256 (8 warps).
 // ---------------------------------------------------------------------------------------------
+constexpr int kSelectRows = 8;
+
 __global__ void __launch_bounds__(256) select_blocks_kernel(const SeqDev* __restrict__ seqs, int seq_index, int heads,
                                                             int head_dim, float tau, const float* __restrict__ qbar,
-                                                            const float* __restrict__ kbar,
+                                                            const float* __restrict__ kbar_t,
                                                             const uint4* __restrict__ keybits, int* __restrict__ cta_list,
                                                             int* __restrict__ cta_count,
                                                             unsigned long long* __restrict__ stats) {
-  extern __shared__ float sm[];                     // [head_dim] pooled query + [n_ktiles] scores + reduction scratch
+  extern __shared__ float sm[];                     // [8][head_dim] pooled queries + [8][n_ktiles] scores
   const SeqDev sq = seqs[seq_index];
-  const int local = blockIdx.x;                     // head-major, query block fastest (= CTA order of the attention kernel)
-  const int head = local / sq.n_qpairs;
-  const int qb = local - head * sq.n_qpairs;
+  const int groups = (sq.n_qpairs + kSelectRows - 1) / kSelectRows;
+  const int head = blockIdx.x / groups;
+  const int qb0 = (blockIdx.x - head * groups) * kSelectRows;
+  const int rows = min(kSelectRows, sq.n_qpairs - qb0);
   const int nk = sq.n_ktiles;
   float* q_s = sm;
-  float* sc = sm + head_dim;
-  float* red = sc + nk;
+  float* sc = sm + kSelectRows * head_dim;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
 
-  for (int d = tid; d < head_dim; d += blockDim.x) q_s[d] = qbar[((long long)head * sq.n_qpairs + qb) * head_dim + d];
+  for (int idx = tid; idx < kSelectRows * head_dim; idx += blockDim.x) {
+    const int r = idx / head_dim, d = idx - r * head_dim;
+    q_s[idx] = r < rows ? qbar[((long long)head * sq.n_qpairs + qb0 + r) * head_dim + d] : 0.f;
+  }
   __syncthreads();
   const float inv_sqrt_d = rsqrtf((float)head_dim);
+  const float* kt = kbar_t + (long long)head * head_dim * nk;
   for (int kb = tid; kb < nk; kb += blockDim.x) {
-    const float* kr = kbar + ((long long)head * nk + kb) * head_dim;
-    float acc = 0.f;
-    for (int d = 0; d < head_dim; ++d) acc = fmaf(q_s[d], __ldg(kr + d), acc);
-    sc[kb] = acc * inv_sqrt_d;
+    float acc[kSelectRows];
+#pragma unroll
+    for (int r = 0; r < kSelectRows; ++r) acc[r] = 0.f;
+    for (int d = 0; d < head_dim; ++d) {
+      const float kv = __ldg(kt + (long long)d * nk + kb);
+#pragma unroll
+      for (int r = 0; r < kSelectRows; ++r) acc[r] = fmaf(q_s[r * head_dim + d], kv, acc[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < kSelectRows; ++r) sc[r * nk + kb] = acc[r] * inv_sqrt_d;
   }
   __syncthreads();
 
-  auto block_sum = [&](float v) -> float {
+  // ---- warp `wid` owns query block qb0 + wid
+  if (wid >= rows) return;
+  const int qb = qb0 + wid;
+  const float* row = sc + wid * nk;
+  auto warp_sum = [&](float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if (lane == 0) red[wid] = v;
-    __syncthreads();
-    float t = 0.f;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
-    __syncthreads();
-    return t;
+    return v;
   };
   float part = 0.f;
-  for (int kb = tid; kb < nk; kb += blockDim.x) part += sc[kb];
-  const float mu = block_sum(part) / (float)nk;
+  for (int kb = lane; kb < nk; kb += 32) part += row[kb];
+  const float mu = warp_sum(part) / (float)nk;
   part = 0.f;
-  for (int kb = tid; kb < nk; kb += blockDim.x) { const float dlt = sc[kb] - mu; part = fmaf(dlt, dlt, part); }
-  const float sigma = sqrtf(block_sum(part) / (float)nk);
+  for (int kb = lane; kb < nk; kb += 32) { const float dlt = row[kb] - mu; part = fmaf(dlt, dlt, part); }
+  const float sigma = sqrtf(warp_sum(part) / (float)nk);
   const float thr = mu + tau * sigma;
   // arg-max (first one on ties) is always kept
   float best = -CUDART_INF_F;
   int best_i = 0x7fffffff;
-  for (int kb = tid; kb < nk; kb += blockDim.x)
-    if (sc[kb] > best) { best = sc[kb]; best_i = kb; }
+  for (int kb = lane; kb < nk; kb += 32)
+    if (row[kb] > best) { best = row[kb]; best_i = kb; }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float ob = __shfl_xor_sync(0xffffffffu, best, o);
     const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
     if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
   }
-  float* red_v = red;
-  int* red_i = reinterpret_cast<int*>(red + 8);
-  if (lane == 0) { red_v[wid] = best; red_i[wid] = best_i; }
-  __syncthreads();
-  for (int w = 0; w < (int)(blockDim.x >> 5); ++w)
-    if (red_v[w] > best || (red_v[w] == best && red_i[w] < best_i)) { best = red_v[w]; best_i = red_i[w]; }
-  __syncthreads();
 
   const int prefix_kblocks = (sq.text_len + 127) / 128;
   const bool dense_row = qb < (sq.text_len + 255) / 256;
   const uint4* kbits = keybits + sq.ktile_start;
-  int* list = cta_list + sq.sparse_list_start + (long long)local * nk;
-  if (wid == 0) {
-    int count = 0;
-    for (int base = 0; base < nk; base += 32) {
-      const int kb = base + lane;
-      bool on = false;
-      if (kb < nk) {
-        on = dense_row || kb < prefix_kblocks || kb == best_i || sc[kb] > thr;
-        const uint4 b = kbits[kb];
-        on = on && ((b.x | b.y | b.z | b.w) != 0u);
-      }
-      const unsigned ballot = __ballot_sync(0xffffffffu, on);
-      if (on) list[count + __popc(ballot & ((1u << lane) - 1u))] = kb;
-      count += __popc(ballot);
+  const long long local = (long long)head * sq.n_qpairs + qb;   // CTA order of the attention kernel
+  int* list = cta_list + sq.sparse_list_start + local * nk;
+  int count = 0;
+  for (int base = 0; base < nk; base += 32) {
+    const int kb = base + lane;
+    bool on = false;
+    if (kb < nk) {
+      on = dense_row || kb < prefix_kblocks || kb == best_i || row[kb] > thr;
+      const uint4 b = kbits[kb];
+      on = on && ((b.x | b.y | b.z | b.w) != 0u);
     }
-    if (lane == 0) {
-      cta_count[sq.work_start + local] = count;
-      atomicAdd(stats, (unsigned long long)count);
-      atomicAdd(stats + 1, (unsigned long long)nk);
-    }
+    const unsigned ballot = __ballot_sync(0xffffffffu, on);
+    if (on) list[count + __popc(ballot & ((1u << lane) - 1u))] = kb;
+    count += __popc(ballot);
+  }
+  if (lane == 0) {
+    cta_count[sq.work_start + local] = count;
+    atomicAdd(stats, (unsigned long long)count);
+    atomicAdd(stats + 1, (unsigned long long)nk);
   }
 }
 
