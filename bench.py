@@ -35,8 +35,8 @@ NOMINAL_BF16 = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from the ncu summaries under
 # profiles/ (attn_fwd_kernel_lowres_ncu_full.md, bench_highres_launch_list.md).
 NCU_TRAFFIC = {
-    "lowres": (1019664128, "ncu capture of this workload"),
-    "highres": (int(1019664128 * 111856 / 25216), "scaled from the lowres capture by tokens x heads"),
+    "lowres": (1020140288, "ncu capture of this workload"),
+    "highres": (int(1020140288 * 111856 / 25216), "scaled from the lowres capture by tokens x heads"),
 }
 
 

@@ -93,7 +93,7 @@ struct RopeArgs {
   RopeGeom g;
 };
 
-__global__ void __launch_bounds__(256) rope_qk_kernel(const RopeArgs a) {
+__global__ void __launch_bounds__(256, 4) rope_qk_kernel(const RopeArgs a) {
   const int chunks = a.g.head_dim >> 3;          // 16-byte chunks per head row (8 or 16: divides the warp)
   const int heads_per_pass = blockDim.x / chunks;
   const int chunk = threadIdx.x % chunks;
@@ -136,39 +136,51 @@ __global__ void __launch_bounds__(256) rope_qk_kernel(const RopeArgs a) {
       const bool norm = a.gain[which] != nullptr;
       const __nv_bfloat16* src = a.x[which] + tok * a.x_tok_stride[which] + chunk * 8;
       __nv_bfloat16* dst = a.y[which] + (tok * a.g.heads) * (long long)a.g.head_dim + chunk * 8;
-      for (int h = hsub; h < a.g.heads; h += heads_per_pass) {
-        // all lanes of a row enter together (the loop bound depends on hsub only)
-        const unsigned lanes = __activemask();
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        float f[8];
+      // heads in groups of kBatch per thread: all loads of a group are issued before any is used
+      constexpr int kBatch = 3;
+      for (int h0 = hsub; h0 < a.g.heads; h0 += kBatch * heads_per_pass) {
+        uint4 v[kBatch];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162*>(&w[u]);
-          f[2 * u] = __low2float(b2);
-          f[2 * u + 1] = __high2float(b2);
+        for (int b = 0; b < kBatch; ++b) {
+          const int h = h0 + b * heads_per_pass;
+          if (h < a.g.heads) v[b] = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
         }
-        if (norm) {
-          float ss = 0.f;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
-          for (int off = chunks >> 1; off > 0; off >>= 1) ss += __shfl_xor_sync(lanes, ss, off);
-          const float r = rsqrtf(ss * inv_d + a.eps);
+        for (int b = 0; b < kBatch; ++b) {
+          const int h = h0 + b * heads_per_pass;
+          if (h >= a.g.heads) break;
+          // all lanes of a row enter together (the bound depends on hsub only)
+          const unsigned lanes = __activemask();
+          const uint32_t w[4] = {v[b].x, v[b].y, v[b].z, v[b].w};
+          float f[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) f[e] = f[e] * r * gn[which][e];
-        }
-        uint32_t o[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          float re = f[2 * u], ro = f[2 * u + 1];
-          if (rotate) {
-            re = f[2 * u] * cs[u].x - f[2 * u + 1] * cs[u].y;
-            ro = f[2 * u] * cs[u].y + f[2 * u + 1] * cs[u].x;
+          for (int u = 0; u < 4; ++u) {
+            const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162*>(&w[u]);
+            f[2 * u] = __low2float(b2);
+            f[2 * u + 1] = __high2float(b2);
           }
-          const __nv_bfloat162 r2 = __floats2bfloat162_rn(re, ro);
-          o[u] = *reinterpret_cast<const uint32_t*>(&r2);
+          if (norm) {
+            float ss = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+            for (int off = chunks >> 1; off > 0; off >>= 1) ss += __shfl_xor_sync(lanes, ss, off);
+            const float r = rsqrtf(ss * inv_d + a.eps);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = f[e] * r * gn[which][e];
+          }
+          uint32_t o[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            float re = f[2 * u], ro = f[2 * u + 1];
+            if (rotate) {
+              re = f[2 * u] * cs[u].x - f[2 * u + 1] * cs[u].y;
+              ro = f[2 * u] * cs[u].y + f[2 * u + 1] * cs[u].x;
+            }
+            const __nv_bfloat162 r2 = __floats2bfloat162_rn(re, ro);
+            o[u] = *reinterpret_cast<const uint32_t*>(&r2);
+          }
+          *reinterpret_cast<uint4*>(dst + (long long)h * a.g.head_dim) = make_uint4(o[0], o[1], o[2], o[3]);
         }
-        *reinterpret_cast<uint4*>(dst + (long long)h * a.g.head_dim) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   }
