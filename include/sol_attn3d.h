@@ -167,6 +167,79 @@ int sol_attn3d_forward_rect(sol_attn3d_plan_t plan, const void* q, const void* k
                             const uint8_t* key_mask, const uint8_t* query_mask, sol_attn3d_stream_t stream);
 
 /*
+ * sol_attn3d_forward with the FP8 output format of Section 3.3 ("Quantized communication": the FP8
+ * alternative transmits 128 raw E4M3 bytes per token/head, without scale metadata or padding; "Joint
+ * optimization with quantized communication": the raw E4M3 values returned by attention feed the quantized
+ * output projection with unit scales).  The epilogue converts O/l from fp32 straight to E4M3 (round to
+ * nearest even, magnitudes above 448 saturate, no bf16 step in between).
+ *   out_e4m3   DEVICE pointer, uint8 [total_tokens, heads, head_dim] with the plan's out strides (counted
+ *              in elements = bytes here), 16-byte aligned; rows of head_dim bytes.
+ * Everything else as for sol_attn3d_forward.
+ */
+int sol_attn3d_forward_e4m3(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out_e4m3,
+                            const uint8_t* key_mask, sol_attn3d_stream_t stream);
+
+/*
+ * Sequence-parallel exchange around the attention (Section 3.3, "Optimized attention collectives"): ranks
+ * hold contiguous ranges of the flat token axis with all heads; attention needs every token for a shard of
+ * the heads.  The paper's path is pack -> all-to-all -> attention -> all-to-all -> head merge with ONE
+ * collective each way; the two layout kernels below are bit-exact copies of 16-byte chunks.
+ */
+#define SOL_ATTN3D_MAX_RANKS 8
+#define SOL_ATTN3D_OUT_BF16 0
+#define SOL_ATTN3D_OUT_E4M3 1
+
+/*
+ * Sender's side, one pass: reads this rank's Q, K, V [n_local, heads, head_dim] (bf16, DEVICE) through their
+ * element strides {token, head} ({0,0} = contiguous; views into a packed QKV buffer are fine) and writes, for
+ * every destination g < n_ranks, heads [g*heads/n_ranks, (g+1)*heads/n_ranks) as rows
+ *   dst[g][dst_row0 + t][which = q,k,v][heads/n_ranks][head_dim].
+ *   dst        HOST array of n_ranks DEVICE pointers, 16-byte aligned, caller-owned.  Either slices of one
+ *              local send buffer with dst_row0 = 0 (then one all-to-all follows), or the ranks' receive
+ *              buffers mapped into this process (peer memory) with dst_row0 = this rank's first token: the
+ *              pack and the transfer are then the same pass of plain peer stores, and the caller needs a
+ *              barrier across ranks before the attention reads the buffer.
+ * After the exchange rank g holds [total_tokens][3][heads/n_ranks][head_dim]; its Q, K, V are views with
+ * token stride 3*heads/n_ranks*head_dim that sol_attn3d_plan_ex takes as they are.
+ * n_local = 0 is a no-op (pointers are not looked at).
+ * Errors: INVALID_ARG (NULL / misaligned pointer, heads not divisible, n_ranks > SOL_ATTN3D_MAX_RANKS), CUDA.
+ */
+int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, const int64_t q_strides[2],
+                                 const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
+                                 int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
+                                 sol_attn3d_stream_t stream);
+
+/*
+ * Receiver's side of the output return (the paper's "inverse head merge"): recv [n_ranks][n_local]
+ * [heads/n_ranks][record_bytes] (DEVICE; slice g = what rank g computed for this rank's tokens) ->
+ * out [n_local][heads][record_bytes] with head = g*heads/n_ranks + local head, the row-major input of the
+ * output projection.  record_bytes is the size of one (token, head) record on the wire, a multiple of 16:
+ * 2*head_dim for bf16, head_dim for raw E4M3.  out_tok_stride_bytes: 0 = dense.  recv and out must not alias.
+ */
+int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local, int heads, int record_bytes,
+                                    int n_ranks, int64_t out_tok_stride_bytes, sol_attn3d_stream_t stream);
+
+/*
+ * sol_attn3d_forward whose epilogue delivers each output row to the owner of its token: the output return
+ * of the exchange and the head merge fused into the attention kernel (no counterpart kernel in the paper,
+ * which returns the output with a collective; same result).  The plan describes this rank's head shard
+ * over all tokens.  Destination g owns flat tokens [tok_begin[g], tok_begin[g+1]) and receives them as rows
+ *   dst[g][token - tok_begin[g]][head_offset + h][head_dim],   row stride dst_heads * head_dim elements.
+ *   n_dst       1 .. SOL_ATTN3D_MAX_RANKS.
+ *   dst         HOST array of n_dst DEVICE pointers (this GPU's memory or a peer's mapped into this process;
+ *               plain stores, whole 16-byte chunks of contiguous rows), 16-byte aligned; may be NULL for an
+ *               owner without tokens.
+ *   tok_begin   HOST array of n_dst+1 ascending token offsets, tok_begin[0] = 0, tok_begin[n_dst] = total.
+ *   dst_heads   heads per row in the destinations (all ranks' shards); head_offset = this shard's first head.
+ *   out_format  SOL_ATTN3D_OUT_BF16 or SOL_ATTN3D_OUT_E4M3 (see sol_attn3d_forward_e4m3).
+ * The arrays are read during the call only.  The caller needs a barrier across ranks before the owners
+ * read their rows.  Everything else as for sol_attn3d_forward.
+ */
+int sol_attn3d_forward_scatter(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v,
+                               const uint8_t* key_mask, int n_dst, void* const* dst, const int64_t* tok_begin,
+                               int dst_heads, int head_offset, int out_format, sol_attn3d_stream_t stream);
+
+/*
  * Block-sparse variant of sol_attn3d_forward: the per-step dynamic sparsity of Section 3.4 ("Sparse
  * Attention") with its safety rails.  An approximation of dense attention.
  *   Query blocks of 256 tokens, KV blocks of 128 tokens, per sequence and head.  Block-level score =

@@ -87,6 +87,16 @@ def _lib():
     lib.sol_attn3d_qknorm_rope.restype = i32
     lib.sol_attn3d_forward_rect.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.sol_attn3d_forward_rect.restype = i32
+    lib.sol_attn3d_forward_e4m3.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.sol_attn3d_forward_e4m3.restype = i32
+    lib.sol_attn3d_forward_scatter.argtypes = [vp, vp, vp, vp, vp, i32, ctypes.POINTER(vp), ctypes.POINTER(i64), i32, i32,
+                                               i32, vp]
+    lib.sol_attn3d_forward_scatter.restype = i32
+    lib.sol_attn3d_exchange_pack_qkv.argtypes = [vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i64),
+                                                 i64, i32, i32, i32, ctypes.POINTER(vp), i64, vp]
+    lib.sol_attn3d_exchange_pack_qkv.restype = i32
+    lib.sol_attn3d_exchange_merge_heads.argtypes = [vp, vp, i64, i32, i32, i32, i64, vp]
+    lib.sol_attn3d_exchange_merge_heads.restype = i32
     lib.sol_attn3d_sparse_workspace_bytes.argtypes = [vp]
     lib.sol_attn3d_sparse_workspace_bytes.restype = ctypes.c_size_t
     lib.sol_attn3d_forward_sparse.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp]
@@ -223,6 +233,69 @@ def sol_attn3d_forward_rect(plan, q, k, v, out, key_mask, query_mask: torch.Tens
         raise ValueError("query_mask must be a contiguous CUDA uint8 tensor")
     _check(_lib().sol_attn3d_forward_rect(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask), _ptr(query_mask),
                                           _stream(stream)), "sol_attn3d_forward_rect")
+
+
+OUT_BF16, OUT_E4M3 = 0, 1
+MAX_RANKS = 8
+
+
+def sol_attn3d_forward_e4m3(plan, q, k, v, out_e4m3: torch.Tensor, key_mask=None, stream=None) -> None:
+    """Forward whose epilogue writes one raw E4M3 byte per output element (unit scale)."""
+    for t in (q, k, v):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v must be CUDA bf16 tensors")
+    if not out_e4m3.is_cuda or out_e4m3.element_size() != 1:
+        raise ValueError("out_e4m3 must be a CUDA tensor of one-byte elements")
+    _check(_lib().sol_attn3d_forward_e4m3(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out_e4m3), _ptr(key_mask),
+                                          _stream(stream)), "sol_attn3d_forward_e4m3")
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    return (ctypes.c_void_p * len(ptrs))(*[ctypes.c_void_p(int(x)) if x else None for x in ptrs])
+
+
+def sol_attn3d_forward_scatter(plan, q, k, v, key_mask, dst: Sequence[int], tok_begin: Sequence[int], dst_heads: int,
+                               head_offset: int, out_format: int = OUT_BF16, stream=None) -> None:
+    """dst: device addresses (ints; this GPU's or peer-mapped) of the token owners' [n_g, dst_heads, D] buffers."""
+    for t in (q, k, v):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v must be CUDA bf16 tensors")
+    if len(tok_begin) != len(dst) + 1:
+        raise ValueError("tok_begin needs len(dst) + 1 entries")
+    tb = (ctypes.c_int64 * len(tok_begin))(*[int(x) for x in tok_begin])
+    _check(_lib().sol_attn3d_forward_scatter(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(key_mask), len(dst), _ptr_array(dst),
+                                             tb, dst_heads, head_offset, out_format, _stream(stream)),
+           "sol_attn3d_forward_scatter")
+
+
+def _strides_of(t: torch.Tensor, head_dim: int):
+    if t.dim() != 3 or t.stride(2) != 1 or t.shape[2] != head_dim:
+        raise ValueError("expected [tokens, heads, head_dim] with contiguous head_dim")
+    tok = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1] * head_dim)
+    return (ctypes.c_int64 * 2)(tok, t.stride(1) if t.shape[1] > 1 else head_dim)
+
+
+def sol_attn3d_exchange_pack_qkv(q, k, v, n_ranks: int, dst: Sequence[int], dst_row0: int = 0, stream=None) -> None:
+    """q, k, v: CUDA bf16 [n_local, heads, D] (any token / head strides); dst: n_ranks device addresses."""
+    n_local, heads, head_dim = q.shape
+    for t in (q, k, v):
+        if not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != (n_local, heads, head_dim):
+            raise ValueError("q, k, v must be CUDA bf16 tensors of one shape")
+    if len(dst) != n_ranks:
+        raise ValueError("one destination per rank")
+    _check(_lib().sol_attn3d_exchange_pack_qkv(_ptr(q), _ptr(k), _ptr(v), _strides_of(q, head_dim), _strides_of(k, head_dim),
+                                               _strides_of(v, head_dim), n_local, heads, head_dim, n_ranks,
+                                               _ptr_array(dst), dst_row0, _stream(stream)),
+           "sol_attn3d_exchange_pack_qkv")
+
+
+def sol_attn3d_exchange_merge_heads(recv: torch.Tensor, out: torch.Tensor, n_local: int, heads: int, record_bytes: int,
+                                    n_ranks: int, out_tok_stride_bytes: int = 0, stream=None) -> None:
+    if not recv.is_cuda or not out.is_cuda or not recv.is_contiguous():
+        raise ValueError("recv and out must be CUDA tensors, recv contiguous")
+    _check(_lib().sol_attn3d_exchange_merge_heads(_ptr(recv), _ptr(out), n_local, heads, record_bytes, n_ranks,
+                                                  out_tok_stride_bytes, _stream(stream)),
+           "sol_attn3d_exchange_merge_heads")
 
 
 def sol_attn3d_sparse_workspace_bytes(plan) -> int:

@@ -11,8 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB_NAME = "libsol_attn3d.so"
 LIB_PATH = os.path.join(HERE, LIB_NAME)
 SOURCES = ["sol_attn3d.cu"]
-HEADERS = ["attn_fwd_sm100.cuh", "prologue_kernels.cuh", "ptx_sm100.cuh", "device_types.cuh",
-           os.path.join("..", "..", "include", "sol_attn3d.h")]
+HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith(".cuh")) + [os.path.join("..", "..", "include", "sol_attn3d.h")]
 
 
 def _nvcc() -> str:

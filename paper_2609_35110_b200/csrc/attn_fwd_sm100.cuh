@@ -98,6 +98,69 @@ __device__ __forceinline__ void softmax_pass(const uint32_t (&r)[128], float c, 
   sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
 }
 
+// Address of output row (flat token, head) in the destination that owns the token.
+__device__ __forceinline__ uint8_t* out_row_ptr(const AttnParams& p, long long tok, int head, int elem_bytes) {
+  int g = 0;
+  while (g + 1 < p.sink.n_dst && tok >= p.sink.tok_begin[g + 1]) ++g;
+  return static_cast<uint8_t*>(p.sink.base[g]) +
+         ((tok - p.sink.tok_begin[g]) * p.o_tok_stride + (long long)head * p.o_head_stride) * elem_bytes;
+}
+
+// Epilogue of one warp: its 32 accumulator rows O * inv -> bf16 (or raw E4M3 bytes) -> staged in the part of
+// the query tile's shared memory that belongs to those rows (every MMA that read it has completed; 16-byte
+// chunks XOR-swizzled by row) -> written out with one 16-byte chunk per lane, so every store instruction
+// covers whole contiguous rows.  Rows beyond the sequence, or not wanted by the query mask, are not stored.
+template <int D, bool kFp8>
+__device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq, int head, int first_row, int lane,
+                                           uint32_t tO, float inv, uint8_t* stage) {
+  constexpr int kRowBytes = kFp8 ? D : D * 2;
+  constexpr int kLanesPerRow = kRowBytes / 16;
+#pragma unroll
+  for (int cch = 0; cch < D / 32; ++cch) {
+    uint32_t o[32];
+    tmem_ld32(tO + cch * 32, o);
+    tmem_wait_ld();
+    if (kFp8) {
+#pragma unroll
+      for (int v4 = 0; v4 < 2; ++v4) {
+        uint4 w;
+        w.x = pack_e4m3x4(__uint_as_float(o[16 * v4 + 0]) * inv, __uint_as_float(o[16 * v4 + 1]) * inv,
+                          __uint_as_float(o[16 * v4 + 2]) * inv, __uint_as_float(o[16 * v4 + 3]) * inv);
+        w.y = pack_e4m3x4(__uint_as_float(o[16 * v4 + 4]) * inv, __uint_as_float(o[16 * v4 + 5]) * inv,
+                          __uint_as_float(o[16 * v4 + 6]) * inv, __uint_as_float(o[16 * v4 + 7]) * inv);
+        w.z = pack_e4m3x4(__uint_as_float(o[16 * v4 + 8]) * inv, __uint_as_float(o[16 * v4 + 9]) * inv,
+                          __uint_as_float(o[16 * v4 + 10]) * inv, __uint_as_float(o[16 * v4 + 11]) * inv);
+        w.w = pack_e4m3x4(__uint_as_float(o[16 * v4 + 12]) * inv, __uint_as_float(o[16 * v4 + 13]) * inv,
+                          __uint_as_float(o[16 * v4 + 14]) * inv, __uint_as_float(o[16 * v4 + 15]) * inv);
+        const int ch = cch * 2 + v4;
+        *reinterpret_cast<uint4*>(stage + lane * kRowBytes + ((ch ^ (lane & (kLanesPerRow - 1))) << 4)) = w;
+      }
+    } else {
+#pragma unroll
+      for (int v4 = 0; v4 < 4; ++v4) {
+        uint4 w;
+        w.x = pack_bf16x2(__uint_as_float(o[8 * v4 + 0]) * inv, __uint_as_float(o[8 * v4 + 1]) * inv);
+        w.y = pack_bf16x2(__uint_as_float(o[8 * v4 + 2]) * inv, __uint_as_float(o[8 * v4 + 3]) * inv);
+        w.z = pack_bf16x2(__uint_as_float(o[8 * v4 + 4]) * inv, __uint_as_float(o[8 * v4 + 5]) * inv);
+        w.w = pack_bf16x2(__uint_as_float(o[8 * v4 + 6]) * inv, __uint_as_float(o[8 * v4 + 7]) * inv);
+        const int ch = cch * 4 + v4;
+        *reinterpret_cast<uint4*>(stage + lane * kRowBytes + ((ch ^ (lane & (kLanesPerRow - 1))) << 4)) = w;
+      }
+    }
+  }
+  __syncwarp();
+  const int ch = lane % kLanesPerRow;
+#pragma unroll 4
+  for (int r0 = 0; r0 < 32; r0 += 32 / kLanesPerRow) {
+    const int rr = r0 + lane / kLanesPerRow;
+    const int qrow = first_row + rr;
+    bool store = qrow < sq.n_tokens;
+    if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
+    const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * kRowBytes + ((ch ^ (rr & (kLanesPerRow - 1))) << 4));
+    if (store) *reinterpret_cast<uint4*>(out_row_ptr(p, sq.tok_start + qrow, head, kFp8 ? 1 : 2) + ch * 16) = w;
+  }
+}
+
 template <int D>
 struct AttnSmem {
   static constexpr int kTile = 128 * D * 2;               // bytes of one 128 x D bf16 tile
@@ -265,61 +328,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_arrive(bar_p_full(t));
     }
 
-    // ---- epilogue: O / l -> bf16 -> shared-memory staging -> coalesced 16-byte stores
-    //      (rows beyond the sequence, or not wanted by the query mask, are not stored)
+    // ---- epilogue: O / l in the output format, staged through shared memory, coalesced 16-byte stores
     if (ok && n_proc > 0) {
       ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(t), (n_proc - 1) & 1, limit));
       if (ok) tc_fence_after();
     }
     if (ok && n_proc > 0) {
-      // Each warp stages its 32 rows (bf16, XOR-swizzled 16-byte chunks) in the part of the query tile's
-      // shared memory that belongs to those rows -- every MMA that read it has completed -- and then writes
-      // them out with D/8 lanes per row, so every store instruction covers whole contiguous rows.
-      constexpr int kRowBytes = D * 2;
-      constexpr int kLanesPerRow = D / 8;
-      uint8_t* stage = smem + L::kOffQ + t * L::kTile + wq * 32 * kRowBytes;
       const float inv = 1.0f / l;
-#pragma unroll
-      for (int cch = 0; cch < D / 32; ++cch) {
-        uint32_t o[32];
-        tmem_ld32(tO + cch * 32, o);
-        tmem_wait_ld();
-#pragma unroll
-        for (int v4 = 0; v4 < 4; ++v4) {
-          uint4 w;
-          w.x = pack_bf16x2(__uint_as_float(o[8 * v4 + 0]) * inv, __uint_as_float(o[8 * v4 + 1]) * inv);
-          w.y = pack_bf16x2(__uint_as_float(o[8 * v4 + 2]) * inv, __uint_as_float(o[8 * v4 + 3]) * inv);
-          w.z = pack_bf16x2(__uint_as_float(o[8 * v4 + 4]) * inv, __uint_as_float(o[8 * v4 + 5]) * inv);
-          w.w = pack_bf16x2(__uint_as_float(o[8 * v4 + 6]) * inv, __uint_as_float(o[8 * v4 + 7]) * inv);
-          const int ch = cch * 4 + v4;
-          *reinterpret_cast<uint4*>(stage + lane * kRowBytes + ((ch ^ (lane & (kLanesPerRow - 1))) << 4)) = w;
-        }
-      }
-      __syncwarp();
-      const int ch = lane % kLanesPerRow;
-#pragma unroll 4
-      for (int r0 = 0; r0 < 32; r0 += 32 / kLanesPerRow) {
-        const int rr = r0 + lane / kLanesPerRow;
-        const int qrow = q_row0 + t * 128 + wq * 32 + rr;
-        bool store = qrow < sq.n_tokens;
-        if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
-        const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * kRowBytes + ((ch ^ (rr & (kLanesPerRow - 1))) << 4));
-        if (store) {
-          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (sq.tok_start + qrow) * p.o_tok_stride +
-                               (long long)head * p.o_head_stride + ch * 8;
-          *reinterpret_cast<uint4*>(dst) = w;
-        }
-      }
+      uint8_t* stage = smem + L::kOffQ + t * L::kTile + wq * 32 * (D * 2);
+      if (p.sink.fmt == kOutE4M3) store_rows<D, true>(p, sq, head, q_row0 + t * 128 + wq * 32, lane, tO, inv, stage);
+      else                        store_rows<D, false>(p, sq, head, q_row0 + t * 128 + wq * 32, lane, tO, inv, stage);
     } else if (ok) {
       // no key tile at all (every key of the sequence masked): the row is defined as zero
       const int qrow = q_row0 + t * 128 + row;
       bool store = qrow < sq.n_tokens;
       if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
       if (store) {
-        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) +
-                             (sq.tok_start + qrow) * p.o_tok_stride + (long long)head * p.o_head_stride;
-#pragma unroll
-        for (int c16 = 0; c16 < D / 8; ++c16) *reinterpret_cast<uint4*>(dst + c16 * 8) = make_uint4(0u, 0u, 0u, 0u);
+        const int row_bytes = p.sink.fmt == kOutE4M3 ? D : D * 2;
+        uint8_t* dst = out_row_ptr(p, sq.tok_start + qrow, head, row_bytes / D);
+        for (int c16 = 0; c16 < row_bytes / 16; ++c16) *reinterpret_cast<uint4*>(dst + c16 * 16) = make_uint4(0u, 0u, 0u, 0u);
       }
     } else if (lane == 0) {
       atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);

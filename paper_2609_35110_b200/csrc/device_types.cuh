@@ -28,6 +28,18 @@ struct RopeGeom {
   int heads;
 };
 
+// Where the output rows go.  Destination g receives the rows of flat tokens [tok_begin[g], tok_begin[g+1]);
+// base[g] addresses row tok_begin[g] (head 0 of this launch) in that destination, which may be this GPU's
+// memory or a peer's mapped into this process.  Plain forward: one destination starting at token 0.
+constexpr int kMaxOutDst = 8;
+enum : int { kOutBf16 = 0, kOutE4M3 = 1 };
+struct OutSink {
+  void* base[kMaxOutDst];
+  long long tok_begin[kMaxOutDst + 1];
+  int n_dst;
+  int fmt;                  // kOutBf16: 2-byte elements; kOutE4M3: one raw E4M3 byte per element (unit scale)
+};
+
 struct AttnParams {
   const SeqDev* seqs;
   int n_seqs;
@@ -39,7 +51,7 @@ struct AttnParams {
   const uint8_t* pair_needed;  // rectangular mode: per (sequence, query pair), nonzero = at least one wanted row
   const int* cta_list;      // block-sparse mode: per CTA, the key tiles it attends (n_ktiles slots each); else nullptr
   const int* cta_count;     // block-sparse mode: per CTA, how many
-  void* out;
+  OutSink sink;
   long long o_tok_stride, o_head_stride;  // in elements
   float scale_log2;         // log2(e) / sqrt(head_dim)
   unsigned int* status;     // 0 = fine; written once on a wait time-out

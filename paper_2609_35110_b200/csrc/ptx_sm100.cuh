@@ -341,6 +341,17 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
+// four floats -> four E4M3 bytes (round to nearest even, saturating at +-448, NaN -> 0x7f), x0 in the lowest byte
+__device__ __forceinline__ uint32_t pack_e4m3x4(float x0, float x1, float x2, float x3) {
+  uint32_t r;
+  asm("{\n\t.reg .b16 lo, hi;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+      "mov.b32 %0, {lo, hi};\n\t}"
+      : "=r"(r) : "f"(x0), "f"(x1), "f"(x2), "f"(x3));
+  return r;
+}
+
 // ------------------------------------------------------------------ packed fp32x2 arithmetic (sm_100)
 __device__ __forceinline__ uint64_t pack_f2(float lo, float hi) {
   uint64_t d;

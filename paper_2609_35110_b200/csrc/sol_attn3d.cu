@@ -13,6 +13,7 @@
 
 #include "attn_fwd_sm100.cuh"
 #include "device_types.cuh"
+#include "exchange_kernels.cuh"
 #include "prologue_kernels.cuh"
 #include "sparse_kernels.cuh"
 
@@ -383,14 +384,27 @@ int sol_attn3d_rope_qk(sol_attn3d_plan_t p, const void* q, const void* k, void* 
 }
 
 namespace {
+// Optional parts of a forward call.
+struct FwdOpts {
+  const float* q_gain = nullptr;      // QK RMS-norm gains (both or neither)
+  const float* k_gain = nullptr;
+  float eps = 0.f;
+  unsigned char* sparse_ws = nullptr; // block-sparse scratch
+  float tau = 0.f;
+  const uint8_t* query_mask = nullptr;
+  int out_fmt = sol::kOutBf16;
+  int n_dst = 0;                      // > 0: rows are scattered to their token owners instead of `out`
+  void* const* dst = nullptr;
+  const int64_t* tok_begin = nullptr;
+  int dst_heads = 0, head_offset = 0;
+};
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
-                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream,
-                 unsigned char* sparse_ws = nullptr, float tau = 0.f, const uint8_t* query_mask = nullptr);
+                 sol_attn3d_stream_t stream, const FwdOpts& o);
 }
 
 int sol_attn3d_forward(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
                        const uint8_t* key_mask, sol_attn3d_stream_t stream) {
-  return forward_impl(p, q, k, v, out, key_mask, nullptr, nullptr, 0.f, stream);
+  return forward_impl(p, q, k, v, out, key_mask, stream, FwdOpts{});
 }
 
 int sol_attn3d_forward_qknorm(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
@@ -399,13 +413,100 @@ int sol_attn3d_forward_qknorm(sol_attn3d_plan_t p, const void* q, const void* k,
   if (q_gain == nullptr || k_gain == nullptr || !(eps >= 0.f)) return SOL_ATTN3D_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(q_gain) & 3u) != 0 || (reinterpret_cast<uintptr_t>(k_gain) & 3u) != 0)
     return SOL_ATTN3D_ERR_INVALID_ARG;
-  return forward_impl(p, q, k, v, out, key_mask, q_gain, k_gain, eps, stream);
+  FwdOpts o;
+  o.q_gain = q_gain;
+  o.k_gain = k_gain;
+  o.eps = eps;
+  return forward_impl(p, q, k, v, out, key_mask, stream, o);
 }
 
 int sol_attn3d_forward_rect(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
                             const uint8_t* key_mask, const uint8_t* query_mask, sol_attn3d_stream_t stream) {
   if (query_mask == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
-  return forward_impl(p, q, k, v, out, key_mask, nullptr, nullptr, 0.f, stream, nullptr, 0.f, query_mask);
+  FwdOpts o;
+  o.query_mask = query_mask;
+  return forward_impl(p, q, k, v, out, key_mask, stream, o);
+}
+
+int sol_attn3d_forward_e4m3(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out_e4m3,
+                            const uint8_t* key_mask, sol_attn3d_stream_t stream) {
+  FwdOpts o;
+  o.out_fmt = sol::kOutE4M3;
+  return forward_impl(p, q, k, v, out_e4m3, key_mask, stream, o);
+}
+
+int sol_attn3d_forward_scatter(sol_attn3d_plan_t p, const void* q, const void* k, const void* v,
+                               const uint8_t* key_mask, int n_dst, void* const* dst, const int64_t* tok_begin,
+                               int dst_heads, int head_offset, int out_format, sol_attn3d_stream_t stream) {
+  if (n_dst < 1 || (out_format != SOL_ATTN3D_OUT_BF16 && out_format != SOL_ATTN3D_OUT_E4M3))
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  FwdOpts o;
+  o.out_fmt = out_format == SOL_ATTN3D_OUT_E4M3 ? sol::kOutE4M3 : sol::kOutBf16;
+  o.n_dst = n_dst;
+  o.dst = dst;
+  o.tok_begin = tok_begin;
+  o.dst_heads = dst_heads;
+  o.head_offset = head_offset;
+  return forward_impl(p, q, k, v, nullptr, key_mask, stream, o);
+}
+
+int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, const int64_t q_strides[2],
+                                 const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
+                                 int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
+                                 sol_attn3d_stream_t stream) {
+  if (n_local < 0 || dst_row0 < 0 || heads < 1 || head_dim < 8 || (head_dim % 8) != 0 || n_ranks < 1 ||
+      n_ranks > sol::kMaxRanks || (heads % n_ranks) != 0)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (n_local == 0) return SOL_ATTN3D_OK;            // a rank without tokens sends nothing (its pointers may be NULL)
+  if (q == nullptr || k == nullptr || v == nullptr || dst == nullptr || q_strides == nullptr || k_strides == nullptr ||
+      v_strides == nullptr)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  sol::PackArgs a{};
+  const void* src[3] = {q, k, v};
+  const int64_t* strides[3] = {q_strides, k_strides, v_strides};
+  for (int w = 0; w < 3; ++w) {
+    const long long tok = strides[w][0] == 0 ? (long long)heads * head_dim : strides[w][0];
+    const long long head = strides[w][1] == 0 ? head_dim : strides[w][1];
+    if (!aligned16(src[w]) || !stride_ok(tok) || !stride_ok(head)) return SOL_ATTN3D_ERR_INVALID_ARG;
+    a.src[w] = static_cast<const uint8_t*>(src[w]);
+    a.tok_stride_bytes[w] = tok * 2;
+    a.head_stride_bytes[w] = head * 2;
+  }
+  for (int g = 0; g < n_ranks; ++g) {
+    if (dst[g] == nullptr || !aligned16(dst[g])) return SOL_ATTN3D_ERR_INVALID_ARG;
+    a.dst[g] = static_cast<uint8_t*>(dst[g]);
+  }
+  a.dst_row0 = dst_row0;
+  a.n_local = n_local;
+  a.heads = heads;
+  a.hl = heads / n_ranks;
+  a.n_ranks = n_ranks;
+  a.chunks = head_dim * 2 / 16;
+  const long long items = n_local * 3ll * heads * a.chunks;
+  const long long want = (items + 256ll * sol::kPackUnroll - 1) / (256ll * sol::kPackUnroll);
+  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>(want, 148ll * 16));
+  sol::exchange_pack_qkv_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
+}
+
+int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local, int heads, int record_bytes,
+                                    int n_ranks, int64_t out_tok_stride_bytes, sol_attn3d_stream_t stream) {
+  if (n_local < 0 || heads < 1 || record_bytes < 16 || (record_bytes % 16) != 0 || n_ranks < 1 ||
+      n_ranks > sol::kMaxRanks || (heads % n_ranks) != 0)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (n_local == 0) return SOL_ATTN3D_OK;            // a rank without tokens receives nothing
+  if (recv == nullptr || out == nullptr || recv == out || !aligned16(recv) || !aligned16(out))
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  const long long dense = (long long)heads * record_bytes;
+  const long long ots = out_tok_stride_bytes == 0 ? dense : out_tok_stride_bytes;
+  if (ots < dense || (ots % 16) != 0) return SOL_ATTN3D_ERR_INVALID_ARG;
+  const int chunks = record_bytes / 16;
+  const long long items = n_local * (long long)heads * chunks;
+  const long long want = (items + 256ll * sol::kPackUnroll - 1) / (256ll * sol::kPackUnroll);
+  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>(want, 148ll * 16));
+  sol::exchange_merge_heads_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint8_t*>(recv), static_cast<uint8_t*>(out), n_local, heads / n_ranks, n_ranks, chunks, ots);
+  return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
 }
 
 size_t sol_attn3d_sparse_workspace_bytes(sol_attn3d_plan_t p) { return p ? p->sp_bytes : 0; }
@@ -416,7 +517,10 @@ int sol_attn3d_forward_sparse(sol_attn3d_plan_t p, const void* q, const void* k,
   if (p == nullptr || !(tau == tau)) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (sparse_ws == nullptr || sparse_ws_bytes < p->sp_bytes || (reinterpret_cast<uintptr_t>(sparse_ws) % kAlign) != 0)
     return SOL_ATTN3D_ERR_NO_WORKSPACE;
-  return forward_impl(p, q, k, v, out, key_mask, nullptr, nullptr, 0.f, stream, static_cast<unsigned char*>(sparse_ws), tau);
+  FwdOpts o;
+  o.sparse_ws = static_cast<unsigned char*>(sparse_ws);
+  o.tau = tau;
+  return forward_impl(p, q, k, v, out, key_mask, stream, o);
 }
 
 int sol_attn3d_sparse_stats(sol_attn3d_plan_t p, const void* sparse_ws, long long* selected_tiles, long long* all_tiles) {
@@ -470,11 +574,44 @@ int sol_attn3d_qknorm_rope(sol_attn3d_plan_t p, const void* q, const void* k, co
 
 namespace {
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
-                 const float* q_gain, const float* k_gain, float eps, sol_attn3d_stream_t stream,
-                 unsigned char* sparse_ws, float tau, const uint8_t* query_mask) {
-  if (p == nullptr || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
-  if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
+                 sol_attn3d_stream_t stream, const FwdOpts& o) {
+  if (p == nullptr || q == nullptr || k == nullptr || v == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  sol::OutSink sink{};
+  sink.fmt = o.out_fmt;
+  long long o_tok_stride = p->so.tok, o_head_stride = p->so.head;
+  if (o.n_dst > 0) {
+    // scatter: destination g owns flat tokens [tok_begin[g], tok_begin[g+1]) as rows [n_g][dst_heads][head_dim]
+    if (o.n_dst > sol::kMaxOutDst || o.dst == nullptr || o.tok_begin == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+    if (o.head_offset < 0 || o.dst_heads < o.head_offset + p->heads) return SOL_ATTN3D_ERR_INVALID_ARG;
+    if (o.tok_begin[0] != 0 || o.tok_begin[o.n_dst] != p->total_tokens) return SOL_ATTN3D_ERR_INVALID_ARG;
+    const size_t esize = o.out_fmt == sol::kOutE4M3 ? 1 : 2;
+    for (int g = 0; g < o.n_dst; ++g) {
+      if (o.tok_begin[g + 1] < o.tok_begin[g]) return SOL_ATTN3D_ERR_INVALID_ARG;
+      const bool empty = o.tok_begin[g + 1] == o.tok_begin[g];
+      if (!empty && (o.dst[g] == nullptr || !aligned16(o.dst[g]))) return SOL_ATTN3D_ERR_INVALID_ARG;
+      if (o.dst[g] == q || o.dst[g] == k || o.dst[g] == v) return SOL_ATTN3D_ERR_INVALID_ARG;
+      sink.base[g] = static_cast<unsigned char*>(o.dst[g]) + (size_t)o.head_offset * p->head_dim * esize;
+      sink.tok_begin[g] = o.tok_begin[g];
+    }
+    sink.tok_begin[o.n_dst] = o.tok_begin[o.n_dst];
+    sink.n_dst = o.n_dst;
+    o_tok_stride = (long long)o.dst_heads * p->head_dim;
+    o_head_stride = p->head_dim;
+  } else {
+    if (out == nullptr || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
+    if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
+    sink.base[0] = out;
+    sink.tok_begin[0] = 0;
+    sink.tok_begin[1] = p->total_tokens;
+    sink.n_dst = 1;
+  }
+  const float* q_gain = o.q_gain;
+  const float* k_gain = o.k_gain;
+  const float eps = o.eps;
+  unsigned char* sparse_ws = o.sparse_ws;
+  const float tau = o.tau;
+  const uint8_t* query_mask = o.query_mask;
   if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
@@ -560,9 +697,9 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.pair_needed = d_pair_needed;
   ap.cta_list = d_cta_list;
   ap.cta_count = d_cta_count;
-  ap.out = out;
-  ap.o_tok_stride = p->so.tok;
-  ap.o_head_stride = p->so.head;
+  ap.sink = sink;
+  ap.o_tok_stride = o_tok_stride;
+  ap.o_head_stride = o_head_stride;
   ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));
   ap.status = reinterpret_cast<unsigned int*>(p->ws + p->off_status);
   ap.wait_limit_ns = p->wait_limit_ns;
@@ -754,7 +891,11 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
   ap.keybits = reinterpret_cast<const uint4*>(d_bits);
   ap.ktile_list = d_list;
   ap.ktile_count = d_count;
-  ap.out = out;
+  ap.sink.base[0] = out;
+  ap.sink.tok_begin[0] = 0;
+  ap.sink.tok_begin[1] = p->total_tokens;
+  ap.sink.n_dst = 1;
+  ap.sink.fmt = sol::kOutBf16;
   ap.o_tok_stride = p->so.tok;
   ap.o_head_stride = p->so.head;
   ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));

@@ -1,0 +1,132 @@
+"""Sequence-parallel attention (Section 3.3 of the paper): every rank holds a contiguous range of the flat token
+axis with all heads; attention runs head-sharded between two exchanges.
+
+Plumbing only: `torch.distributed` carries the two all-to-alls (NCCL on GPUs), every byte that moves on the
+device is moved by the library's kernels (stride-aware QKV pack, attention, inverse head merge).  One
+collective each way, as in the paper; the packed QKV receive buffer is consumed by the attention through strides,
+and the attention's own output buffer is the send buffer of the return path, so neither side makes a layout copy
+beyond the pack and the merge.
+
+Transport "peer" (optional; needs `torch.distributed._symmetric_memory`, one node): the pack kernel stores
+straight into the owners' receive buffers and the attention epilogue stores each output row straight into its
+token owner's merged buffer, so the only collectives left are two barriers.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+from . import binding as B
+
+
+def shard_ranges(total: int, n_ranks: int) -> List[Tuple[int, int]]:
+    """Contiguous token ranges per rank: ceil(total / n_ranks) tokens each, trailing ranks shorter or empty."""
+    per = (total + n_ranks - 1) // n_ranks
+    return [(min(g * per, total), min((g + 1) * per, total)) for g in range(n_ranks)]
+
+
+class ExchangePlan:
+    """Host-side description of the two all-to-alls for one rank (pure Python, no device work)."""
+
+    def __init__(self, total_tokens: int, heads: int, head_dim: int, n_ranks: int, rank: int, out_record_bytes: int):
+        if n_ranks < 1 or n_ranks > B.MAX_RANKS:
+            raise ValueError(f"1 <= n_ranks <= {B.MAX_RANKS}")
+        if heads % n_ranks:
+            raise ValueError("heads must be divisible by the number of ranks")
+        if not 0 <= rank < n_ranks:
+            raise ValueError("rank out of range")
+        self.total, self.heads, self.head_dim, self.n_ranks, self.rank = total_tokens, heads, head_dim, n_ranks, rank
+        self.hl = heads // n_ranks
+        self.ranges = shard_ranges(total_tokens, n_ranks)
+        self.tok_begin = [a for a, _ in self.ranges] + [total_tokens]
+        self.n_local = self.ranges[rank][1] - self.ranges[rank][0]
+        self.first_token = self.ranges[rank][0]
+        qkv_row = 3 * self.hl * head_dim                       # elements per token in the QKV exchange
+        # split sizes are in ELEMENTS of the exchanged tensors
+        # QKV exchange: this rank sends n_local rows to everyone and receives n_s rows from rank s
+        self.qkv_send_splits = [self.n_local * qkv_row] * n_ranks
+        self.qkv_recv_splits = [(b - a) * qkv_row for a, b in self.ranges]
+        out_row = self.hl * head_dim                           # elements per token in the output return
+        self.out_record_bytes = out_record_bytes               # bytes of one (token, head) record on the wire
+        # output return: this rank owes rows [a_g, b_g) to rank g and receives its own n_local rows from everyone
+        self.out_send_splits = [(b - a) * out_row for a, b in self.ranges]
+        self.out_recv_splits = [self.n_local * out_row] * n_ranks
+
+
+class SequenceParallelAttn3d:
+    """One DiT-block attention over a sequence-sharded Q, K, V.  forward() returns this rank's token rows."""
+
+    def __init__(self, seqs: Sequence[Tuple[int, int, int, int]], heads: int, head_dim: int, rope_dims, theta: float = 10000.0,
+                 group=None, device="cuda", out_format: str = "bf16", transport: str = "collective"):
+        import torch.distributed as dist
+        self.dist = dist
+        self.group = group
+        self.n_ranks = dist.get_world_size(group)
+        self.rank = dist.get_rank(group)
+        if out_format not in ("bf16", "e4m3"):
+            raise ValueError("out_format: 'bf16' or 'e4m3'")
+        if transport not in ("collective", "peer"):
+            raise ValueError("transport: 'collective' or 'peer'")
+        self.fp8 = out_format == "e4m3"
+        self.transport = transport
+        self.heads, self.head_dim = heads, head_dim
+        total = sum(L + T * H * W for (L, T, H, W) in seqs)
+        self.xp = ExchangePlan(total, heads, head_dim, self.n_ranks, self.rank, head_dim * (1 if self.fp8 else 2))
+        hl, D = self.xp.hl, head_dim
+        qkv_strides = (3 * hl * D, D)
+        self.attn = B.Attn3d(seqs, hl, D, rope_dims, theta, device, q_strides=qkv_strides, k_strides=qkv_strides,
+                             v_strides=qkv_strides)
+        self.out_dtype = torch.uint8 if self.fp8 else torch.bfloat16
+        n_local = self.xp.n_local
+        if transport == "collective":
+            self.qkv = torch.empty((total, 3, hl, D), dtype=torch.bfloat16, device=device)
+            self.send = torch.empty((self.n_ranks, n_local, 3, hl, D), dtype=torch.bfloat16, device=device)
+            self.out_shard = torch.empty((total, hl, D), dtype=self.out_dtype, device=device)
+            self.recv_out = torch.empty((self.n_ranks, n_local, hl, D), dtype=self.out_dtype, device=device)
+        else:
+            import torch.distributed._symmetric_memory as symm
+            per = self.xp.ranges[0][1] - self.xp.ranges[0][0]          # largest shard: same size on every rank
+            self.qkv = symm.empty((total, 3, hl, D), dtype=torch.bfloat16, device=device)
+            self.merged = symm.empty((max(per, 1), heads, D), dtype=self.out_dtype, device=device)
+            gname = (group or dist.group.WORLD).group_name
+            self.qkv_handle = symm.rendezvous(self.qkv, gname)
+            self.merged_handle = symm.rendezvous(self.merged, gname)
+            self.qkv_peers = [int(p) for p in self.qkv_handle.buffer_ptrs]
+            self.merged_peers = [int(p) for p in self.merged_handle.buffer_ptrs]
+            self._token = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def _barrier(self):
+        # stream-ordered: every rank's earlier kernels on this stream are complete when the reduction returns
+        self.dist.all_reduce(self._token, group=self.group)
+
+    def forward(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, key_mask: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q, k, v: [n_local, heads, D] bf16 (any strides, e.g. views into packed QKV); key_mask: uint8 [total] or None."""
+        xp = self.xp
+        if tuple(q.shape) != (xp.n_local, self.heads, self.head_dim):
+            raise ValueError(f"expected [{xp.n_local}, {self.heads}, {self.head_dim}] on rank {self.rank}")
+        qv, kv, vv = self.qkv[:, 0], self.qkv[:, 1], self.qkv[:, 2]
+        if self.transport == "collective":
+            B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, [self.send[g].data_ptr() for g in range(self.n_ranks)], 0)
+            self.dist.all_to_all_single(self.qkv.view(-1), self.send.view(-1), xp.qkv_recv_splits, xp.qkv_send_splits,
+                                        group=self.group)
+            if self.fp8:
+                B.sol_attn3d_forward_e4m3(self.attn.plan, qv, kv, vv, self.out_shard, key_mask)
+            else:
+                B.sol_attn3d_forward(self.attn.plan, qv, kv, vv, self.out_shard, key_mask)
+            self.dist.all_to_all_single(self.recv_out.view(-1), self.out_shard.view(-1), xp.out_recv_splits,
+                                        xp.out_send_splits, group=self.group)
+            out = torch.empty((xp.n_local, self.heads, self.head_dim), dtype=self.out_dtype, device=q.device)
+            B.sol_attn3d_exchange_merge_heads(self.recv_out, out, xp.n_local, self.heads, xp.out_record_bytes, self.n_ranks)
+            return out
+        # peer transport: stores into the owners' buffers, barriers instead of payload collectives
+        self._barrier()                                       # everyone is done reading last call's buffers
+        B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, self.qkv_peers, xp.first_token)
+        self._barrier()
+        B.sol_attn3d_forward_scatter(self.attn.plan, qv, kv, vv, key_mask, self.merged_peers, xp.tok_begin, self.heads,
+                                     self.rank * xp.hl, B.OUT_E4M3 if self.fp8 else B.OUT_BF16)
+        self._barrier()
+        return self.merged[:xp.n_local]
+
+    def close(self):
+        self.attn.close()

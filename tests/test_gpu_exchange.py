@@ -1,0 +1,297 @@
+"""GPU: E4M3 output epilogue and the sequence-parallel exchange kernels (Section 3.3 of the paper).
+
+One GPU stands in for the G ranks: their shards and buffers all live on it and the kernels of the "ranks" run one
+after another (nothing waits on anything), which exercises exactly the addresses a real run would use with peer
+pointers in place of local ones.  Layout kernels must be bit-exact against the oracle's reference permutations;
+the end-to-end result must be the single-device attention."""
+import os
+from dataclasses import replace
+
+import pytest
+import torch
+
+from oracle import attn3d_oracle as orc
+from oracle import exchange_oracle as xo
+from paper_2609_35110_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL_MAX_ABS = 2e-2
+TOL_REL_L2 = 5e-3
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2609_35110_b200 import binding
+    binding._lib()
+    return binding
+
+
+def seq_tuples(w):
+    return [(s.text_len, s.T, s.H, s.W) for s in w.seqs]
+
+
+def oracle_dense(w, inp):
+    return orc.attn3d_oracle(inp.q.cpu(), inp.k.cpu(), inp.v.cpu(), seq_tuples(w), w.rope_dims, w.theta,
+                             None if inp.key_mask is None else inp.key_mask.cpu())
+
+
+# ------------------------------------------------------------------------------------------ E4M3 epilogue
+def in_band(codes, centre, tol):
+    """The code space is monotone, so 'the value that was rounded lies within centre -/+ tol' is the same as
+    'the code lies between the encodings of centre - tol and centre + tol'."""
+    got = xo.e4m3_decode(codes)
+    lo = xo.e4m3_decode(xo.e4m3_encode(centre - tol))
+    hi = xo.e4m3_decode(xo.e4m3_encode(centre + tol))
+    return (got >= lo) & (got <= hi)
+
+
+def check_e4m3(codes: torch.Tensor, ref: torch.Tensor, bf16_out: torch.Tensor = None):
+    """codes: uint8 from the GPU; ref: fp64 oracle rows; bf16_out: the GPU's bf16 forward of the same inputs.
+
+    A float decides an integer here, so the decision is checked in the kernel's precision: the E4M3 epilogue and
+    the bf16 epilogue round the SAME fp32 value x, and bf16_out pins x to within 2^-9 relative, so the code must
+    lie between the encodings of bf16_out * (1 -/+ 2^-8) -- one code almost everywhere.  Against the fp64 oracle
+    the band is the attention's own error (measured max-abs on these inputs is 2e-3; contract 2e-2)."""
+    codes = codes.cpu()
+    got = xo.e4m3_decode(codes)
+    assert not torch.isnan(got).any()
+    stats = {}
+    if bf16_out is not None:
+        b = bf16_out.cpu().double()
+        assert bool(in_band(codes, b, b.abs() * 2.0 ** -8 + 1e-30).all()), "E4M3 code is not a rounding of the kernel's value"
+        stats["same_as_encoded_bf16"] = (codes == xo.e4m3_encode(b)).double().mean().item()
+        assert stats["same_as_encoded_bf16"] > 0.95, stats   # bf16-then-E4M3 double rounding differs ~3 % of the time
+    tol = 5e-3 * ref.abs() + 3e-3
+    assert bool(in_band(codes, ref, tol).all()), "E4M3 code outside the band allowed by the attention tolerance"
+    stats["same_as_encoded_oracle"] = (codes == xo.e4m3_encode(ref)).double().mean().item()
+    assert stats["same_as_encoded_oracle"] > 0.8, stats
+    # and as numbers: half a step of a 3-bit mantissa, or half a subnormal step, plus the attention tolerance
+    assert bool(((got - ref).abs() <= ref.abs() * 2.0 ** -4 + 2.0 ** -10 + tol).all())
+    return stats
+
+
+@pytest.mark.parametrize("name", ["tiny", "lowres", "cfg_batch", "varlen"])
+def test_e4m3_output_matches_encoded_oracle(B, name):
+    w = wl.shrunk(name)
+    inp = wl.make_inputs(w, "cuda")
+    attn = B.Attn3d.from_workload(w, "cuda")
+    n = w.total_tokens * w.heads * w.head_dim
+    guard = 4096
+    buf = torch.full((n + 2 * guard,), 0x7F, dtype=torch.uint8, device="cuda")      # NaN code: unwritten rows show up
+    out = buf[guard:guard + n].view(w.total_tokens, w.heads, w.head_dim)
+    B.sol_attn3d_forward_e4m3(attn.plan, inp.q, inp.k, inp.v, out, inp.key_mask)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert bool((buf[:guard] == 0x7F).all()) and bool((buf[-guard:] == 0x7F).all()), "store outside the output tensor"
+    # the same call twice gives the same bytes, and the bf16 forward of the same plan still works afterwards
+    out2 = torch.empty_like(out)
+    B.sol_attn3d_forward_e4m3(attn.plan, inp.q, inp.k, inp.v, out2, inp.key_mask)
+    ob = attn.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    print(name, check_e4m3(out, oracle_dense(w, inp), ob))
+    attn.close()
+
+
+def test_e4m3_saturates_and_keeps_signs(B):
+    # V = +-1000 everywhere: every output is +-1000 exactly in fp32, far above 448 -> saturated codes 0x7e / 0xfe
+    w = wl.shrunk("tiny")
+    inp = wl.make_inputs(w, "cuda")
+    v = torch.full_like(inp.v, 1000.0)
+    v[:, 1::2] = -1000.0
+    attn = B.Attn3d.from_workload(w, "cuda")
+    out = torch.empty((w.total_tokens, w.heads, w.head_dim), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_forward_e4m3(attn.plan, inp.q, inp.k, v, out, None)
+    torch.cuda.synchronize()
+    assert bool((out[:, 0::2] == 0x7E).all()) and bool((out[:, 1::2] == 0xFE).all())
+    attn.close()
+
+
+# ------------------------------------------------------------------------------------------ layout kernels
+@pytest.mark.parametrize("G,n_local,heads,D", [(2, 300, 8, 128), (4, 77, 8, 64), (8, 33, 40, 128), (1, 10, 3, 64), (3, 0, 6, 64)])
+def test_pack_qkv_is_the_reference_permutation(B, G, n_local, heads, D):
+    g = torch.Generator(device="cuda").manual_seed(100 + G)
+    # Q, K, V as views into one packed QKV buffer (token stride 3*heads*D), as the paper's packed storage
+    packed = torch.randn((max(n_local, 1), 3, heads, D), generator=g, device="cuda").to(torch.bfloat16)[:n_local]
+    q, k, v = packed[:, 0], packed[:, 1], packed[:, 2]
+    hl = heads // G
+    send = torch.full((G, n_local, 3, hl, D), -7.0, dtype=torch.bfloat16, device="cuda")
+    dummy = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_pack_qkv(q, k, v, G, [send[r].data_ptr() if n_local else dummy.data_ptr() for r in range(G)], 0)
+    torch.cuda.synchronize()
+    want = xo.pack_qkv_reference(q.cpu(), k.cpu(), v.cpu(), G)
+    assert torch.equal(send.cpu().view(torch.int16), want.view(torch.int16))
+    # contiguous inputs give the same bytes
+    if n_local:
+        send2 = torch.empty_like(send)
+        B.sol_attn3d_exchange_pack_qkv(q.contiguous(), k.contiguous(), v.contiguous(), G, [send2[r].data_ptr() for r in range(G)], 0)
+        torch.cuda.synchronize()
+        assert torch.equal(send2, send)
+
+
+@pytest.mark.parametrize("G,n_local,heads,record", [(2, 300, 8, 256), (4, 77, 8, 128), (8, 33, 40, 144), (1, 5, 3, 64), (2, 129, 4, 16)])
+def test_merge_heads_is_the_reference_permutation(B, G, n_local, heads, record):
+    g = torch.Generator(device="cuda").manual_seed(200 + G)
+    hl = heads // G
+    recv = torch.randint(0, 256, (G, n_local, hl, record), generator=g, device="cuda", dtype=torch.uint8)
+    pad = 32                                                    # output rows with a stride larger than dense
+    out = torch.full((n_local, heads * record + pad), 0xAB, dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_merge_heads(recv, out, n_local, heads, record, G, out.stride(0))
+    torch.cuda.synchronize()
+    want = xo.merge_heads_reference(recv.cpu())
+    assert torch.equal(out[:, :heads * record].cpu().view(n_local, heads, record), want)
+    assert bool((out[:, heads * record:] == 0xAB).all())
+    dense = torch.empty((n_local, heads, record), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_merge_heads(recv, dense, n_local, heads, record, G)
+    torch.cuda.synchronize()
+    assert torch.equal(dense.cpu(), want)
+
+
+def test_exchange_entry_points_reject_bad_arguments(B):
+    x = torch.zeros((4, 6, 64), dtype=torch.bfloat16, device="cuda")
+    dst = torch.zeros(4 * 3 * 6 * 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.SolAttn3dError):
+        B.sol_attn3d_exchange_pack_qkv(x, x, x, 4, [dst.data_ptr()] * 4, 0)                 # 6 heads, 4 ranks
+    with pytest.raises(B.SolAttn3dError):
+        B.sol_attn3d_exchange_pack_qkv(x, x, x, 2, [dst.data_ptr(), dst.data_ptr() + 2], 0)  # misaligned destination
+    r = torch.zeros((2, 4, 3, 40), dtype=torch.uint8, device="cuda")
+    o = torch.zeros((4, 6, 40), dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.SolAttn3dError):
+        B.sol_attn3d_exchange_merge_heads(r, o, 4, 6, 40, 2)                                # record not a multiple of 16
+
+
+# ------------------------------------------------------------------------------------------ the whole exchange
+def virtual_ranks_forward(B, w, inp, G, fmt, peer_style):
+    """All G ranks on this GPU, one after another.  Returns the per-rank merged outputs [n_r, heads, D]."""
+    total, heads, D = w.total_tokens, w.heads, w.head_dim
+    hl = heads // G
+    ranges = xo.shard_ranges(total, G)
+    tok_begin = [a for a, _ in ranges] + [total]
+    out_dtype = torch.uint8 if fmt == B.OUT_E4M3 else torch.bfloat16
+    qkv = [torch.full((total, 3, hl, D), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(G)]
+    # (1) QKV exchange
+    if peer_style:
+        for s, (a, b) in enumerate(ranges):                    # rank s stores straight into every owner's buffer
+            B.sol_attn3d_exchange_pack_qkv(inp.q[a:b], inp.k[a:b], inp.v[a:b], G, [t.data_ptr() for t in qkv], a)
+    else:
+        for s, (a, b) in enumerate(ranges):
+            send = torch.empty((G, b - a, 3, hl, D), dtype=torch.bfloat16, device="cuda")
+            B.sol_attn3d_exchange_pack_qkv(inp.q[a:b], inp.k[a:b], inp.v[a:b], G,
+                                           [send[r].data_ptr() if b > a else qkv[0].data_ptr() for r in range(G)], 0)
+            for r in range(G):                                 # the all-to-all, by hand
+                qkv[r][a:b] = send[r]
+    for r in range(G):                                         # every rank now holds its head shard of everything
+        for wh, full in enumerate((inp.q, inp.k, inp.v)):
+            assert torch.equal(qkv[r][:, wh], full[:, r * hl:(r + 1) * hl])
+    # (2) head-sharded attention, (3) output return + merge
+    strides = (3 * hl * D, D)
+    merged = [torch.full((b - a, heads, D), 0x7F if fmt == B.OUT_E4M3 else float("nan"), dtype=out_dtype, device="cuda")
+              for (a, b) in ranges]
+    recv = [torch.empty((G, b - a, hl, D), dtype=out_dtype, device="cuda") for (a, b) in ranges]
+    for r in range(G):
+        attn = B.Attn3d(seq_tuples(w), hl, D, w.rope_dims, w.theta, "cuda", q_strides=strides, k_strides=strides, v_strides=strides)
+        qv, kv, vv = qkv[r][:, 0], qkv[r][:, 1], qkv[r][:, 2]
+        if peer_style:
+            B.sol_attn3d_forward_scatter(attn.plan, qv, kv, vv, inp.key_mask, [m.data_ptr() if m.numel() else 0 for m in merged],
+                                         tok_begin, heads, r * hl, fmt)
+        else:
+            shard = torch.empty((total, hl, D), dtype=out_dtype, device="cuda")
+            if fmt == B.OUT_E4M3:
+                B.sol_attn3d_forward_e4m3(attn.plan, qv, kv, vv, shard, inp.key_mask)
+            else:
+                B.sol_attn3d_forward(attn.plan, qv, kv, vv, shard, inp.key_mask)
+            for o, (a, b) in enumerate(ranges):                # the all-to-all, by hand
+                recv[o][r] = shard[a:b]
+        torch.cuda.synchronize()
+        assert attn.status() == 0
+        attn.close()
+    if not peer_style:
+        for o, (a, b) in enumerate(ranges):
+            B.sol_attn3d_exchange_merge_heads(recv[o], merged[o], b - a, heads, D * merged[o].element_size(), G)
+    torch.cuda.synchronize()
+    return merged
+
+
+@pytest.mark.parametrize("name,heads,G", [("tiny", 4, 2), ("lowres", 8, 4), ("lowres", 8, 8), ("cfg_batch", 4, 2), ("varlen", 6, 3)])
+@pytest.mark.parametrize("peer_style", [False, True])
+def test_exchange_returns_the_single_device_attention(B, name, heads, G, peer_style):
+    w = replace(wl.shrunk(name), heads=heads)
+    inp = wl.make_inputs(w, "cuda")
+    single = B.Attn3d.from_workload(w, "cuda")
+    want = single.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    torch.cuda.synchronize()
+    single.close()
+    merged = virtual_ranks_forward(B, w, inp, G, B.OUT_BF16, peer_style)
+    got = torch.cat(merged, dim=0)
+    # heads are independent and a CTA's arithmetic does not depend on the grid around it: bit-identical
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    max_abs, rel_l2 = orc.compare(got.cpu(), oracle_dense(w, inp))
+    assert max_abs <= TOL_MAX_ABS and rel_l2 <= TOL_REL_L2, (max_abs, rel_l2)
+
+
+@pytest.mark.parametrize("peer_style", [False, True])
+def test_exchange_with_e4m3_return(B, peer_style):
+    w = replace(wl.shrunk("lowres"), heads=8)
+    inp = wl.make_inputs(w, "cuda")
+    merged = virtual_ranks_forward(B, w, inp, 4, B.OUT_E4M3, peer_style)
+    got = torch.cat(merged, dim=0)
+    check_e4m3(got, oracle_dense(w, inp))
+    single = B.Attn3d.from_workload(w, "cuda")
+    want = torch.empty((w.total_tokens, w.heads, w.head_dim), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_forward_e4m3(single.plan, inp.q, inp.k, inp.v, want, inp.key_mask)
+    torch.cuda.synchronize()
+    assert torch.equal(got, want)
+    single.close()
+
+
+def test_scatter_rejects_bad_arguments(B):
+    w = wl.shrunk("tiny")
+    inp = wl.make_inputs(w, "cuda")
+    attn = B.Attn3d.from_workload(w, "cuda")
+    total = w.total_tokens
+    buf = torch.empty((total, w.heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
+    ok = [buf.data_ptr()]
+    with pytest.raises(B.SolAttn3dError):
+        B.sol_attn3d_forward_scatter(attn.plan, inp.q, inp.k, inp.v, None, ok, [0, total - 1], w.heads, 0)   # does not cover
+    with pytest.raises(B.SolAttn3dError):
+        B.sol_attn3d_forward_scatter(attn.plan, inp.q, inp.k, inp.v, None, ok, [0, total], w.heads - 1, 0)   # rows too narrow
+    with pytest.raises(B.SolAttn3dError):
+        B.sol_attn3d_forward_scatter(attn.plan, inp.q, inp.k, inp.v, None, [0], [0, total], w.heads, 0)      # NULL owner with rows
+    with pytest.raises(B.SolAttn3dError):
+        B.sol_attn3d_forward_scatter(attn.plan, inp.q, inp.k, inp.v, None, ok, [0, total], w.heads, 0, 7)    # unknown format
+    B.sol_attn3d_forward_scatter(attn.plan, inp.q, inp.k, inp.v, None, ok, [0, total], w.heads, 0)
+    torch.cuda.synchronize()
+    want = attn.forward(inp.q, inp.k, inp.v, None)
+    torch.cuda.synchronize()
+    assert torch.equal(buf, want)
+    attn.close()
+
+
+def test_sequence_parallel_module_with_one_rank(B):
+    """The torch.distributed plumbing itself (NCCL all-to-all with a single rank is a device copy)."""
+    import torch.distributed as dist
+    from paper_2609_35110_b200.sequence_parallel import SequenceParallelAttn3d
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", str(29400 + os.getpid() % 500))
+    created = False
+    if not dist.is_initialized():
+        dist.init_process_group("nccl", rank=0, world_size=1)
+        created = True
+    try:
+        w = wl.shrunk("cfg_batch")
+        inp = wl.make_inputs(w, "cuda")
+        single = B.Attn3d.from_workload(w, "cuda")
+        want = single.forward(inp.q, inp.k, inp.v, inp.key_mask)
+        sp = SequenceParallelAttn3d(seq_tuples(w), w.heads, w.head_dim, w.rope_dims, w.theta)
+        got = sp.forward(inp.q, inp.k, inp.v, inp.key_mask)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
+        sp8 = SequenceParallelAttn3d(seq_tuples(w), w.heads, w.head_dim, w.rope_dims, w.theta, out_format="e4m3")
+        got8 = sp8.forward(inp.q, inp.k, inp.v, inp.key_mask)
+        torch.cuda.synchronize()
+        check_e4m3(got8, oracle_dense(w, inp))
+        sp.close(); sp8.close(); single.close()
+    finally:
+        if created:
+            dist.destroy_process_group()
