@@ -24,9 +24,13 @@ What it states (Section 3.3 of the paper, "Optimized attention collectives", "Qu
       included) saturate to +-448, NaN -> 0x7f.  (The paper fixes the format, not the rounding rule; this
       is the rule of the hardware conversion instruction and of the OCP text's "saturating" mode.)
 
+  X8-X11  the block-INT8 wire formats: see the comment block above ue5m3_decode.
+
 Pins: tests/test_oracle_pins_exchange.py (code table values, round trip of all codes, ties, nearest-code brute
-force, the library cast as a special case; permutation brute force, exchange-then-merge identity, and the
-end-to-end identity X6 on a tiny problem).
+force, the library cast as a special case; permutation brute force, exchange-then-merge identity, the
+end-to-end identity X6 on a tiny problem; for the block-INT8 formats: scale-table constants, smallest-scale rule
+by brute force and at exact boundaries, error bound, power-of-two scaling and sign symmetries, byte positions of a
+hand-made record).
 """
 from __future__ import annotations
 
@@ -133,3 +137,110 @@ def ulysses_reference(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, G: int,
         stacked = torch.stack([back[s][g] for s in range(G)], dim=0)  # [G, n_g, heads/G, D]
         merged.append(merge_heads_reference(stacked))
     return merged
+
+
+# --------------------------------------------------------------------------------------------- block-INT8 wire formats
+#
+# Section 3.3, "Quantized communication".  What the paper fixes: the QKV record of one (token, head) is 384 int8
+# values, twelve scale codes (one per group of 32 values, "finite-positive UE5M3"), four zero bytes = 400 bytes; the
+# output record is 128 values, four scale codes, padded from 132 to 144 bytes; all padding bytes are written.
+# What it leaves open, and the reading taken here (X8-X11):
+#   X8   UE5M3 = unsigned 8-bit float, 5 exponent bits (bias 15), 3 mantissa bits: code c, e = c >> 3, m = c & 7,
+#        value (8 + m) * 2^(e - 18) for 1 <= e <= 30 and m * 2^-17 for e = 0; e = 31 is reserved.  "Finite-positive":
+#        only codes 0x01 .. 0xf7 are ever produced;
+#   X9   the scale of a group is the SMALLEST such value s with 127 * s >= max|x| (nothing clips; 127 * s is exact in
+#        fp32 and fp64, so the choice does not depend on the precision it is made in); an all-zero group gets 0x01;
+#   X10  q = clamp(round_half_even(x * (1 / s)), -127, 127) with the reciprocal and the product each rounded to
+#        fp32: a float decides an integer here, so the decision is taken in the kernel's precision (IEEE fp32,
+#        round to nearest) and is reproducible bit for bit; dequantised value = q * s (exact in fp32);
+#   X11  record layout, head_dim D (D = 128 in the paper): [q values D | k values D | v values D | D/32 q codes |
+#        D/32 k codes | D/32 v codes | zeros up to a multiple of 16 bytes] (396 -> 400); output record [values D |
+#        D/32 codes | zeros up to a multiple of 16 bytes] (132 -> 144, "to align each record to 16 bytes").
+
+GROUP = 32
+
+
+def ue5m3_decode(codes: torch.Tensor) -> torch.Tensor:
+    c = codes.to(torch.int64)
+    e = c >> 3
+    m = (c & 7).to(torch.float64)
+    normal = torch.ldexp(8.0 + m, (e - 18).to(torch.int32))
+    sub = m * 2.0 ** -17
+    val = torch.where(e == 0, sub, normal)
+    return torch.where(e == 31, torch.full_like(val, float("nan")), val)
+
+
+def ue5m3_encode_up(bound127: torch.Tensor) -> torch.Tensor:
+    """Smallest code in 0x01..0xf7 whose value s satisfies 127 * s >= bound127 (X9)."""
+    table = ue5m3_decode(torch.arange(1, 0xF8, dtype=torch.uint8)) * 127.0      # ascending, exact
+    idx = torch.searchsorted(table, bound127.to(torch.float64).contiguous(), right=False)
+    return (torch.clamp(idx, max=table.numel() - 1) + 1).to(torch.uint8)
+
+
+def block_int8_quantize(x: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """x [..., D] (D a multiple of 32) -> (int8 values [..., D], uint8 scale codes [..., D/32])  (X9, X10)."""
+    D = x.shape[-1]
+    xg = x.to(torch.float64).reshape(*x.shape[:-1], D // GROUP, GROUP)
+    amax = xg.abs().amax(dim=-1)
+    codes = ue5m3_encode_up(amax)
+    s32 = ue5m3_decode(codes).to(torch.float32)
+    inv = torch.reciprocal(s32)                                                  # fp32, round to nearest
+    q = torch.round(xg.to(torch.float32) * inv[..., None])                      # fp32 product, half-even
+    q = torch.clamp(q, -127.0, 127.0).to(torch.int8)
+    return q.reshape(x.shape), codes
+
+
+def block_int8_dequantize(q: torch.Tensor, codes: torch.Tensor) -> torch.Tensor:
+    D = q.shape[-1]
+    s = ue5m3_decode(codes)
+    return (q.to(torch.float64).reshape(*q.shape[:-1], D // GROUP, GROUP) * s[..., None]).reshape(q.shape)
+
+
+def _padded(n: int) -> int:
+    return (n + 15) // 16 * 16
+
+
+def qkv_record_bytes(D: int) -> int:
+    return _padded(3 * D + 3 * D // GROUP)
+
+
+def out_record_bytes(D: int) -> int:
+    return _padded(D + D // GROUP)
+
+
+def qkv_records(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor) -> torch.Tensor:
+    """[n, heads, D] x 3 -> uint8 [n, heads, qkv_record_bytes(D)]  (X11)."""
+    n, heads, D = q.shape
+    rec = torch.zeros((n, heads, qkv_record_bytes(D)), dtype=torch.uint8)
+    ng = D // GROUP
+    for w, x in enumerate((q, k, v)):
+        vals, codes = block_int8_quantize(x)
+        rec[:, :, w * D:(w + 1) * D] = vals.view(torch.uint8)
+        rec[:, :, 3 * D + w * ng:3 * D + (w + 1) * ng] = codes
+    return rec
+
+
+def qkv_from_records(rec: torch.Tensor, D: int) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """uint8 records -> dequantised q, k, v in fp64 (each value is exactly representable in fp32)."""
+    ng = D // GROUP
+    out = []
+    for w in range(3):
+        vals = rec[..., w * D:(w + 1) * D].contiguous().view(torch.int8)
+        codes = rec[..., 3 * D + w * ng:3 * D + (w + 1) * ng]
+        out.append(block_int8_dequantize(vals, codes))
+    return tuple(out)
+
+
+def out_records(o: torch.Tensor) -> torch.Tensor:
+    """[n, heads, D] -> uint8 [n, heads, out_record_bytes(D)]  (X11)."""
+    n, heads, D = o.shape
+    rec = torch.zeros((n, heads, out_record_bytes(D)), dtype=torch.uint8)
+    vals, codes = block_int8_quantize(o)
+    rec[:, :, :D] = vals.view(torch.uint8)
+    rec[:, :, D:D + D // GROUP] = codes
+    return rec
+
+
+def out_from_records(rec: torch.Tensor, D: int) -> torch.Tensor:
+    vals = rec[..., :D].contiguous().view(torch.int8)
+    return block_int8_dequantize(vals, rec[..., D:D + D // GROUP])

@@ -153,3 +153,104 @@ def test_exchange_around_the_attention_equals_single_device_attention():
         got = torch.cat(outs, dim=0)
         assert got.shape == full.shape
         assert (got - full).abs().max().item() < 1e-13
+
+
+# ------------------------------------------------------------------------------------------------ block-INT8
+def test_ue5m3_table_constants_and_order():
+    dec = xo.ue5m3_decode(torch.arange(256, dtype=torch.uint8))
+    assert dec[0x78].item() == 1.0                     # e = 15, m = 0
+    assert dec[0x7C].item() == 1.5 and dec[0x80].item() == 2.0
+    assert dec[0x01].item() == 2.0 ** -17 and dec[0x07].item() == 7 * 2.0 ** -17
+    assert dec[0x08].item() == 2.0 ** -14              # first normal continues the subnormal ladder
+    assert dec[0xF7].item() == 15 * 2.0 ** 12 == 61440.0
+    assert dec[0x00].item() == 0.0 and torch.isnan(dec[0xF8:]).all()
+    pos = dec[1:0xF8]
+    assert (pos[1:] > pos[:-1]).all()
+    # neighbouring values are never more than 9/8 apart once normal: the scale wastes at most 12.5 % of the range
+    assert ((pos[8:] / pos[7:-1]).max().item() <= 9.0 / 8.0 + 1e-15)
+
+
+def test_ue5m3_encode_up_brute_force_and_boundaries():
+    table = [xo.ue5m3_decode(torch.tensor([c], dtype=torch.uint8)).item() for c in range(1, 0xF8)]
+    g = torch.Generator().manual_seed(2)
+    amax = torch.cat([torch.rand(300, generator=g, dtype=F64) * s for s in (1e-6, 1e-3, 1.0, 50.0, 5e4)])
+    amax = torch.cat([amax, torch.tensor([0.0, 127.0, 127.0 * 1.125, 127.0 * 2.0 ** -17, 1e9], dtype=F64)])
+    got = xo.ue5m3_encode_up(amax).tolist()
+    for a, c in zip(amax.tolist(), got):
+        want = next((i + 1 for i, v in enumerate(table) if 127.0 * v >= a), 0xF7)
+        assert c == want, (a, c, want)
+    # exactly on a grid point -> that point; one ulp above -> the next one
+    for c in (0x01, 0x08, 0x40, 0x78, 0x7F, 0xF6):
+        on = 127.0 * table[c - 1]
+        assert xo.ue5m3_encode_up(torch.tensor([on], dtype=F64)).item() == c
+        assert xo.ue5m3_encode_up(torch.tensor([math.nextafter(on, math.inf)], dtype=F64)).item() == c + 1
+
+
+def test_block_int8_error_bound_range_use_and_symmetries():
+    g = torch.Generator().manual_seed(4)
+    x = (torch.randn(64, 3, 128, generator=g) * torch.tensor([0.01, 1.0, 40.0])[None, :, None]).to(torch.bfloat16)
+    x[0, 0, :32] = 0                                                  # an all-zero group
+    q, codes = xo.block_int8_quantize(x)
+    assert q.dtype == torch.int8 and codes.dtype == torch.uint8 and codes.shape == (64, 3, 4)
+    assert int(q.to(torch.int32).abs().max()) <= 127 and int(codes.min()) >= 1 and int(codes.max()) <= 0xF7
+    assert codes[0, 0, 0].item() == 1 and not q[0, 0, :32].any()
+    s = xo.ue5m3_decode(codes)
+    xg = x.to(F64).reshape(64, 3, 4, 32)
+    amax = xg.abs().amax(-1)
+    # smallest scale that does not clip: 127 s >= amax, and the next smaller scale would clip
+    assert bool((127.0 * s >= amax).all())
+    prev = xo.ue5m3_decode((codes.to(torch.int64) - 1).clamp(min=0).to(torch.uint8))
+    assert bool(((127.0 * prev < amax) | (codes == 1)).all())
+    # rounding error at most half a step (+ fp32 rounding of the product), the largest element uses >= 8/9 of the range
+    deq = xo.block_int8_dequantize(q, codes)
+    err = (deq - x.to(F64)).reshape(64, 3, 4, 32).abs()
+    assert bool((err <= s[..., None] * (0.5 + 1e-5)).all())
+    qmax = q.to(torch.int32).reshape(64, 3, 4, 32).abs().amax(-1)
+    assert bool(((qmax >= 112) | (amax == 0) | (codes <= 8)).all())
+    # x -> 2^k x: same integers, codes move by 8 k (every step is exact for powers of two)
+    q2, c2 = xo.block_int8_quantize((x.to(F64) * 8.0).to(torch.bfloat16))
+    keep = (codes > 8) & (amax > 0)                                       # away from the subnormal codes
+    assert torch.equal(q2.reshape(64, 3, 4, 32)[keep], q.reshape(64, 3, 4, 32)[keep])
+    assert torch.equal(c2[keep].to(torch.int64), codes[keep].to(torch.int64) + 24)
+    # x -> -x: integers negate, codes stay
+    q3, c3 = xo.block_int8_quantize(-x)
+    assert torch.equal(q3, -q) and torch.equal(c3, codes)
+
+
+def test_block_int8_hand_made_group():
+    # amax = 127 -> s = 1 exactly (code 0x78) and q = x for integers; amax = 128 -> next scale 1.125 (0x79)
+    x = torch.zeros(1, 32, dtype=F64)
+    x[0, :5] = torch.tensor([127.0, -3.0, 2.5, 3.5, -0.5])
+    q, c = xo.block_int8_quantize(x)
+    assert c.item() == 0x78 and q[0, :5].tolist() == [127, -3, 2, 4, 0]            # ties to even: 2.5 -> 2, 3.5 -> 4, -0.5 -> 0
+    x[0, 0] = 128.0
+    q, c = xo.block_int8_quantize(x)
+    assert c.item() == 0x79 and q[0, 0].item() == 114                              # 128 / 1.125 = 113.78
+
+
+def test_record_layouts_byte_for_byte():
+    assert xo.qkv_record_bytes(128) == 400 and xo.out_record_bytes(128) == 144     # the paper's sizes
+    assert xo.qkv_record_bytes(64) == 208 and xo.out_record_bytes(64) == 80
+    D = 128
+    q = torch.zeros(2, 3, D, dtype=F64); k = torch.zeros_like(q); v = torch.zeros_like(q)
+    q[1, 2, 0] = 127.0            # group 0 of q: scale 1, value 127
+    q[1, 2, 33] = -254.0          # group 1 of q: scale 2 (0x80), value -127
+    k[1, 2, 127] = 63.5           # group 3 of k: scale 0.5 (0x70), value 127
+    v[1, 2, 64] = 1.0             # group 2 of v: smallest s with 127 s >= 1: 2^-7 * 1.125 = 0.0087890625 (0x41): q = 114
+    rec = xo.qkv_records(q, k, v)
+    assert rec.shape == (2, 3, 400) and rec.dtype == torch.uint8
+    r = rec[1, 2].tolist()
+    assert r[0] == 127 and r[33] == 0x81 and r[128 + 127] == 127 and r[256 + 64] == 114
+    assert r[384:388] == [0x78, 0x80, 0x01, 0x01]
+    assert r[388:392] == [0x01, 0x01, 0x01, 0x70]
+    assert r[392:396] == [0x01, 0x01, 0x41, 0x01]
+    assert r[396:400] == [0, 0, 0, 0]
+    assert not rec[0].view(-1)[:384].any()                                         # other records: zero values, code 1
+    dq, dk, dv = xo.qkv_from_records(rec, D)
+    assert dq[1, 2, 0].item() == 127.0 and dq[1, 2, 33].item() == -254.0 and dk[1, 2, 127].item() == 63.5
+    assert abs(dv[1, 2, 64].item() - 1.0) <= 0.0087890625 / 2
+    orec = xo.out_records(q)
+    assert orec.shape == (2, 3, 144)
+    ro = orec[1, 2].tolist()
+    assert ro[0] == 127 and ro[33] == 0x81 and ro[128:132] == [0x78, 0x80, 0x01, 0x01] and ro[132:144] == [0] * 12
+    assert torch.equal(xo.out_from_records(orec, D), xo.block_int8_dequantize(*xo.block_int8_quantize(q)))
