@@ -220,6 +220,55 @@ int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local
                                     int n_ranks, int64_t out_tok_stride_bytes, sol_attn3d_stream_t stream);
 
 /*
+ * Quantized wire formats of the exchange (Section 3.3, "Quantized communication").  One record per (token,
+ * head); head_dim 64 or 128:
+ *   QKV block-INT8   [q int8 x D | k int8 x D | v int8 x D | D/32 q scale codes | D/32 k codes | D/32 v codes |
+ *                    zeros to a multiple of 16 bytes]                      D = 128: 384 + 12 + 4 = 400 bytes
+ *   out block-INT8   [o int8 x D | D/32 scale codes | zeros to a multiple of 16 bytes]   D = 128: 144 bytes
+ *   out E4M3         D raw bytes (sol_attn3d_forward_e4m3 writes them; no kernel here)
+ * Scale code: unsigned 8-bit float, 5 exponent bits (bias 15), 3 mantissa bits (value (8+m) * 2^(e-18), or
+ * m * 2^-17 for e = 0), one per group of 32 values; only finite positive codes 0x01..0xf7 are written.  The
+ * paper fixes the record sizes and the scale format; the rule is this library's: scale = smallest value s with
+ * 127 * s >= max|x| of the group (nothing clips; all-zero group -> 0x01), q = clamp(rint(x * (1/s)), -127, 127)
+ * with the reciprocal and the product rounded to fp32 (round to nearest even), value = q * s.  All padding
+ * bytes are written.  Both formats are approximate.
+ */
+#define SOL_ATTN3D_WIRE_QKV_BF16 0
+#define SOL_ATTN3D_WIRE_QKV_INT8 1
+#define SOL_ATTN3D_WIRE_OUT_BF16 2
+#define SOL_ATTN3D_WIRE_OUT_E4M3 3
+#define SOL_ATTN3D_WIRE_OUT_INT8 4
+/* Bytes of one (token, head) record of the given kind; 0 for an unknown kind or head_dim. */
+size_t sol_attn3d_exchange_record_bytes(int kind, int head_dim);
+
+/*
+ * sol_attn3d_exchange_pack_qkv that quantises on the way: same arguments and destinations, but destination g
+ * receives records  dst[g][dst_row0 + t][heads/n_ranks][record_bytes(QKV_INT8)]  (one pass: bf16 in, records out).
+ */
+int sol_attn3d_exchange_pack_qkv_int8(const void* q, const void* k, const void* v, const int64_t q_strides[2],
+                                      const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
+                                      int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
+                                      sol_attn3d_stream_t stream);
+
+/*
+ * Receiver's side: records [n_rows][heads][record_bytes(QKV_INT8)] (DEVICE; heads = this rank's shard) -> qkv
+ * bf16 [n_rows][3][heads][head_dim] (DEVICE, 16-byte aligned, caller-owned), the packed tensor whose three
+ * strided views feed sol_attn3d_forward.  q * s is exact in fp32 and rounded once to bf16.
+ */
+int sol_attn3d_exchange_unpack_qkv_int8(const void* records, void* qkv, int64_t n_rows, int heads, int head_dim,
+                                        sol_attn3d_stream_t stream);
+
+/*
+ * Output rows bf16 [n_rows][heads][head_dim] (element strides {token, head}, {0,0} = dense) -> records
+ * [n_rows][heads][record_bytes(OUT_INT8)]; and back to dense bf16 rows.  Records travel through
+ * sol_attn3d_exchange_merge_heads like any other record (record_bytes = 144 for head_dim 128).
+ */
+int sol_attn3d_exchange_quantize_out_int8(const void* out_rows, const int64_t out_strides[2], int64_t n_rows, int heads,
+                                          int head_dim, void* records, sol_attn3d_stream_t stream);
+int sol_attn3d_exchange_dequantize_out_int8(const void* records, void* out_rows, int64_t n_rows, int heads, int head_dim,
+                                            sol_attn3d_stream_t stream);
+
+/*
  * sol_attn3d_forward whose epilogue delivers each output row to the owner of its token: the output return
  * of the exchange and the head merge fused into the attention kernel (no counterpart kernel in the paper,
  * which returns the output with a collective; same result).  The plan describes this rank's head shard

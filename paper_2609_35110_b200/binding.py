@@ -97,6 +97,16 @@ def _lib():
     lib.sol_attn3d_exchange_pack_qkv.restype = i32
     lib.sol_attn3d_exchange_merge_heads.argtypes = [vp, vp, i64, i32, i32, i32, i64, vp]
     lib.sol_attn3d_exchange_merge_heads.restype = i32
+    lib.sol_attn3d_exchange_record_bytes.argtypes = [i32, i32]
+    lib.sol_attn3d_exchange_record_bytes.restype = ctypes.c_size_t
+    lib.sol_attn3d_exchange_pack_qkv_int8.argtypes = lib.sol_attn3d_exchange_pack_qkv.argtypes
+    lib.sol_attn3d_exchange_pack_qkv_int8.restype = i32
+    lib.sol_attn3d_exchange_unpack_qkv_int8.argtypes = [vp, vp, i64, i32, i32, vp]
+    lib.sol_attn3d_exchange_unpack_qkv_int8.restype = i32
+    lib.sol_attn3d_exchange_quantize_out_int8.argtypes = [vp, ctypes.POINTER(i64), i64, i32, i32, vp, vp]
+    lib.sol_attn3d_exchange_quantize_out_int8.restype = i32
+    lib.sol_attn3d_exchange_dequantize_out_int8.argtypes = [vp, vp, i64, i32, i32, vp]
+    lib.sol_attn3d_exchange_dequantize_out_int8.restype = i32
     lib.sol_attn3d_sparse_workspace_bytes.argtypes = [vp]
     lib.sol_attn3d_sparse_workspace_bytes.restype = ctypes.c_size_t
     lib.sol_attn3d_forward_sparse.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp]
@@ -287,6 +297,55 @@ def sol_attn3d_exchange_pack_qkv(q, k, v, n_ranks: int, dst: Sequence[int], dst_
                                                _strides_of(v, head_dim), n_local, heads, head_dim, n_ranks,
                                                _ptr_array(dst), dst_row0, _stream(stream)),
            "sol_attn3d_exchange_pack_qkv")
+
+
+WIRE_QKV_BF16, WIRE_QKV_INT8, WIRE_OUT_BF16, WIRE_OUT_E4M3, WIRE_OUT_INT8 = 0, 1, 2, 3, 4
+
+
+def sol_attn3d_exchange_record_bytes(kind: int, head_dim: int) -> int:
+    n = int(_lib().sol_attn3d_exchange_record_bytes(kind, head_dim))
+    if n == 0:
+        raise ValueError("unknown wire format or head_dim")
+    return n
+
+
+def sol_attn3d_exchange_pack_qkv_int8(q, k, v, n_ranks: int, dst: Sequence[int], dst_row0: int = 0, stream=None) -> None:
+    """As sol_attn3d_exchange_pack_qkv, but the destinations receive block-INT8 records."""
+    n_local, heads, head_dim = q.shape
+    for t in (q, k, v):
+        if not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != (n_local, heads, head_dim):
+            raise ValueError("q, k, v must be CUDA bf16 tensors of one shape")
+    if len(dst) != n_ranks:
+        raise ValueError("one destination per rank")
+    _check(_lib().sol_attn3d_exchange_pack_qkv_int8(_ptr(q), _ptr(k), _ptr(v), _strides_of(q, head_dim),
+                                                    _strides_of(k, head_dim), _strides_of(v, head_dim), n_local, heads,
+                                                    head_dim, n_ranks, _ptr_array(dst), dst_row0, _stream(stream)),
+           "sol_attn3d_exchange_pack_qkv_int8")
+
+
+def sol_attn3d_exchange_unpack_qkv_int8(records: torch.Tensor, qkv: torch.Tensor, n_rows: int, heads: int, head_dim: int,
+                                        stream=None) -> None:
+    if not records.is_cuda or not qkv.is_cuda or qkv.dtype != torch.bfloat16 or not qkv.is_contiguous():
+        raise ValueError("records: CUDA bytes; qkv: contiguous CUDA bf16 [rows, 3, heads, D]")
+    _check(_lib().sol_attn3d_exchange_unpack_qkv_int8(_ptr(records), _ptr(qkv), n_rows, heads, head_dim, _stream(stream)),
+           "sol_attn3d_exchange_unpack_qkv_int8")
+
+
+def sol_attn3d_exchange_quantize_out_int8(out_rows: torch.Tensor, records: torch.Tensor, stream=None) -> None:
+    n_rows, heads, head_dim = out_rows.shape
+    if not out_rows.is_cuda or out_rows.dtype != torch.bfloat16 or not records.is_cuda:
+        raise ValueError("out_rows: CUDA bf16 [rows, heads, D]; records: CUDA bytes")
+    _check(_lib().sol_attn3d_exchange_quantize_out_int8(_ptr(out_rows), _strides_of(out_rows, head_dim), n_rows, heads,
+                                                        head_dim, _ptr(records), _stream(stream)),
+           "sol_attn3d_exchange_quantize_out_int8")
+
+
+def sol_attn3d_exchange_dequantize_out_int8(records: torch.Tensor, out_rows: torch.Tensor, stream=None) -> None:
+    n_rows, heads, head_dim = out_rows.shape
+    if not out_rows.is_cuda or out_rows.dtype != torch.bfloat16 or not out_rows.is_contiguous() or not records.is_cuda:
+        raise ValueError("out_rows: contiguous CUDA bf16 [rows, heads, D]; records: CUDA bytes")
+    _check(_lib().sol_attn3d_exchange_dequantize_out_int8(_ptr(records), _ptr(out_rows), n_rows, heads, head_dim,
+                                                          _stream(stream)), "sol_attn3d_exchange_dequantize_out_int8")
 
 
 def sol_attn3d_exchange_merge_heads(recv: torch.Tensor, out: torch.Tensor, n_local: int, heads: int, record_bytes: int,

@@ -509,6 +509,114 @@ int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local
   return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
 }
 
+size_t sol_attn3d_exchange_record_bytes(int kind, int head_dim) {
+  if (head_dim != 64 && head_dim != 128) return 0;
+  const size_t groups = (size_t)head_dim / 32;
+  switch (kind) {
+    case SOL_ATTN3D_WIRE_QKV_BF16: return 3u * head_dim * 2u;
+    case SOL_ATTN3D_WIRE_QKV_INT8: return (3u * head_dim + 3u * groups + 15u) / 16u * 16u;
+    case SOL_ATTN3D_WIRE_OUT_BF16: return (size_t)head_dim * 2u;
+    case SOL_ATTN3D_WIRE_OUT_E4M3: return (size_t)head_dim;
+    case SOL_ATTN3D_WIRE_OUT_INT8: return ((size_t)head_dim + groups + 15u) / 16u * 16u;
+    default: return 0;
+  }
+}
+
+extern "C++" {
+namespace {
+template <int NW>
+int launch_quantize(const void* const src[3], const int64_t* const strides[3], int64_t n_rows, int heads, int head_dim,
+                    int n_ranks, void* const* dst, int64_t dst_row0, size_t rec_bytes, cudaStream_t st) {
+  if (n_rows < 0 || dst_row0 < 0 || heads < 1 || (head_dim != 64 && head_dim != 128) || n_ranks < 1 ||
+      n_ranks > sol::kMaxRanks || (heads % n_ranks) != 0)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (n_rows == 0) return SOL_ATTN3D_OK;
+  if (dst == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  sol::QuantArgs a{};
+  for (int w = 0; w < NW; ++w) {
+    if (src[w] == nullptr || strides[w] == nullptr || !aligned16(src[w])) return SOL_ATTN3D_ERR_INVALID_ARG;
+    const long long tok = strides[w][0] == 0 ? (long long)heads * head_dim : strides[w][0];
+    const long long head = strides[w][1] == 0 ? head_dim : strides[w][1];
+    if (!stride_ok(tok) || !stride_ok(head)) return SOL_ATTN3D_ERR_INVALID_ARG;
+    a.src[w] = static_cast<const uint8_t*>(src[w]);
+    a.tok_stride_bytes[w] = tok * 2;
+    a.head_stride_bytes[w] = head * 2;
+  }
+  for (int g = 0; g < n_ranks; ++g) {
+    if (dst[g] == nullptr || !aligned16(dst[g])) return SOL_ATTN3D_ERR_INVALID_ARG;
+    a.dst[g] = static_cast<uint8_t*>(dst[g]);
+  }
+  a.dst_row0 = dst_row0;
+  a.n_rows = n_rows;
+  a.heads = heads;
+  a.hl = heads / n_ranks;
+  a.n_ranks = n_ranks;
+  a.head_dim = head_dim;
+  a.rec_bytes = (int)rec_bytes;
+  const int per_rec = NW * head_dim / 8;
+  const int recs = std::min(16, 256 / per_rec);
+  const long long n_recs = n_rows * heads;
+  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((n_recs + recs - 1) / recs, 148ll * 32));
+  sol::quantize_records_kernel<NW><<<blocks, per_rec * recs, 0, st>>>(a);
+  return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
+}
+}  // namespace
+}  // extern "C++"
+
+int sol_attn3d_exchange_pack_qkv_int8(const void* q, const void* k, const void* v, const int64_t q_strides[2],
+                                      const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
+                                      int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
+                                      sol_attn3d_stream_t stream) {
+  const void* const src[3] = {q, k, v};
+  const int64_t* const strides[3] = {q_strides, k_strides, v_strides};
+  return launch_quantize<3>(src, strides, n_local, heads, head_dim, n_ranks, dst, dst_row0,
+                            sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_QKV_INT8, head_dim),
+                            static_cast<cudaStream_t>(stream));
+}
+
+int sol_attn3d_exchange_quantize_out_int8(const void* out_rows, const int64_t out_strides[2], int64_t n_rows, int heads,
+                                          int head_dim, void* records, sol_attn3d_stream_t stream) {
+  const void* const src[3] = {out_rows, nullptr, nullptr};
+  const int64_t* const strides[3] = {out_strides, nullptr, nullptr};
+  void* const dst[1] = {records};
+  return launch_quantize<1>(src, strides, n_rows, heads, head_dim, 1, dst, 0,
+                            sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_OUT_INT8, head_dim),
+                            static_cast<cudaStream_t>(stream));
+}
+
+extern "C++" {
+namespace {
+template <int NW>
+int launch_dequantize(const void* records, void* out, int64_t n_rows, int heads, int head_dim, size_t rec_bytes,
+                      cudaStream_t st) {
+  if (n_rows < 0 || heads < 1 || (head_dim != 64 && head_dim != 128)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (n_rows == 0) return SOL_ATTN3D_OK;
+  if (records == nullptr || out == nullptr || records == out || !aligned16(records) || !aligned16(out))
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  const long long items = n_rows * (long long)heads * NW * (head_dim / 8);
+  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((items + 255) / 256, 148ll * 32));
+  sol::dequantize_records_kernel<NW><<<blocks, 256, 0, st>>>(static_cast<const uint8_t*>(records),
+                                                              static_cast<__nv_bfloat16*>(out), n_rows, heads, head_dim,
+                                                              (int)rec_bytes);
+  return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
+}
+}  // namespace
+}  // extern "C++"
+
+int sol_attn3d_exchange_unpack_qkv_int8(const void* records, void* qkv, int64_t n_rows, int heads, int head_dim,
+                                        sol_attn3d_stream_t stream) {
+  return launch_dequantize<3>(records, qkv, n_rows, heads, head_dim,
+                              sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_QKV_INT8, head_dim),
+                              static_cast<cudaStream_t>(stream));
+}
+
+int sol_attn3d_exchange_dequantize_out_int8(const void* records, void* out_rows, int64_t n_rows, int heads, int head_dim,
+                                            sol_attn3d_stream_t stream) {
+  return launch_dequantize<1>(records, out_rows, n_rows, heads, head_dim,
+                              sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_OUT_INT8, head_dim),
+                              static_cast<cudaStream_t>(stream));
+}
+
 size_t sol_attn3d_sparse_workspace_bytes(sol_attn3d_plan_t p) { return p ? p->sp_bytes : 0; }
 
 int sol_attn3d_forward_sparse(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,

@@ -29,7 +29,10 @@ def shard_ranges(total: int, n_ranks: int) -> List[Tuple[int, int]]:
 class ExchangePlan:
     """Host-side description of the two all-to-alls for one rank (pure Python, no device work)."""
 
-    def __init__(self, total_tokens: int, heads: int, head_dim: int, n_ranks: int, rank: int, out_record_bytes: int):
+    def __init__(self, total_tokens: int, heads: int, head_dim: int, n_ranks: int, rank: int, out_record_bytes: int,
+                 qkv_record_elems: int = 0, out_record_elems: int = 0):
+        """qkv_record_elems / out_record_elems: elements of the exchanged tensors per (token, head) record
+        (default: 3*head_dim and head_dim, the unquantised layouts; the block-INT8 records are 400 / 144 bytes)."""
         if n_ranks < 1 or n_ranks > B.MAX_RANKS:
             raise ValueError(f"1 <= n_ranks <= {B.MAX_RANKS}")
         if heads % n_ranks:
@@ -42,12 +45,12 @@ class ExchangePlan:
         self.tok_begin = [a for a, _ in self.ranges] + [total_tokens]
         self.n_local = self.ranges[rank][1] - self.ranges[rank][0]
         self.first_token = self.ranges[rank][0]
-        qkv_row = 3 * self.hl * head_dim                       # elements per token in the QKV exchange
+        qkv_row = self.hl * (qkv_record_elems or 3 * head_dim)  # elements per token in the QKV exchange
         # split sizes are in ELEMENTS of the exchanged tensors
         # QKV exchange: this rank sends n_local rows to everyone and receives n_s rows from rank s
         self.qkv_send_splits = [self.n_local * qkv_row] * n_ranks
         self.qkv_recv_splits = [(b - a) * qkv_row for a, b in self.ranges]
-        out_row = self.hl * head_dim                           # elements per token in the output return
+        out_row = self.hl * (out_record_elems or head_dim)      # elements per token in the output return
         self.out_record_bytes = out_record_bytes               # bytes of one (token, head) record on the wire
         # output return: this rank owes rows [a_g, b_g) to rank g and receives its own n_local rows from everyone
         self.out_send_splits = [(b - a) * out_row for a, b in self.ranges]
@@ -58,22 +61,37 @@ class SequenceParallelAttn3d:
     """One DiT-block attention over a sequence-sharded Q, K, V.  forward() returns this rank's token rows."""
 
     def __init__(self, seqs: Sequence[Tuple[int, int, int, int]], heads: int, head_dim: int, rope_dims, theta: float = 10000.0,
-                 group=None, device="cuda", out_format: str = "bf16", transport: str = "collective"):
+                 group=None, device="cuda", out_format: str = "bf16", transport: str = "collective", qkv_wire: str = "bf16"):
+        """out_format: what travels back and is returned -- "bf16", "e4m3" (raw bytes, returned as uint8) or "int8"
+        (block-INT8 records on the wire, dequantised to bf16 on arrival).  qkv_wire: "bf16" or "int8" (block-INT8
+        records on the wire, dequantised to bf16 before the attention).  The quantised formats are approximate."""
         import torch.distributed as dist
         self.dist = dist
         self.group = group
         self.n_ranks = dist.get_world_size(group)
         self.rank = dist.get_rank(group)
-        if out_format not in ("bf16", "e4m3"):
-            raise ValueError("out_format: 'bf16' or 'e4m3'")
+        if out_format not in ("bf16", "e4m3", "int8"):
+            raise ValueError("out_format: 'bf16', 'e4m3' or 'int8'")
+        if qkv_wire not in ("bf16", "int8"):
+            raise ValueError("qkv_wire: 'bf16' or 'int8'")
         if transport not in ("collective", "peer"):
             raise ValueError("transport: 'collective' or 'peer'")
+        if transport == "peer" and (qkv_wire != "bf16" or out_format == "int8"):
+            raise ValueError("transport 'peer' carries bf16 QKV and bf16 / e4m3 output")
         self.fp8 = out_format == "e4m3"
+        self.out_int8 = out_format == "int8"
+        self.qkv_int8 = qkv_wire == "int8"
         self.transport = transport
         self.heads, self.head_dim = heads, head_dim
         total = sum(L + T * H * W for (L, T, H, W) in seqs)
-        self.xp = ExchangePlan(total, heads, head_dim, self.n_ranks, self.rank, head_dim * (1 if self.fp8 else 2))
-        hl, D = self.xp.hl, head_dim
+        D = head_dim
+        self.rb_in = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D) if self.qkv_int8 else 3 * D * 2
+        self.rb_out = B.sol_attn3d_exchange_record_bytes(
+            B.WIRE_OUT_INT8 if self.out_int8 else B.WIRE_OUT_E4M3 if self.fp8 else B.WIRE_OUT_BF16, D)
+        self.xp = ExchangePlan(total, heads, D, self.n_ranks, self.rank, self.rb_out,
+                               qkv_record_elems=self.rb_in if self.qkv_int8 else 0,
+                               out_record_elems=self.rb_out if self.out_int8 else 0)
+        hl = self.xp.hl
         qkv_strides = (3 * hl * D, D)
         self.attn = B.Attn3d(seqs, hl, D, rope_dims, theta, device, q_strides=qkv_strides, k_strides=qkv_strides,
                              v_strides=qkv_strides)
@@ -81,9 +99,17 @@ class SequenceParallelAttn3d:
         n_local = self.xp.n_local
         if transport == "collective":
             self.qkv = torch.empty((total, 3, hl, D), dtype=torch.bfloat16, device=device)
-            self.send = torch.empty((self.n_ranks, n_local, 3, hl, D), dtype=torch.bfloat16, device=device)
+            if self.qkv_int8:
+                self.send = torch.empty((self.n_ranks, n_local, hl, self.rb_in), dtype=torch.uint8, device=device)
+                self.qkv_records = torch.empty((total, hl, self.rb_in), dtype=torch.uint8, device=device)
+            else:
+                self.send = torch.empty((self.n_ranks, n_local, 3, hl, D), dtype=torch.bfloat16, device=device)
             self.out_shard = torch.empty((total, hl, D), dtype=self.out_dtype, device=device)
-            self.recv_out = torch.empty((self.n_ranks, n_local, hl, D), dtype=self.out_dtype, device=device)
+            if self.out_int8:
+                self.out_records = torch.empty((total, hl, self.rb_out), dtype=torch.uint8, device=device)
+                self.recv_out = torch.empty((self.n_ranks, n_local, hl, self.rb_out), dtype=torch.uint8, device=device)
+            else:
+                self.recv_out = torch.empty((self.n_ranks, n_local, hl, D), dtype=self.out_dtype, device=device)
         else:
             import torch.distributed._symmetric_memory as symm
             per = self.xp.ranges[0][1] - self.xp.ranges[0][0]          # largest shard: same size on every rank
@@ -107,17 +133,33 @@ class SequenceParallelAttn3d:
             raise ValueError(f"expected [{xp.n_local}, {self.heads}, {self.head_dim}] on rank {self.rank}")
         qv, kv, vv = self.qkv[:, 0], self.qkv[:, 1], self.qkv[:, 2]
         if self.transport == "collective":
-            B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, [self.send[g].data_ptr() for g in range(self.n_ranks)], 0)
-            self.dist.all_to_all_single(self.qkv.view(-1), self.send.view(-1), xp.qkv_recv_splits, xp.qkv_send_splits,
-                                        group=self.group)
+            dsts = [self.send[g].data_ptr() for g in range(self.n_ranks)]
+            if self.qkv_int8:
+                B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, self.n_ranks, dsts, 0)
+                self.dist.all_to_all_single(self.qkv_records.view(-1), self.send.view(-1), xp.qkv_recv_splits,
+                                            xp.qkv_send_splits, group=self.group)
+                B.sol_attn3d_exchange_unpack_qkv_int8(self.qkv_records, self.qkv, xp.total, xp.hl, self.head_dim)
+            else:
+                B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, dsts, 0)
+                self.dist.all_to_all_single(self.qkv.view(-1), self.send.view(-1), xp.qkv_recv_splits, xp.qkv_send_splits,
+                                            group=self.group)
             if self.fp8:
                 B.sol_attn3d_forward_e4m3(self.attn.plan, qv, kv, vv, self.out_shard, key_mask)
             else:
                 B.sol_attn3d_forward(self.attn.plan, qv, kv, vv, self.out_shard, key_mask)
-            self.dist.all_to_all_single(self.recv_out.view(-1), self.out_shard.view(-1), xp.out_recv_splits,
-                                        xp.out_send_splits, group=self.group)
+            wire = self.out_shard
+            if self.out_int8:
+                B.sol_attn3d_exchange_quantize_out_int8(self.out_shard, self.out_records)
+                wire = self.out_records
+            self.dist.all_to_all_single(self.recv_out.view(-1), wire.view(-1), xp.out_recv_splits, xp.out_send_splits,
+                                        group=self.group)
             out = torch.empty((xp.n_local, self.heads, self.head_dim), dtype=self.out_dtype, device=q.device)
-            B.sol_attn3d_exchange_merge_heads(self.recv_out, out, xp.n_local, self.heads, xp.out_record_bytes, self.n_ranks)
+            if self.out_int8:
+                merged = torch.empty((xp.n_local, self.heads, self.rb_out), dtype=torch.uint8, device=q.device)
+                B.sol_attn3d_exchange_merge_heads(self.recv_out, merged, xp.n_local, self.heads, self.rb_out, self.n_ranks)
+                B.sol_attn3d_exchange_dequantize_out_int8(merged, out)
+            else:
+                B.sol_attn3d_exchange_merge_heads(self.recv_out, out, xp.n_local, self.heads, self.rb_out, self.n_ranks)
             return out
         # peer transport: stores into the owners' buffers, barriers instead of payload collectives
         self._barrier()                                       # everyone is done reading last call's buffers

@@ -291,7 +291,154 @@ def test_sequence_parallel_module_with_one_rank(B):
         got8 = sp8.forward(inp.q, inp.k, inp.v, inp.key_mask)
         torch.cuda.synchronize()
         check_e4m3(got8, oracle_dense(w, inp))
-        sp.close(); sp8.close(); single.close()
+        # block-INT8 both ways: equals the same kernels called by hand on one rank
+        spq = SequenceParallelAttn3d(seq_tuples(w), w.heads, w.head_dim, w.rope_dims, w.theta, out_format="int8", qkv_wire="int8")
+        gotq = spq.forward(inp.q, inp.k, inp.v, inp.key_mask)
+        torch.cuda.synchronize()
+        D = w.head_dim
+        rec = torch.empty((w.total_tokens, w.heads, B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)), dtype=torch.uint8, device="cuda")
+        B.sol_attn3d_exchange_pack_qkv_int8(inp.q, inp.k, inp.v, 1, [rec.data_ptr()], 0)
+        qkv = torch.empty((w.total_tokens, 3, w.heads, D), dtype=torch.bfloat16, device="cuda")
+        B.sol_attn3d_exchange_unpack_qkv_int8(rec, qkv, w.total_tokens, w.heads, D)
+        st = (3 * w.heads * D, D)
+        a2 = B.Attn3d(seq_tuples(w), w.heads, D, w.rope_dims, w.theta, "cuda", q_strides=st, k_strides=st, v_strides=st)
+        o2 = a2.forward(qkv[:, 0], qkv[:, 1], qkv[:, 2], inp.key_mask)
+        orec = torch.empty((w.total_tokens, w.heads, B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, D)), dtype=torch.uint8, device="cuda")
+        B.sol_attn3d_exchange_quantize_out_int8(o2, orec)
+        wantq = torch.empty_like(o2)
+        B.sol_attn3d_exchange_dequantize_out_int8(orec, wantq)
+        torch.cuda.synchronize()
+        assert torch.equal(gotq, wantq)
+        rel = float(torch.linalg.vector_norm(gotq.double() - want.double()) / torch.linalg.vector_norm(want.double()))
+        assert rel < 3e-2, rel
+        sp.close(); sp8.close(); spq.close(); a2.close(); single.close()
     finally:
         if created:
             dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------ block-INT8 wire formats
+@pytest.mark.parametrize("G,n_local,heads,D", [(1, 50, 3, 128), (4, 301, 8, 128), (8, 33, 40, 128), (2, 77, 6, 64), (3, 0, 6, 64)])
+def test_int8_qkv_records_are_bit_exact(B, G, n_local, heads, D):
+    g = torch.Generator(device="cuda").manual_seed(300 + G)
+    packed = torch.randn((max(n_local, 1), 3, heads, D), generator=g, device="cuda")
+    packed[:, 1] *= 0.05                                     # different ranges per tensor, as K after QK-norm
+    packed[:, 2] *= 30.0
+    packed = packed.to(torch.bfloat16)[:n_local]
+    if n_local > 2:
+        packed[1, 0, 0, :32] = 0                             # an all-zero group
+        packed[2, 2, 1, 5] = 127.0 * 64                      # a maximum that sits exactly on a scale (s = 64)
+    q, k, v = packed[:, 0], packed[:, 1], packed[:, 2]
+    hl = heads // G
+    rb = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)
+    assert rb == xo.qkv_record_bytes(D)
+    send = torch.full((G, n_local, hl, rb), 0xEE, dtype=torch.uint8, device="cuda")
+    dummy = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, G, [send[r].data_ptr() if n_local else dummy.data_ptr() for r in range(G)], 0)
+    torch.cuda.synchronize()
+    want = xo.qkv_records(q.cpu(), k.cpu(), v.cpu())          # [n, heads, rb]
+    for r in range(G):
+        assert torch.equal(send[r].cpu(), want[:, r * hl:(r + 1) * hl]), f"records for rank {r}"
+    if n_local == 0:
+        return
+    # receiver: dequantise into the packed [rows][3][hl][D] tensor; exact product, one rounding to bf16
+    for r in range(G):
+        qkv = torch.full((n_local, 3, hl, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        B.sol_attn3d_exchange_unpack_qkv_int8(send[r], qkv, n_local, hl, D)
+        torch.cuda.synchronize()
+        dq = xo.qkv_from_records(want[:, r * hl:(r + 1) * hl].contiguous(), D)
+        for wch in range(3):
+            assert torch.equal(qkv[:, wch].cpu().view(torch.int16), dq[wch].to(torch.bfloat16).view(torch.int16))
+    # and the quantisation error as a number: half a step of the group's scale
+    dq_all = xo.qkv_from_records(want, D)
+    for wch, x in enumerate((q, k, v)):
+        err = (dq_all[wch] - x.cpu().double()).abs().reshape(n_local, heads, D // 32, 32)
+        amax = x.cpu().double().abs().reshape(n_local, heads, D // 32, 32).amax(-1, keepdim=True)
+        assert bool((err <= amax / 127.0 * 1.125 * 0.5001 + 2.0 ** -17).all())
+
+
+@pytest.mark.parametrize("n,heads,D", [(200, 5, 128), (77, 40, 128), (64, 3, 64), (0, 4, 128)])
+def test_int8_output_records_are_bit_exact(B, n, heads, D):
+    g = torch.Generator(device="cuda").manual_seed(400 + n)
+    wide = (torch.randn((max(n, 1), heads + 2, D), generator=g, device="cuda") * 0.3).to(torch.bfloat16)[:n]
+    rows = wide[:, 1:heads + 1]                               # a strided view: token stride (heads+2)*D
+    rb = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, D)
+    assert rb == xo.out_record_bytes(D)
+    rec = torch.full((max(n, 1), heads, rb), 0xEE, dtype=torch.uint8, device="cuda")[:n]
+    B.sol_attn3d_exchange_quantize_out_int8(rows, rec)
+    torch.cuda.synchronize()
+    want = xo.out_records(rows.cpu())
+    assert torch.equal(rec.cpu(), want)
+    if n == 0:
+        return
+    back = torch.full((n, heads, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.sol_attn3d_exchange_dequantize_out_int8(rec, back)
+    torch.cuda.synchronize()
+    assert torch.equal(back.cpu().view(torch.int16), xo.out_from_records(want, D).to(torch.bfloat16).view(torch.int16))
+
+
+def test_exchange_with_int8_wire_formats(B):
+    """Whole exchange, 4 virtual ranks, block-INT8 both ways.  Approximate by design, so two checks: the GPU
+    pipeline equals the oracle pipeline fed with the same records (attention tolerance), and the end result stays
+    within the quantisation error of the unquantised attention."""
+    w = replace(wl.shrunk("lowres"), heads=8)
+    inp = wl.make_inputs(w, "cuda")
+    G, total, heads, D = 4, w.total_tokens, w.heads, w.head_dim
+    hl = heads // G
+    ranges = xo.shard_ranges(total, G)
+    rb_in = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)
+    rb_out = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, D)
+    recv = [torch.empty((total, hl, rb_in), dtype=torch.uint8, device="cuda") for _ in range(G)]
+    for s, (a, b) in enumerate(ranges):                        # peer style: records land in the owners' buffers
+        B.sol_attn3d_exchange_pack_qkv_int8(inp.q[a:b], inp.k[a:b], inp.v[a:b], G, [t.data_ptr() for t in recv], a)
+    torch.cuda.synchronize()
+    want_rec = xo.qkv_records(inp.q.cpu(), inp.k.cpu(), inp.v.cpu())
+    strides = (3 * hl * D, D)
+    back = [torch.empty((G, b - a, hl, rb_out), dtype=torch.uint8, device="cuda") for (a, b) in ranges]
+    ref_shards = []
+    for r in range(G):
+        assert torch.equal(recv[r].cpu(), want_rec[:, r * hl:(r + 1) * hl])
+        qkv = torch.empty((total, 3, hl, D), dtype=torch.bfloat16, device="cuda")
+        B.sol_attn3d_exchange_unpack_qkv_int8(recv[r], qkv, total, hl, D)
+        attn = B.Attn3d(seq_tuples(w), hl, D, w.rope_dims, w.theta, "cuda", q_strides=strides, k_strides=strides, v_strides=strides)
+        shard = attn.forward(qkv[:, 0], qkv[:, 1], qkv[:, 2], inp.key_mask)
+        rec = torch.empty((total, hl, rb_out), dtype=torch.uint8, device="cuda")
+        B.sol_attn3d_exchange_quantize_out_int8(shard, rec)
+        torch.cuda.synchronize()
+        assert attn.status() == 0
+        attn.close()
+        # oracle attention on the dequantised (bf16-rounded) inputs the GPU attention saw
+        dq = [x.to(torch.bfloat16) for x in xo.qkv_from_records(want_rec[:, r * hl:(r + 1) * hl].contiguous(), D)]
+        ref = orc.attn3d_oracle(dq[0], dq[1], dq[2], seq_tuples(w), w.rope_dims, w.theta, None)
+        max_abs, rel_l2 = orc.compare(shard.cpu(), ref)
+        assert max_abs <= TOL_MAX_ABS and rel_l2 <= TOL_REL_L2, (max_abs, rel_l2)
+        assert torch.equal(rec.cpu(), xo.out_records(shard.cpu()))
+        ref_shards.append(ref)
+        for o, (a, b) in enumerate(ranges):
+            back[o][r] = rec[a:b]
+    outs = []
+    for o, (a, b) in enumerate(ranges):
+        merged = torch.empty((b - a, heads, rb_out), dtype=torch.uint8, device="cuda")
+        B.sol_attn3d_exchange_merge_heads(back[o], merged, b - a, heads, rb_out, G)
+        rows = torch.empty((b - a, heads, D), dtype=torch.bfloat16, device="cuda")
+        B.sol_attn3d_exchange_dequantize_out_int8(merged, rows)
+        outs.append(rows)
+    torch.cuda.synchronize()
+    got = torch.cat(outs, 0).cpu().double()
+    # against the oracle of the same pipeline: attention error + half an output step
+    ref_pipeline = torch.cat(ref_shards, dim=1)
+    step = ref_pipeline.abs().reshape(total, heads, D // 32, 32).amax(-1, keepdim=True) / 127.0 * 1.125
+    assert bool(((got - ref_pipeline).reshape(total, heads, D // 32, 32).abs() <= 0.5 * step + 2e-3 + 2.0 ** -8 * step * 127).all())
+    # against the unquantised attention: a few per cent, as the paper says "approximate"
+    exact = oracle_dense(w, replace_mask(inp))
+    rel = float(torch.linalg.vector_norm(got - exact) / torch.linalg.vector_norm(exact))
+    print("int8 both ways: rel-L2 vs unquantised attention", rel)
+    assert rel < 3e-2
+
+
+def replace_mask(inp):
+    class _I:
+        pass
+    o = _I()
+    o.q, o.k, o.v, o.key_mask = inp.q, inp.k, inp.v, None
+    return o
