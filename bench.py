@@ -157,6 +157,86 @@ def cpu_sample_spec(w, scale=1.0):
     return list(range(0, w.heads, step))[:n_heads], (w.rows_per_head or 0)
 
 
+def exchange_bench(args, w, dev, B, peaks, config):
+    """One rank's share of a G-way sequence-parallel exchange around the attention: the layout / quantisation
+    kernels and the head-sharded attention, each timed alone with CUDA events (best and mean of `steps`)."""
+    G = args.exchange
+    heads, D, total = w.heads, w.head_dim, w.total_tokens
+    if heads % G or G > B.MAX_RANKS:
+        raise SystemExit(f"--exchange {G}: heads ({heads}) must be divisible and G <= {B.MAX_RANKS}")
+    hl = heads // G
+    n_local = -(-total // G)
+    gen = torch.Generator(device=dev).manual_seed(w.seed)
+    packed = torch.randn((n_local, 3, heads, D), generator=gen, device=dev).to(torch.bfloat16)   # packed QKV storage
+    q, k, v = packed[:, 0], packed[:, 1], packed[:, 2]
+    send = torch.empty((G, n_local, 3, hl, D), dtype=torch.bfloat16, device=dev)
+    rb_in = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)
+    rb_out = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, D)
+    send8 = torch.empty((G, n_local, hl, rb_in), dtype=torch.uint8, device=dev)
+    qkv = torch.randn((total, 3, hl, D), generator=gen, device=dev).to(torch.bfloat16)
+    rec_in = torch.randint(1, 120, (total, hl, rb_in), generator=gen, device=dev, dtype=torch.uint8)
+    shard = (0.1 * torch.randn((total, hl, D), generator=gen, device=dev)).to(torch.bfloat16)
+    shard8 = torch.empty((total, hl, D), dtype=torch.uint8, device=dev)
+    rec_out = torch.empty((total, hl, rb_out), dtype=torch.uint8, device=dev)
+    recv = torch.randn((G, n_local, hl, D), generator=gen, device=dev).to(torch.bfloat16)
+    recv_rec = torch.randint(1, 120, (n_local, heads, rb_out), generator=gen, device=dev, dtype=torch.uint8)
+    merged = torch.empty((n_local, heads, D), dtype=torch.bfloat16, device=dev)
+    st = (3 * hl * D, D)
+    seqs = [(s.text_len, s.T, s.H, s.W) for s in w.seqs]
+    attn = B.Attn3d(seqs, hl, D, w.rope_dims, w.theta, dev, q_strides=st, k_strides=st, v_strides=st)
+    per = -(-total // G)
+    tok_begin = [min(g * per, total) for g in range(G)] + [total]
+    owners = [torch.empty((max(tok_begin[g + 1] - tok_begin[g], 1), heads, D), dtype=torch.bfloat16, device=dev) for g in range(G)]
+    sptr = [send[g].data_ptr() for g in range(G)]
+    sptr8 = [send8[g].data_ptr() for g in range(G)]
+    bf = 2
+    kernels = {
+        # name: (callable, bytes read + written)
+        "pack_qkv": (lambda: B.sol_attn3d_exchange_pack_qkv(q, k, v, G, sptr, 0), 2 * packed.numel() * bf),
+        "merge_heads_bf16": (lambda: B.sol_attn3d_exchange_merge_heads(recv, merged, n_local, heads, D * bf, G), 2 * recv.numel() * bf),
+        "pack_qkv_int8": (lambda: B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, G, sptr8, 0), packed.numel() * bf + send8.numel()),
+        "unpack_qkv_int8": (lambda: B.sol_attn3d_exchange_unpack_qkv_int8(rec_in, qkv, total, hl, D), rec_in.numel() + qkv.numel() * bf),
+        "quantize_out_int8": (lambda: B.sol_attn3d_exchange_quantize_out_int8(shard, rec_out), shard.numel() * bf + rec_out.numel()),
+        "dequantize_out_int8": (lambda: B.sol_attn3d_exchange_dequantize_out_int8(recv_rec, merged), recv_rec.numel() + merged.numel() * bf),
+        "attention_shard_bf16": (lambda: B.sol_attn3d_forward(attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], shard, None), None),
+        "attention_shard_e4m3": (lambda: B.sol_attn3d_forward_e4m3(attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], shard8, None), None),
+        "attention_shard_scatter": (lambda: B.sol_attn3d_forward_scatter(attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], None,
+                                                                         [o.data_ptr() for o in owners], tok_begin, heads, 0), None),
+    }
+    if args.exchange_kernel != "all":
+        kernels = {args.exchange_kernel: kernels[args.exchange_kernel]}
+    hbm = peaks.get("hbm_gbs") if isinstance(peaks, dict) else None
+    shard_flops = w.flops() / G
+    res = {}
+    for name, (fn, nbytes) in kernels.items():
+        for _ in range(max(3, args.warmup)):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ms = sum(ts) / len(ts)
+        r = {"ms": ms, "ms_best": min(ts)}
+        if nbytes is not None:
+            r["bytes"] = nbytes
+            r["gbps"] = nbytes / ms / 1e6
+            if hbm:
+                r["frac_of_measured_hbm"] = r["gbps"] / hbm
+        else:
+            r["tflops"] = shard_flops / ms / 1e9
+        res[name] = r
+    assert attn.status() == 0
+    print(json.dumps({"metric": "exchange_kernels_ms", "unit": "ms", "n_gpus": 1, "steps": args.steps,
+                      "warmup": max(3, args.warmup), "exchange_ranks": G, "tokens_per_rank": n_local, "heads_per_rank": hl,
+                      "hbm_peak_gbs": hbm, "config": config, "data": "synthetic", "kernels": res}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -170,6 +250,11 @@ def main():
                     help="time sol_attn3d_forward_sparse with this tau (block-sparse variant of Section 3.4)")
     ap.add_argument("--qknorm", action="store_true",
                     help="time sol_attn3d_forward_qknorm (QK RMS-norm fused into the rotary producer) instead")
+    ap.add_argument("--exchange", type=int, default=0, metavar="G",
+                    help="instead of the forward: time one rank's kernels of a G-way sequence-parallel exchange "
+                         "(Section 3.3) at the workload's shape and print their ms and GB/s")
+    ap.add_argument("--exchange-kernel", default="all",
+                    help="with --exchange: run only this kernel (e.g. for a profiler capture)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -221,6 +306,9 @@ def main():
         import torch.distributed as dist_
         dist = dist_
         dist.init_process_group("nccl", device_id=dev)
+
+    if args.exchange:
+        return exchange_bench(args, w, dev, B, peaks, config)
 
     warmup = max(3, args.warmup)
     inp = wl.make_inputs(w, dev)

@@ -10,6 +10,19 @@ namespace sol {
 
 constexpr int kMaxRanks = 8;
 
+// x = q * d + r.  Index spaces here almost always fit 32 bits, where the division is several times cheaper;
+// `small` (uniform across the grid) says so.
+__device__ __forceinline__ void divmod(long long x, int d, bool small, long long& q, int& r) {
+  if (small) {
+    const unsigned xq = (unsigned)x / (unsigned)d;
+    q = xq;
+    r = (int)((unsigned)x - xq * (unsigned)d);
+  } else {
+    q = x / d;
+    r = (int)(x - q * d);
+  }
+}
+
 // Sender's side of the packed QKV exchange.  This rank holds n_local tokens of Q, K and V with all heads,
 // read through their own strides (views into a packed QKV buffer are fine).  Destination g receives heads
 // [g*hl, (g+1)*hl) of every local token as rows [dst_row0 + t][3][hl][row_bytes]:
@@ -33,8 +46,9 @@ constexpr int kPackUnroll = 4;
 __global__ void __launch_bounds__(256) exchange_pack_qkv_kernel(const PackArgs a) {
   // one item = one 16-byte chunk; items ordered (token, which, head, chunk): a warp reads a contiguous
   // stretch of one source row and writes contiguous stretches of hl * row_bytes per destination
-  const long long per_tok = 3ll * a.heads * a.chunks;
+  const int per_tok = 3 * a.heads * a.chunks;
   const long long items = a.n_local * per_tok;
+  const bool small = items < (1ll << 32);
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long base = (long long)blockIdx.x * blockDim.x + threadIdx.x; base < items; base += stride * kPackUnroll) {
     uint4 v[kPackUnroll];
@@ -44,8 +58,9 @@ __global__ void __launch_bounds__(256) exchange_pack_qkv_kernel(const PackArgs a
       const long long i = base + u * stride;
       out[u] = nullptr;
       if (i < items) {
-        const long long t = i / per_tok;
-        int r = (int)(i - t * per_tok);
+        long long t;
+        int r;
+        divmod(i, per_tok, small, t, r);
         const int which = r / (a.heads * a.chunks);
         r -= which * a.heads * a.chunks;
         const int h = r / a.chunks;
@@ -69,8 +84,9 @@ __global__ void __launch_bounds__(256) exchange_merge_heads_kernel(const uint8_t
                                                                    uint8_t* __restrict__ out, long long n, int hl,
                                                                    int n_ranks, int chunks,
                                                                    long long out_tok_stride_bytes) {
-  const long long per_tok = (long long)n_ranks * hl * chunks;
+  const int per_tok = n_ranks * hl * chunks;
   const long long items = n * per_tok;
+  const bool small = items < (1ll << 32);
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long base = (long long)blockIdx.x * blockDim.x + threadIdx.x; base < items; base += stride * kPackUnroll) {
     uint4 v[kPackUnroll];
@@ -80,8 +96,9 @@ __global__ void __launch_bounds__(256) exchange_merge_heads_kernel(const uint8_t
       const long long i = base + u * stride;
       dst[u] = nullptr;
       if (i < items) {
-        const long long t = i / per_tok;
-        int r = (int)(i - t * per_tok);
+        long long t;
+        int r;
+        divmod(i, per_tok, small, t, r);
         const int g = r / (hl * chunks);
         r -= g * hl * chunks;                                   // (local head, chunk) within the shard
         v[u] = __ldg(reinterpret_cast<const uint4*>(recv + (((long long)g * n + t) * hl * chunks + r) * 16));
@@ -136,71 +153,71 @@ struct QuantArgs {
 };
 
 // NW = 3: the quantising QKV pack (sender's side of the exchange); NW = 1: output rows -> output records.
-// One thread per 8 values; the 4 threads of a 32-value group sit in adjacent lanes.  A block of
-// (threads per record) x (at most 16 records) threads handles that many records per iteration; their scale
-// codes meet in shared memory and leave as one 16-byte tail each (both record kinds end in exactly 16 bytes
-// of codes + zeros for head_dim 64 and 128).
+// rint(x) clamped to int8 in one instruction; |x| <= 127 (1 + 2^-22) here, so the result is within +-127
+__device__ __forceinline__ uint32_t rint_sat_s8(float x) {
+  int q;
+  asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(q) : "f"(x));
+  return (uint32_t)q;
+}
+// low bytes of four registers -> one word, a in the lowest byte
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+
+// One thread per group of 32 values (64 contiguous bytes in, 32 bytes + one scale code out): the scale search
+// and the reciprocal are paid once per group and nothing is exchanged between lanes.  Items are ordered
+// (record, tensor, group), so adjacent threads read adjacent 64-byte pieces.
 template <int NW>
 __global__ void __launch_bounds__(256) quantize_records_kernel(const QuantArgs a) {
-  const int chunks = a.head_dim >> 3;
-  const int per_rec = NW * chunks;                              // threads per record
-  const int recs = blockDim.x / per_rec;                        // records per block iteration
   const int ng = a.head_dim >> 5;                               // groups (= scale codes) per tensor
-  __shared__ __align__(16) uint8_t tails[16][16];
-  const int r_in = threadIdx.x / per_rec;
-  const int rem = threadIdx.x - r_in * per_rec;
-  const int which = rem / chunks;
-  const int c = rem - which * chunks;
-  const long long n_recs = a.n_rows * a.heads;
-  for (long long rec0 = (long long)blockIdx.x * recs; rec0 < n_recs; rec0 += (long long)gridDim.x * recs) {
-    const long long rec = rec0 + r_in;
-    const bool valid = r_in < recs && rec < n_recs;
-    float f[8];
+  const int per_rec = NW * ng;                                  // threads per record
+  const long long n_items = a.n_rows * a.heads * per_rec;
+  const bool small = n_items < (1ll << 32);
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_items; i += (long long)gridDim.x * blockDim.x) {
+    long long rec, t;
+    int rem, h;
+    divmod(i, per_rec, small, rec, rem);
+    divmod(rec, a.heads, small, t, h);
+    const int which = rem / ng;
+    const int grp = rem - which * ng;
+    const uint4* src = reinterpret_cast<const uint4*>(a.src[which] + t * a.tok_stride_bytes[which] +
+                                                      h * a.head_stride_bytes[which] + grp * 64);
+    uint4 v[4];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) f[e] = 0.f;
-    long long t = 0;
-    int h = 0;
-    if (valid) {
-      t = rec / a.heads;
-      h = (int)(rec - t * a.heads);
-      const uint4 v = __ldg(reinterpret_cast<const uint4*>(a.src[which] + t * a.tok_stride_bytes[which] +
-                                                          h * a.head_stride_bytes[which] + c * 16));
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    for (int j = 0; j < 4; ++j) v[j] = __ldg(src + j);
+    float f[32];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162*>(&w[u]);
-        f[2 * u] = __low2float(b2);
-        f[2 * u + 1] = __high2float(b2);
+        f[8 * j + 2 * u] = __uint_as_float(w[u] << 16);          // bf16 -> fp32 is a shift
+        f[8 * j + 2 * u + 1] = __uint_as_float(w[u] & 0xffff0000u);
       }
     }
     float amax = 0.f;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(f[e]));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    for (int e = 0; e < 32; ++e) amax = fmaxf(amax, fabsf(f[e]));
     const int code = ue5m3_smallest_cover(amax);
     const float inv = __frcp_rn(ue5m3_value(code));
-    uint32_t packed[2] = {0u, 0u};
+    uint32_t o[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      int q = __float2int_rn(__fmul_rn(f[e], inv));
-      q = min(max(q, -127), 127);
-      packed[e >> 2] |= (uint32_t)(q & 0xff) << (8 * (e & 3));
+    for (int j = 0; j < 8; ++j)
+      o[j] = pack_low_bytes(rint_sat_s8(__fmul_rn(f[4 * j], inv)), rint_sat_s8(__fmul_rn(f[4 * j + 1], inv)),
+                            rint_sat_s8(__fmul_rn(f[4 * j + 2], inv)), rint_sat_s8(__fmul_rn(f[4 * j + 3], inv)));
+    const int g = h / a.hl;
+    uint8_t* out = a.dst[g] + ((a.dst_row0 + t) * a.hl + (h - g * a.hl)) * a.rec_bytes;
+    uint4* dst = reinterpret_cast<uint4*>(out + which * a.head_dim + grp * 32);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    // tail of the record: the scale codes, then zeros up to the record size (written by the record's last thread)
+    const int tail = NW * a.head_dim;
+    out[tail + rem] = (uint8_t)code;
+    if (rem == per_rec - 1) {
+      int b = tail + per_rec;
+      for (; (b & 3) != 0 && b < a.rec_bytes; ++b) out[b] = 0;
+      for (; b < a.rec_bytes; b += 4) *reinterpret_cast<uint32_t*>(out + b) = 0u;   // record sizes are multiples of 16
     }
-    uint8_t* out = nullptr;
-    if (valid) {
-      const int g = h / a.hl;
-      out = a.dst[g] + ((a.dst_row0 + t) * a.hl + (h - g * a.hl)) * a.rec_bytes;
-      *reinterpret_cast<uint2*>(out + which * a.head_dim + c * 8) = make_uint2(packed[0], packed[1]);
-    }
-    // zero the tail first (codes overwrite their slots after the barrier)
-    if (r_in < recs)
-      for (int b = rem; b < 16; b += per_rec) tails[r_in][b] = 0;
-    __syncthreads();
-    if (r_in < recs && (c & 3) == 0) tails[r_in][which * ng + (c >> 2)] = (uint8_t)code;
-    __syncthreads();
-    if (valid && rem == 0) *reinterpret_cast<uint4*>(out + NW * a.head_dim) = *reinterpret_cast<const uint4*>(tails[r_in]);
-    __syncthreads();
   }
 }
 
@@ -210,30 +227,35 @@ template <int NW>
 __global__ void __launch_bounds__(256) dequantize_records_kernel(const uint8_t* __restrict__ recs,
                                                                  __nv_bfloat16* __restrict__ out, long long n_rows,
                                                                  int heads, int head_dim, int rec_bytes) {
-  const int chunks = head_dim >> 3;
-  const long long per_row = (long long)heads * NW * chunks;
-  const long long items = n_rows * per_row;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (long long)gridDim.x * blockDim.x) {
-    const long long t = i / per_row;
-    int r = (int)(i - t * per_row);
-    const int h = r / (NW * chunks);
-    r -= h * NW * chunks;
-    const int which = r / chunks;
-    const int c = r - which * chunks;
-    const uint8_t* rec = recs + (t * heads + h) * rec_bytes;
-    const uint2 v = __ldg(reinterpret_cast<const uint2*>(rec + which * head_dim + c * 8));
-    const float s = ue5m3_value(__ldg(rec + NW * head_dim + which * (head_dim >> 5) + (c >> 2)));
-    const uint32_t w[2] = {v.x, v.y};
-    uint32_t o[4];
+  // one thread per group of 32 values: 32 bytes + one code in, 64 bytes out; items ordered (record, tensor, group)
+  const int ng = head_dim >> 5;
+  const int per_rec = NW * ng;
+  const long long n_items = n_rows * heads * per_rec;
+  const bool small = n_items < (1ll << 32);
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_items; i += (long long)gridDim.x * blockDim.x) {
+    long long rec, t;
+    int rem, h;
+    divmod(i, per_rec, small, rec, rem);
+    divmod(rec, heads, small, t, h);
+    const int which = rem / ng;
+    const int grp = rem - which * ng;
+    const uint8_t* r = recs + rec * rec_bytes;
+    const uint4* src = reinterpret_cast<const uint4*>(r + which * head_dim + grp * 32);
+    const uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
+    const float s = ue5m3_value(__ldg(r + NW * head_dim + rem));
+    const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    uint32_t o[16];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int q0 = (int)(int8_t)((w[u >> 1] >> (16 * (u & 1))) & 0xff);
-      const int q1 = (int)(int8_t)((w[u >> 1] >> (16 * (u & 1) + 8)) & 0xff);
-      const __nv_bfloat162 b2 = __floats2bfloat162_rn((float)q0 * s, (float)q1 * s);
-      o[u] = *reinterpret_cast<const uint32_t*>(&b2);
+    for (int j = 0; j < 8; ++j) {
+      const float q0 = (float)(int)(int8_t)(w[j] & 0xffu), q1 = (float)(int)(int8_t)((w[j] >> 8) & 0xffu);
+      const float q2 = (float)(int)(int8_t)((w[j] >> 16) & 0xffu), q3 = (float)(int)(int8_t)(w[j] >> 24);
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(q0 * s, q1 * s), hi = __floats2bfloat162_rn(q2 * s, q3 * s);
+      o[2 * j] = *reinterpret_cast<const uint32_t*>(&lo);
+      o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&hi);
     }
-    *reinterpret_cast<uint4*>(out + (((t * NW + which) * heads + h) * (long long)head_dim + c * 8)) =
-        make_uint4(o[0], o[1], o[2], o[3]);
+    uint4* dst = reinterpret_cast<uint4*>(out + (((t * NW + which) * heads + h) * (long long)head_dim + grp * 32));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
   }
 }
 

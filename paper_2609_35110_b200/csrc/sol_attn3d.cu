@@ -553,11 +553,9 @@ int launch_quantize(const void* const src[3], const int64_t* const strides[3], i
   a.n_ranks = n_ranks;
   a.head_dim = head_dim;
   a.rec_bytes = (int)rec_bytes;
-  const int per_rec = NW * head_dim / 8;
-  const int recs = std::min(16, 256 / per_rec);
-  const long long n_recs = n_rows * heads;
-  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((n_recs + recs - 1) / recs, 148ll * 32));
-  sol::quantize_records_kernel<NW><<<blocks, per_rec * recs, 0, st>>>(a);
+  const long long n_items = n_rows * heads * (long long)(NW * head_dim / 32);      // one thread per group of 32 values
+  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((n_items + 255) / 256, 148ll * 16));
+  sol::quantize_records_kernel<NW><<<blocks, 256, 0, st>>>(a);
   return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
 }
 }  // namespace
@@ -593,8 +591,8 @@ int launch_dequantize(const void* records, void* out, int64_t n_rows, int heads,
   if (n_rows == 0) return SOL_ATTN3D_OK;
   if (records == nullptr || out == nullptr || records == out || !aligned16(records) || !aligned16(out))
     return SOL_ATTN3D_ERR_INVALID_ARG;
-  const long long items = n_rows * (long long)heads * NW * (head_dim / 8);
-  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((items + 255) / 256, 148ll * 32));
+  const long long items = n_rows * (long long)heads * NW * (head_dim / 32);          // one thread per group of 32 values
+  const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((items + 255) / 256, 148ll * 16));
   sol::dequantize_records_kernel<NW><<<blocks, 256, 0, st>>>(static_cast<const uint8_t*>(records),
                                                               static_cast<__nv_bfloat16*>(out), n_rows, heads, head_dim,
                                                               (int)rec_bytes);
