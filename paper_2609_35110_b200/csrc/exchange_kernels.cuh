@@ -41,73 +41,73 @@ struct PackArgs {
   int chunks;                 // 16-byte chunks per head row
 };
 
-constexpr int kPackUnroll = 4;
+constexpr int kPackVec = 4;      // 16-byte chunks per thread: the index arithmetic is paid once per 64 bytes
 
 __global__ void __launch_bounds__(256) exchange_pack_qkv_kernel(const PackArgs a) {
-  // one item = one 16-byte chunk; items ordered (token, which, head, chunk): a warp reads a contiguous
-  // stretch of one source row and writes contiguous stretches of hl * row_bytes per destination
-  const int per_tok = 3 * a.heads * a.chunks;
+  // one item = up to kPackVec consecutive chunks of one head row; items ordered (token, which, head, piece):
+  // a warp reads a contiguous stretch of one source row and writes contiguous stretches of hl * row_bytes
+  const int pieces = (a.chunks + kPackVec - 1) / kPackVec;
+  const int per_tok = 3 * a.heads * pieces;
   const long long items = a.n_local * per_tok;
   const bool small = items < (1ll << 32);
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long base = (long long)blockIdx.x * blockDim.x + threadIdx.x; base < items; base += stride * kPackUnroll) {
-    uint4 v[kPackUnroll];
-    uint8_t* out[kPackUnroll];
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (long long)gridDim.x * blockDim.x) {
+    long long t;
+    int r;
+    divmod(i, per_tok, small, t, r);
+    const int which = r / (a.heads * pieces);
+    r -= which * a.heads * pieces;
+    const int h = r / pieces;
+    const int c0 = (r - h * pieces) * kPackVec;
+    const int g = h / a.hl;
+    const uint4* src = reinterpret_cast<const uint4*>(a.src[which] + t * a.tok_stride_bytes[which] +
+                                                      h * a.head_stride_bytes[which]) + c0;
+    uint4* dst = reinterpret_cast<uint4*>(a.dst[g]) + (((a.dst_row0 + t) * 3 + which) * a.hl + (h - g * a.hl)) * a.chunks + c0;
+    uint4 v[kPackVec];
 #pragma unroll
-    for (int u = 0; u < kPackUnroll; ++u) {
-      const long long i = base + u * stride;
-      out[u] = nullptr;
-      if (i < items) {
-        long long t;
-        int r;
-        divmod(i, per_tok, small, t, r);
-        const int which = r / (a.heads * a.chunks);
-        r -= which * a.heads * a.chunks;
-        const int h = r / a.chunks;
-        const int c = r - h * a.chunks;
-        const int g = h / a.hl;
-        v[u] = __ldg(reinterpret_cast<const uint4*>(a.src[which] + t * a.tok_stride_bytes[which] +
-                                                    h * a.head_stride_bytes[which] + c * 16));
-        out[u] = a.dst[g] + ((((a.dst_row0 + t) * 3 + which) * a.hl + (h - g * a.hl)) * a.chunks + c) * 16;
-      }
-    }
+    for (int u = 0; u < kPackVec; ++u)
+      if (c0 + u < a.chunks) v[u] = __ldg(src + u);
 #pragma unroll
-    for (int u = 0; u < kPackUnroll; ++u)
-      if (out[u] != nullptr) *reinterpret_cast<uint4*>(out[u]) = v[u];
+    for (int u = 0; u < kPackVec; ++u)
+      if (c0 + u < a.chunks) dst[u] = v[u];
   }
 }
 
 // Receiver's side of the output return: recv[g][t][hl][row_bytes] (what rank g computed for this rank's n
 // tokens) -> out[t][g*hl + h][row_bytes], the row-major input of the output projection.  row_bytes is
-// whatever one (token, head) record takes on the wire (2*head_dim for bf16, head_dim for raw E4M3).
+// whatever one (token, head) record takes on the wire (2*head_dim for bf16, head_dim for raw E4M3, 144 for
+// block-INT8 records).  The hl records of one (rank, token) are contiguous on both sides: one run.
+constexpr int kMergeUnroll = 4;  // independent 16-byte copies in flight per thread
+
 __global__ void __launch_bounds__(256) exchange_merge_heads_kernel(const uint8_t* __restrict__ recv,
                                                                    uint8_t* __restrict__ out, long long n, int hl,
                                                                    int n_ranks, int chunks,
                                                                    long long out_tok_stride_bytes) {
-  const int per_tok = n_ranks * hl * chunks;
+  // one item = one 16-byte chunk, adjacent lanes take adjacent chunks (measured faster here than 64 bytes per lane)
+  const int run = hl * chunks;                                  // chunks per (rank, token): contiguous on both sides
+  const int per_tok = n_ranks * run;
   const long long items = n * per_tok;
   const bool small = items < (1ll << 32);
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long base = (long long)blockIdx.x * blockDim.x + threadIdx.x; base < items; base += stride * kPackUnroll) {
-    uint4 v[kPackUnroll];
-    uint8_t* dst[kPackUnroll];
+  for (long long base = (long long)blockIdx.x * blockDim.x + threadIdx.x; base < items; base += stride * kMergeUnroll) {
+    uint4 v[kMergeUnroll];
+    uint4* dst[kMergeUnroll];
 #pragma unroll
-    for (int u = 0; u < kPackUnroll; ++u) {
+    for (int u = 0; u < kMergeUnroll; ++u) {
       const long long i = base + u * stride;
       dst[u] = nullptr;
       if (i < items) {
         long long t;
         int r;
         divmod(i, per_tok, small, t, r);
-        const int g = r / (hl * chunks);
-        r -= g * hl * chunks;                                   // (local head, chunk) within the shard
-        v[u] = __ldg(reinterpret_cast<const uint4*>(recv + (((long long)g * n + t) * hl * chunks + r) * 16));
-        dst[u] = out + t * out_tok_stride_bytes + ((long long)g * hl * chunks + r) * 16;
+        const int g = r / run;
+        r -= g * run;
+        v[u] = __ldg(reinterpret_cast<const uint4*>(recv) + ((long long)g * n + t) * run + r);
+        dst[u] = reinterpret_cast<uint4*>(out + t * out_tok_stride_bytes) + (long long)g * run + r;
       }
     }
 #pragma unroll
-    for (int u = 0; u < kPackUnroll; ++u)
-      if (dst[u] != nullptr) *reinterpret_cast<uint4*>(dst[u]) = v[u];
+    for (int u = 0; u < kMergeUnroll; ++u)
+      if (dst[u] != nullptr) *dst[u] = v[u];
   }
 }
 

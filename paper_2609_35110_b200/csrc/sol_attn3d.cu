@@ -482,8 +482,8 @@ int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, co
   a.hl = heads / n_ranks;
   a.n_ranks = n_ranks;
   a.chunks = head_dim * 2 / 16;
-  const long long items = n_local * 3ll * heads * a.chunks;
-  const long long want = (items + 256ll * sol::kPackUnroll - 1) / (256ll * sol::kPackUnroll);
+  const long long items = n_local * 3ll * heads * ((a.chunks + sol::kPackVec - 1) / sol::kPackVec);
+  const long long want = (items + 255) / 256;
   const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>(want, 148ll * 16));
   sol::exchange_pack_qkv_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
   return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
@@ -502,7 +502,7 @@ int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local
   if (ots < dense || (ots % 16) != 0) return SOL_ATTN3D_ERR_INVALID_ARG;
   const int chunks = record_bytes / 16;
   const long long items = n_local * (long long)heads * chunks;
-  const long long want = (items + 256ll * sol::kPackUnroll - 1) / (256ll * sol::kPackUnroll);
+  const long long want = (items + 256ll * sol::kMergeUnroll - 1) / (256ll * sol::kMergeUnroll);
   const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>(want, 148ll * 16));
   sol::exchange_merge_heads_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const uint8_t*>(recv), static_cast<uint8_t*>(out), n_local, heads / n_ranks, n_ranks, chunks, ots);
