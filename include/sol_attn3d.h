@@ -289,6 +289,27 @@ int sol_attn3d_forward_scatter(sol_attn3d_plan_t plan, const void* q, const void
                                int dst_heads, int head_offset, int out_format, sol_attn3d_stream_t stream);
 
 /*
+ * sol_attn3d_forward on HOST buffers: q, k, v are read from and out is written to host memory (pinned, or the
+ * copies will not overlap), through caller-owned device staging memory.  The heads are served in n_groups
+ * groups (heads are independent): the host-to-device copy of group g+1 and the device-to-host copy of group
+ * g-1 run on two internal streams while the kernels of group g run on `stream`, so that only the first
+ * group's inputs and the last group's outputs are exposed.  On return everything is enqueued; `stream` has
+ * been made to wait for the last device-to-host copy, so synchronising `stream` is enough before reading out.
+ *   q_host, k_host, v_host, out_host   HOST pointers, bf16, dense [total_tokens, heads, head_dim] (the plan must use
+ *                  the default strides); key_mask_host HOST uint8 [total_tokens] or NULL.
+ *   staging        DEVICE memory, 256-byte aligned, >= sol_attn3d_host_staging_bytes(plan) (four tensors and the
+ *                  mask), caller-owned, must stay untouched until `stream` has passed this call.
+ *   n_groups       1 .. 8; 0 = default (8); clamped to the number of heads.
+ * The first call creates two streams and a few events (no device memory); sol_attn3d_destroy releases them.
+ * Result: bit-identical to sol_attn3d_forward on device copies of the same tensors.
+ * Errors: INVALID_ARG, NO_WORKSPACE (plan workspace or staging), UNSUPPORTED_SHAPE (strided plan), CUDA.
+ */
+size_t sol_attn3d_host_staging_bytes(sol_attn3d_plan_t plan);
+int sol_attn3d_forward_host(sol_attn3d_plan_t plan, const void* q_host, const void* k_host, const void* v_host,
+                            void* out_host, const uint8_t* key_mask_host, void* staging, size_t staging_bytes,
+                            int n_groups, sol_attn3d_stream_t stream);
+
+/*
  * Block-sparse variant of sol_attn3d_forward: the per-step dynamic sparsity of Section 3.4 ("Sparse
  * Attention") with its safety rails.  An approximation of dense attention.
  *   Query blocks of 256 tokens, KV blocks of 128 tokens, per sequence and head.  Block-level score =

@@ -107,6 +107,10 @@ def _lib():
     lib.sol_attn3d_exchange_quantize_out_int8.restype = i32
     lib.sol_attn3d_exchange_dequantize_out_int8.argtypes = [vp, vp, i64, i32, i32, vp]
     lib.sol_attn3d_exchange_dequantize_out_int8.restype = i32
+    lib.sol_attn3d_host_staging_bytes.argtypes = [vp]
+    lib.sol_attn3d_host_staging_bytes.restype = ctypes.c_size_t
+    lib.sol_attn3d_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i32, vp]
+    lib.sol_attn3d_forward_host.restype = i32
     lib.sol_attn3d_sparse_workspace_bytes.argtypes = [vp]
     lib.sol_attn3d_sparse_workspace_bytes.restype = ctypes.c_size_t
     lib.sol_attn3d_forward_sparse.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, vp]
@@ -243,6 +247,26 @@ def sol_attn3d_forward_rect(plan, q, k, v, out, key_mask, query_mask: torch.Tens
         raise ValueError("query_mask must be a contiguous CUDA uint8 tensor")
     _check(_lib().sol_attn3d_forward_rect(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(key_mask), _ptr(query_mask),
                                           _stream(stream)), "sol_attn3d_forward_rect")
+
+
+def sol_attn3d_host_staging_bytes(plan) -> int:
+    return int(_lib().sol_attn3d_host_staging_bytes(plan))
+
+
+def sol_attn3d_forward_host(plan, q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor, out_host: torch.Tensor,
+                            key_mask_host: Optional[torch.Tensor], staging: torch.Tensor, n_groups: int = 0, stream=None) -> None:
+    """Forward on host tensors (pinned bf16, dense [tokens, heads, D]) through a device staging buffer; copies of one
+    head group overlap the kernels of another.  Synchronise the stream before reading out_host."""
+    for t in (q_host, k_host, v_host, out_host):
+        if t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU bf16 tensors")
+    if key_mask_host is not None and (key_mask_host.is_cuda or key_mask_host.dtype != torch.uint8 or not key_mask_host.is_contiguous()):
+        raise ValueError("key_mask_host must be a contiguous CPU uint8 tensor")
+    if not staging.is_cuda:
+        raise ValueError("staging must be a CUDA tensor")
+    _check(_lib().sol_attn3d_forward_host(plan, _ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(out_host), _ptr(key_mask_host),
+                                          _ptr(staging), staging.numel() * staging.element_size(), n_groups, _stream(stream)),
+           "sol_attn3d_forward_host")
 
 
 OUT_BF16, OUT_E4M3 = 0, 1

@@ -207,17 +207,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   if (tmem_ptr_smem[1] != 0) return;
 
   // ---- which work item
+  const int cta = (int)blockIdx.x + p.cta_offset;
   int si = 0;
-  while (si + 1 < p.n_seqs && (int)blockIdx.x >= p.seqs[si + 1].work_start) ++si;
+  while (si + 1 < p.n_seqs && cta >= p.seqs[si + 1].work_start) ++si;
   const SeqDev sq = p.seqs[si];
-  const int local = (int)blockIdx.x - sq.work_start;
+  const int local = cta - sq.work_start;
   const int head = local / sq.n_qpairs;
   const int pair = local - head * sq.n_qpairs;
+  // a launch may serve a range of heads only (CTA-uniform, before any set-up)
+  if (head < p.head_begin || head >= p.head_end) return;
   // rectangular mode: a query pair without a wanted row has nothing to do (CTA-uniform, before any set-up)
   if (p.pair_needed != nullptr && p.pair_needed[sq.pair_start + pair] == 0) return;
   // dense: every CTA of a sequence walks the same list of key tiles; block-sparse: each CTA has its own
   const bool sparse = p.cta_list != nullptr;
-  const int n_proc = sparse ? p.cta_count[blockIdx.x] : p.ktile_count[si];
+  const int n_proc = sparse ? p.cta_count[cta] : p.ktile_count[si];
   const int* __restrict__ ktiles =
       sparse ? p.cta_list + sq.sparse_list_start + (long long)local * sq.n_ktiles : p.ktile_list + sq.ktile_start;
   const uint4* __restrict__ keybits = p.keybits + sq.ktile_start;
@@ -436,7 +439,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tc_commit_elect(bar_s_full(0));
           issue_qk(tS1, q_lo1, st);
           // (test hook: CTA 0 withholds this signal so that the waits downstream run into their limit)
-          if (!(p.fault_inject == 1u && blockIdx.x == 0)) tc_commit_elect(bar_s_full(1));
+          if (!(p.fault_inject == 1u && cta == 0)) tc_commit_elect(bar_s_full(1));
           tc_commit_elect(bar_kv_empty(st));
           advance();
         }

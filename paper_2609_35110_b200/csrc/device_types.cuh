@@ -44,6 +44,8 @@ struct AttnParams {
   const SeqDev* seqs;
   int n_seqs;
   int heads;
+  int head_begin, head_end; // this launch serves heads [head_begin, head_end) (all heads: 0, heads)
+  int cta_offset;           // work item of CTA 0 of this launch (a head range of one sequence is a contiguous range)
   const uint4* keybits;     // [ktile] 128 validity bits (bit b of word w = key 32*w + b of the tile)
   const int* ktile_list;    // per sequence, tiles that hold at least one valid key, ascending
   const int* ktile_count;   // per sequence (schedule order)

@@ -91,6 +91,7 @@ struct RopeArgs {
   long long total_tokens;
   const float2* tables;
   RopeGeom g;
+  int head_begin, head_end;   // heads [head_begin, head_end) are produced by this launch
 };
 
 __global__ void __launch_bounds__(256, 4) rope_qk_kernel(const RopeArgs a) {
@@ -138,17 +139,17 @@ __global__ void __launch_bounds__(256, 4) rope_qk_kernel(const RopeArgs a) {
       __nv_bfloat16* dst = a.y[which] + (tok * a.g.heads) * (long long)a.g.head_dim + chunk * 8;
       // heads in groups of kBatch per thread: all loads of a group are issued before any is used
       constexpr int kBatch = 3;
-      for (int h0 = hsub; h0 < a.g.heads; h0 += kBatch * heads_per_pass) {
+      for (int h0 = a.head_begin + hsub; h0 < a.head_end; h0 += kBatch * heads_per_pass) {
         uint4 v[kBatch];
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
           const int h = h0 + b * heads_per_pass;
-          if (h < a.g.heads) v[b] = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
+          if (h < a.head_end) v[b] = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
         }
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
           const int h = h0 + b * heads_per_pass;
-          if (h >= a.g.heads) break;
+          if (h >= a.head_end) break;
           // all lanes of a row enter together (the bound depends on hsub only)
           const unsigned lanes = __activemask();
           const uint32_t w[4] = {v[b].x, v[b].y, v[b].z, v[b].w};

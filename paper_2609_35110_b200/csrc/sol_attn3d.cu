@@ -66,6 +66,9 @@ struct sol_attn3d_plan_s {
   unsigned int fault_inject = 0;
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
   bool prof = false, prof_valid = false, prof_bits = false;
+  // sol_attn3d_forward_host: copy streams and events, created on first use
+  cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[8] = {}, ev_out[8] = {};
 };
 
 namespace {
@@ -258,7 +261,7 @@ int encode_map(sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides s
 bool aligned16(const void* x) { return (reinterpret_cast<uintptr_t>(x) & 15u) == 0; }
 
 int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, void* kr, const float* q_gain,
-                const float* k_gain, float eps, cudaStream_t st) {
+                const float* k_gain, float eps, cudaStream_t st, int head_begin = 0, int head_end = 0) {
   sol::RopeArgs a{};
   a.gain[0] = q_gain;
   a.gain[1] = k_gain;
@@ -276,8 +279,10 @@ int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, voi
   for (int i = 0; i < 3; ++i) { a.g.rope[i] = p->rope[i]; a.g.tab_off[i] = p->tab_off[i]; }
   a.g.head_dim = p->head_dim;
   a.g.heads = p->heads;
+  a.head_begin = head_begin;
+  a.head_end = head_end > 0 ? head_end : p->heads;
   const int chunks = p->head_dim / 8;
-  const int hpp = std::max(1, std::min(p->heads, 256 / chunks));
+  const int hpp = std::max(1, std::min(a.head_end - a.head_begin, 256 / chunks));
   const int threads = chunks * hpp;
   const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
   sol::rope_qk_kernel<<<(unsigned)blocks, threads, 0, st>>>(a);
@@ -397,6 +402,8 @@ struct FwdOpts {
   void* const* dst = nullptr;
   const int64_t* tok_begin = nullptr;
   int dst_heads = 0, head_offset = 0;
+  int head_begin = 0, head_end = 0;   // serve heads [head_begin, head_end) only (0, 0 = all)
+  bool skip_keybits = false;          // the key-validity bits of this mask were built by an earlier call
 };
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
                  sol_attn3d_stream_t stream, const FwdOpts& o);
@@ -727,13 +734,15 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   int* d_list = reinterpret_cast<int*>(p->ws + p->off_list);
   int* d_count = reinterpret_cast<int*>(p->ws + p->off_count);
 
+  const int head_begin = o.head_begin, head_end = o.head_end > 0 ? o.head_end : p->heads;
+  if (head_begin < 0 || head_end > p->heads || head_begin >= head_end) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (p->prof) {
     p->prof_valid = false;
     if ((e = cudaEventRecord(p->ev[0], st)) != cudaSuccess) return fail_cuda(p, e);
   }
   // (1) validity bits per key tile: rebuilt whenever a mask is given (its contents may have changed)
   p->prof_bits = false;
-  if (key_mask != nullptr || p->keybits_state != 1) {
+  if (!o.skip_keybits && (key_mask != nullptr || p->keybits_state != 1)) {
     p->prof_bits = true;
     sol::keybits_kernel<<<p->n_seqs, 256, 0, st>>>(d_seqs, key_mask, d_bits, d_list, d_count);
     if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
@@ -743,7 +752,7 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   if (p->prof && (e = cudaEventRecord(p->ev[1], st)) != cudaSuccess) return fail_cuda(p, e);
 
   // (2) rotary prologue: Q~, K~ into the workspace
-  int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, q_gain, k_gain, eps, st);
+  int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, q_gain, k_gain, eps, st, head_begin, head_end);
   if (rc != SOL_ATTN3D_OK) return rc;
   if (p->prof && (e = cudaEventRecord(p->ev[2], st)) != cudaSuccess) return fail_cuda(p, e);
 
@@ -812,12 +821,20 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.v_lbo = p->v_lbo;
   ap.v_sbo = p->v_sbo;
   ap.fault_inject = p->fault_inject;
+  ap.head_begin = head_begin;
+  ap.head_end = head_end;
+  // one sequence: the CTAs of a head range are a contiguous range of work items; several sequences: launch
+  // everything and let the CTAs of other heads leave at the door
+  int grid = p->total_work;
+  ap.cta_offset = 0;
+  if (p->n_seqs == 1) {
+    ap.cta_offset = head_begin * p->sched[0].n_qpairs;
+    grid = (head_end - head_begin) * p->sched[0].n_qpairs;
+  }
   if (p->head_dim == 128) {
-    sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(p->tm_q, p->tm_k,
-                                                                                                      p->tm_v, ap);
+    sol::attn_fwd_kernel<128><<<grid, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(p->tm_q, p->tm_k, p->tm_v, ap);
   } else {
-    sol::attn_fwd_kernel<64><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(p->tm_q, p->tm_k,
-                                                                                                    p->tm_v, ap);
+    sol::attn_fwd_kernel<64><<<grid, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(p->tm_q, p->tm_k, p->tm_v, ap);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
   if (p->prof) {
@@ -977,6 +994,8 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
     for (int i = 0; i < 3; ++i) { a.g.rope[i] = p->rope[i]; a.g.tab_off[i] = p->tab_off[i]; }
     a.g.head_dim = p->head_dim;
     a.g.heads = p->heads;
+    a.head_begin = 0;
+    a.head_end = p->heads;
     const int chunks = p->head_dim / 8;
     const int hpp = std::max(1, std::min(p->heads, 256 / chunks));
     const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
@@ -1002,6 +1021,9 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
   ap.sink.tok_begin[1] = p->total_tokens;
   ap.sink.n_dst = 1;
   ap.sink.fmt = sol::kOutBf16;
+  ap.head_begin = 0;
+  ap.head_end = p->heads;
+  ap.cta_offset = 0;
   ap.o_tok_stride = p->so.tok;
   ap.o_head_stride = p->so.head;
   ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));
@@ -1018,6 +1040,90 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
                                                                                                     ap);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+  return SOL_ATTN3D_OK;
+}
+
+size_t sol_attn3d_host_staging_bytes(sol_attn3d_plan_t p) {
+  if (p == nullptr) return 0;
+  const size_t tensor = align_up((size_t)p->total_tokens * p->heads * p->head_dim * 2);
+  return 4 * tensor + align_up((size_t)p->total_tokens);
+}
+
+int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void* k_host, const void* v_host,
+                            void* out_host, const uint8_t* key_mask_host, void* staging, size_t staging_bytes,
+                            int n_groups, sol_attn3d_stream_t stream) {
+  if (p == nullptr || q_host == nullptr || k_host == nullptr || v_host == nullptr || out_host == nullptr)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  if (staging == nullptr || staging_bytes < sol_attn3d_host_staging_bytes(p) ||
+      (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0)
+    return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  const long long dense_tok = (long long)p->heads * p->head_dim;
+  for (const Strides* s : {&p->sq, &p->sk, &p->sv, &p->so})
+    if (s->tok != dense_tok || s->head != p->head_dim) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;   // dense tensors only
+  if (n_groups <= 0) n_groups = 8;
+  n_groups = std::min(std::min(n_groups, 8), p->heads);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if (p->s_h2d == nullptr) {
+    if ((e = cudaStreamCreateWithFlags(&p->s_h2d, cudaStreamNonBlocking)) != cudaSuccess) return fail_cuda(p, e);
+    if ((e = cudaStreamCreateWithFlags(&p->s_d2h, cudaStreamNonBlocking)) != cudaSuccess) return fail_cuda(p, e);
+    if ((e = cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
+    if ((e = cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
+    for (int g = 0; g < 8; ++g) {
+      if ((e = cudaEventCreateWithFlags(&p->ev_in[g], cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
+      if ((e = cudaEventCreateWithFlags(&p->ev_out[g], cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
+    }
+  }
+  const size_t tensor = align_up((size_t)p->total_tokens * p->heads * p->head_dim * 2);
+  unsigned char* base = static_cast<unsigned char*>(staging);
+  unsigned char* dq = base;
+  unsigned char* dk = base + tensor;
+  unsigned char* dv = base + 2 * tensor;
+  unsigned char* dout = base + 3 * tensor;
+  uint8_t* dmask = key_mask_host ? base + 4 * tensor : nullptr;
+  const size_t pitch = (size_t)dense_tok * 2;
+
+  // everything the caller queued before this call (an earlier forward reading the staging buffers included)
+  // comes before the first copy
+  if ((e = cudaEventRecord(p->ev_start, st)) != cudaSuccess) return fail_cuda(p, e);
+  if ((e = cudaStreamWaitEvent(p->s_h2d, p->ev_start, 0)) != cudaSuccess) return fail_cuda(p, e);
+  if ((e = cudaStreamWaitEvent(p->s_d2h, p->ev_start, 0)) != cudaSuccess) return fail_cuda(p, e);
+  if (dmask != nullptr &&
+      (e = cudaMemcpyAsync(dmask, key_mask_host, (size_t)p->total_tokens, cudaMemcpyHostToDevice, p->s_h2d)) != cudaSuccess)
+    return fail_cuda(p, e);
+  const bool was_prof = p->prof;
+  p->prof = false;                                   // per-kernel events describe one launch set, not a pipeline
+  int rc = SOL_ATTN3D_OK;
+  for (int g = 0; g < n_groups && rc == SOL_ATTN3D_OK; ++g) {
+    const int h0 = (int)((long long)p->heads * g / n_groups), h1 = (int)((long long)p->heads * (g + 1) / n_groups);
+    const size_t off = (size_t)h0 * p->head_dim * 2, width = (size_t)(h1 - h0) * p->head_dim * 2;
+    // K and V first: the rotary producer and the attention of this group need all three
+    const void* srcs[3] = {k_host, v_host, q_host};
+    unsigned char* dsts[3] = {dk, dv, dq};
+    for (int w = 0; w < 3; ++w)
+      if ((e = cudaMemcpy2DAsync(dsts[w] + off, pitch, static_cast<const unsigned char*>(srcs[w]) + off, pitch, width,
+                                 (size_t)p->total_tokens, cudaMemcpyHostToDevice, p->s_h2d)) != cudaSuccess)
+        return fail_cuda(p, e);
+    if ((e = cudaEventRecord(p->ev_in[g], p->s_h2d)) != cudaSuccess) return fail_cuda(p, e);
+    if ((e = cudaStreamWaitEvent(st, p->ev_in[g], 0)) != cudaSuccess) return fail_cuda(p, e);
+    FwdOpts o;
+    o.head_begin = h0;
+    o.head_end = h1;
+    o.skip_keybits = g > 0;
+    rc = forward_impl(p, dq, dk, dv, dout, dmask, stream, o);
+    if (rc != SOL_ATTN3D_OK) break;
+    if ((e = cudaEventRecord(p->ev_out[g], st)) != cudaSuccess) return fail_cuda(p, e);
+    if ((e = cudaStreamWaitEvent(p->s_d2h, p->ev_out[g], 0)) != cudaSuccess) return fail_cuda(p, e);
+    if ((e = cudaMemcpy2DAsync(static_cast<unsigned char*>(out_host) + off, pitch, dout + off, pitch, width,
+                               (size_t)p->total_tokens, cudaMemcpyDeviceToHost, p->s_d2h)) != cudaSuccess)
+      return fail_cuda(p, e);
+  }
+  p->prof = was_prof;
+  if (rc != SOL_ATTN3D_OK) return rc;
+  // the caller's stream continues only when the last rows have reached the host
+  if ((e = cudaEventRecord(p->ev_done, p->s_d2h)) != cudaSuccess) return fail_cuda(p, e);
+  if ((e = cudaStreamWaitEvent(st, p->ev_done, 0)) != cudaSuccess) return fail_cuda(p, e);
   return SOL_ATTN3D_OK;
 }
 
@@ -1055,6 +1161,16 @@ const char* sol_attn3d_strerror(int code) {
 
 int sol_attn3d_destroy(sol_attn3d_plan_t p) {
   if (p != nullptr && p->prof) (void)sol_attn3d_set_profiling(p, 0);
+  if (p != nullptr && p->s_h2d != nullptr) {
+    (void)cudaStreamDestroy(p->s_h2d);
+    (void)cudaStreamDestroy(p->s_d2h);
+    (void)cudaEventDestroy(p->ev_start);
+    (void)cudaEventDestroy(p->ev_done);
+    for (int g = 0; g < 8; ++g) {
+      (void)cudaEventDestroy(p->ev_in[g]);
+      (void)cudaEventDestroy(p->ev_out[g]);
+    }
+  }
   delete p;
   return SOL_ATTN3D_OK;
 }
