@@ -442,3 +442,42 @@ def replace_mask(inp):
     o = _I()
     o.q, o.k, o.v, o.key_mask = inp.q, inp.k, inp.v, None
     return o
+
+
+# ------------------------------------------------------------------------------------------ full size, sampled rows
+def test_full_size_lowres_e4m3_and_scatter_sampled_rows(B):
+    """The low-resolution contract shape at full size: E4M3 output, and one rank's shard of a 4-way exchange with
+    the scatter epilogue, on sampled rows of two heads against the oracle (same sampling as the bf16 parity test)."""
+    w = wl.CONFIGS["lowres"]
+    inp = wl.make_inputs(w, "cuda")
+    attn = B.Attn3d.from_workload(w, "cuda")
+    out8 = torch.full((w.total_tokens, w.heads, w.head_dim), 0x7F, dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_forward_e4m3(attn.plan, inp.q, inp.k, inp.v, out8, inp.key_mask)
+    out16 = attn.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert not bool((out8 == 0x7F).any()), "an output byte was never written"
+    attn.close()
+    qc, kc, vc = inp.q.cpu(), inp.k.cpu(), inp.v.cpu()
+    select = [(0, h, torch.from_numpy(wl.sample_rows(w, 0, h, 1024))) for h in (0, w.heads - 1)]
+    refs = orc.attn3d_oracle(qc, kc, vc, seq_tuples(w), w.rope_dims, w.theta, None, select=select)
+    for (_, h, rows), ref in zip(select, refs):
+        idx = rows.cuda()
+        print("head", h, check_e4m3(out8[idx, h], ref, out16[idx, h]))
+    # rank 1 of a 4-way exchange: heads [10, 20) from a packed QKV buffer, rows scattered to four owners
+    G, r = 4, 1
+    hl = w.heads // G
+    qkv = torch.stack((inp.q[:, r * hl:(r + 1) * hl], inp.k[:, r * hl:(r + 1) * hl], inp.v[:, r * hl:(r + 1) * hl]), dim=1).contiguous()
+    st = (3 * hl * w.head_dim, w.head_dim)
+    shard = B.Attn3d(seq_tuples(w), hl, w.head_dim, w.rope_dims, w.theta, "cuda", q_strides=st, k_strides=st, v_strides=st)
+    ranges = xo.shard_ranges(w.total_tokens, G)
+    owners = [torch.full((b - a, w.heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda") for (a, b) in ranges]
+    B.sol_attn3d_forward_scatter(shard.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], None, [o.data_ptr() for o in owners],
+                                 [a for a, _ in ranges] + [w.total_tokens], w.heads, r * hl)
+    torch.cuda.synchronize()
+    assert shard.status() == 0
+    shard.close()
+    got = torch.cat(owners, dim=0)
+    assert torch.equal(got[:, r * hl:(r + 1) * hl].view(torch.int16), out16[:, r * hl:(r + 1) * hl].view(torch.int16))
+    assert bool(torch.isnan(got[:, :r * hl].float()).all()) and bool(torch.isnan(got[:, (r + 1) * hl:].float()).all()), \
+        "the scatter epilogue wrote outside its head columns"
