@@ -124,6 +124,8 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t plan, void* device_ptr, size_t by
  *   key_mask      DEVICE pointer, uint8 [total_tokens] (i.e. [B, N]), nonzero = attend; applies to
  *                 keys only, broadcast over heads and queries; NULL = all keys valid.
  *   K and V values at masked positions must be finite (0 * inf inside the tensor core is NaN).
+ * The call only enqueues kernels (no allocation, no synchronisation, no host-device copy), so it may be
+ * stream-captured into a CUDA graph and replayed (profiling off).
  * Errors: INVALID_ARG (NULL / misaligned pointer), NO_WORKSPACE, CUDA.  Device-side time-outs are
  * reported by sol_attn3d_status after the caller has synchronised the stream.
  */

@@ -68,3 +68,32 @@ def test_exactly_one_and_two_tiles_and_partial_rope_d128():
         w = wl.Workload(name="edge", seqs=(wl.SeqSpec(0, 1, n_h, n_w),), heads=2, head_dim=128,
                         rope_dims=(0, 40, 24), seed=34)
         _check(B, w, wl.make_inputs(w, "cuda"))
+
+
+def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
+    """The forward enqueues kernels only (no allocation, no synchronisation), so it can be stream-captured once
+    and replayed; replays see the tensors' current contents."""
+    from paper_2609_35110_b200 import binding as B
+    from paper_2609_35110_b200 import workloads as wl
+    w = wl.shrunk("cfg_batch")
+    inp = wl.make_inputs(w, "cuda")
+    attn = B.Attn3d.from_workload(w, "cuda")
+    want = attn.forward(inp.q, inp.k, inp.v, inp.key_mask).clone()       # also builds the TMA map of V outside the capture
+    out = torch.zeros_like(want)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=s):
+        B.sol_attn3d_forward(attn.plan, inp.q, inp.k, inp.v, out, inp.key_mask, stream=torch.cuda.current_stream())
+    out.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, want) and attn.status() == 0
+    # new contents, same addresses: the replay recomputes
+    inp.v.mul_(2.0)
+    want2 = attn.forward(inp.q, inp.k, inp.v, inp.key_mask).clone()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, want2) and not torch.equal(want2, want)
+    attn.close()
