@@ -151,7 +151,7 @@ def cpu_sample_spec(w, scale=1.0):
     """How much oracle work to time: about 10-30 s on a 16-core host."""
     if w.name == "tiny":
         return list(range(w.heads)), 0
-    n_heads = {"lowres": 24, "highres": 6, "cfg_batch": 3, "varlen": 6}.get(w.name, 2)
+    n_heads = {"lowres": 40, "highres": 18, "cfg_batch": 9, "varlen": 18}.get(w.name, 2)
     n_heads = max(1, min(w.heads, int(round(n_heads * scale))))
     step = max(1, w.heads // n_heads)
     return list(range(0, w.heads, step))[:n_heads], (w.rows_per_head or 0)
