@@ -97,3 +97,26 @@ def test_forward_can_be_captured_in_a_cuda_graph_and_replayed():
     torch.cuda.synchronize()
     assert torch.equal(out, want2) and not torch.equal(want2, want)
     attn.close()
+
+
+def test_one_very_long_sequence_sampled_rows():
+    """262,181 tokens (2,049 key tiles, ragged tail of 37) with one head: index arithmetic far beyond the contract
+    sizes (token offsets x strides, tile counts, TMA coordinates), checked on sampled rows."""
+    from paper_2609_35110_b200 import binding as B
+    w = wl.Workload(name="long", seqs=(wl.SeqSpec(37, 64, 64, 64),), heads=1, head_dim=128, rope_dims=(32, 48, 48), seed=77)
+    assert w.total_tokens == 262181
+    inp = wl.make_inputs(w, "cuda")
+    attn = B.Attn3d.from_workload(w, "cuda")
+    out = torch.full((w.total_tokens, 1, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.sol_attn3d_forward(attn.plan, inp.q, inp.k, inp.v, out, None)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert not bool(torch.isnan(out.float()).any())
+    rows = torch.from_numpy(wl.sample_rows(w, 0, 0, 256))
+    assert int(rows[0]) == 0 and int(rows[-1]) == w.total_tokens - 1
+    ref = orc.attn3d_oracle(inp.q.cpu(), inp.k.cpu(), inp.v.cpu(), [(37, 64, 64, 64)], w.rope_dims, w.theta, None,
+                            select=[(0, 0, rows)])[0]
+    max_abs, rel_l2 = orc.compare(out[rows.cuda(), 0].cpu(), ref)
+    print("long:", max_abs, rel_l2)
+    assert max_abs <= 2e-2 and rel_l2 <= 5e-3
+    attn.close()
