@@ -203,13 +203,16 @@ int sol_attn3d_forward_e4m3(sol_attn3d_plan_t plan, const void* q, const void* k
  *              barrier across ranks before the attention reads the buffer.
  * After the exchange rank g holds [total_tokens][3][heads/n_ranks][head_dim]; its Q, K, V are views with
  * token stride 3*heads/n_ranks*head_dim that sol_attn3d_plan_ex takes as they are.
+ *   group_begin, group_heads   send only heads [group_begin, group_begin + group_heads) of every rank's shard (a head
+ *              group; rows then hold group_heads heads), so that the exchange of one group can run under the
+ *              attention of another; 0, 0 = the whole shard.
  * n_local = 0 is a no-op (pointers are not looked at).
  * Errors: INVALID_ARG (NULL / misaligned pointer, heads not divisible, n_ranks > SOL_ATTN3D_MAX_RANKS), CUDA.
  */
 int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, const int64_t q_strides[2],
                                  const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
-                                 int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
-                                 sol_attn3d_stream_t stream);
+                                 int head_dim, int n_ranks, int group_begin, int group_heads, void* const* dst,
+                                 int64_t dst_row0, sol_attn3d_stream_t stream);
 
 /*
  * Receiver's side of the output return (the paper's "inverse head merge"): recv [n_ranks][n_local]
@@ -217,9 +220,13 @@ int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, co
  * out [n_local][heads][record_bytes] with head = g*heads/n_ranks + local head, the row-major input of the
  * output projection.  record_bytes is the size of one (token, head) record on the wire, a multiple of 16:
  * 2*head_dim for bf16, head_dim for raw E4M3.  out_tok_stride_bytes: 0 = dense.  recv and out must not alias.
+ * out_rank_stride_bytes: distance between rank g's and rank g+1's heads inside an output row; 0 = adjacent
+ * (heads/n_ranks * record_bytes).  When recv holds one head group of every rank, pass the full shard's size here
+ * and point `out` at the group's first head: the group lands in its place in the full row.
  */
 int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local, int heads, int record_bytes,
-                                    int n_ranks, int64_t out_tok_stride_bytes, sol_attn3d_stream_t stream);
+                                    int n_ranks, int64_t out_tok_stride_bytes, int64_t out_rank_stride_bytes,
+                                    sol_attn3d_stream_t stream);
 
 /*
  * Quantized wire formats of the exchange (Section 3.3, "Quantized communication").  One record per (token,
@@ -249,8 +256,8 @@ size_t sol_attn3d_exchange_record_bytes(int kind, int head_dim);
  */
 int sol_attn3d_exchange_pack_qkv_int8(const void* q, const void* k, const void* v, const int64_t q_strides[2],
                                       const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
-                                      int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
-                                      sol_attn3d_stream_t stream);
+                                      int head_dim, int n_ranks, int group_begin, int group_heads, void* const* dst,
+                                      int64_t dst_row0, sol_attn3d_stream_t stream);
 
 /*
  * Receiver's side: records [n_rows][heads][record_bytes(QKV_INT8)] (DEVICE; heads = this rank's shard) -> qkv

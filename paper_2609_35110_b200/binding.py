@@ -93,9 +93,9 @@ def _lib():
                                                i32, vp]
     lib.sol_attn3d_forward_scatter.restype = i32
     lib.sol_attn3d_exchange_pack_qkv.argtypes = [vp, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i64),
-                                                 i64, i32, i32, i32, ctypes.POINTER(vp), i64, vp]
+                                                 i64, i32, i32, i32, i32, i32, ctypes.POINTER(vp), i64, vp]
     lib.sol_attn3d_exchange_pack_qkv.restype = i32
-    lib.sol_attn3d_exchange_merge_heads.argtypes = [vp, vp, i64, i32, i32, i32, i64, vp]
+    lib.sol_attn3d_exchange_merge_heads.argtypes = [vp, vp, i64, i32, i32, i32, i64, i64, vp]
     lib.sol_attn3d_exchange_merge_heads.restype = i32
     lib.sol_attn3d_exchange_record_bytes.argtypes = [i32, i32]
     lib.sol_attn3d_exchange_record_bytes.restype = ctypes.c_size_t
@@ -309,8 +309,10 @@ def _strides_of(t: torch.Tensor, head_dim: int):
     return (ctypes.c_int64 * 2)(tok, t.stride(1) if t.shape[1] > 1 else head_dim)
 
 
-def sol_attn3d_exchange_pack_qkv(q, k, v, n_ranks: int, dst: Sequence[int], dst_row0: int = 0, stream=None) -> None:
-    """q, k, v: CUDA bf16 [n_local, heads, D] (any token / head strides); dst: n_ranks device addresses."""
+def sol_attn3d_exchange_pack_qkv(q, k, v, n_ranks: int, dst: Sequence[int], dst_row0: int = 0, stream=None,
+                                 group_begin: int = 0, group_heads: int = 0) -> None:
+    """q, k, v: CUDA bf16 [n_local, heads, D] (any token / head strides); dst: n_ranks device addresses.
+    group_begin / group_heads: send only that head group of every rank's shard (0, 0 = the whole shard)."""
     n_local, heads, head_dim = q.shape
     for t in (q, k, v):
         if not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != (n_local, heads, head_dim):
@@ -318,8 +320,8 @@ def sol_attn3d_exchange_pack_qkv(q, k, v, n_ranks: int, dst: Sequence[int], dst_
     if len(dst) != n_ranks:
         raise ValueError("one destination per rank")
     _check(_lib().sol_attn3d_exchange_pack_qkv(_ptr(q), _ptr(k), _ptr(v), _strides_of(q, head_dim), _strides_of(k, head_dim),
-                                               _strides_of(v, head_dim), n_local, heads, head_dim, n_ranks,
-                                               _ptr_array(dst), dst_row0, _stream(stream)),
+                                               _strides_of(v, head_dim), n_local, heads, head_dim, n_ranks, group_begin,
+                                               group_heads, _ptr_array(dst), dst_row0, _stream(stream)),
            "sol_attn3d_exchange_pack_qkv")
 
 
@@ -333,7 +335,8 @@ def sol_attn3d_exchange_record_bytes(kind: int, head_dim: int) -> int:
     return n
 
 
-def sol_attn3d_exchange_pack_qkv_int8(q, k, v, n_ranks: int, dst: Sequence[int], dst_row0: int = 0, stream=None) -> None:
+def sol_attn3d_exchange_pack_qkv_int8(q, k, v, n_ranks: int, dst: Sequence[int], dst_row0: int = 0, stream=None,
+                                      group_begin: int = 0, group_heads: int = 0) -> None:
     """As sol_attn3d_exchange_pack_qkv, but the destinations receive block-INT8 records."""
     n_local, heads, head_dim = q.shape
     for t in (q, k, v):
@@ -343,7 +346,8 @@ def sol_attn3d_exchange_pack_qkv_int8(q, k, v, n_ranks: int, dst: Sequence[int],
         raise ValueError("one destination per rank")
     _check(_lib().sol_attn3d_exchange_pack_qkv_int8(_ptr(q), _ptr(k), _ptr(v), _strides_of(q, head_dim),
                                                     _strides_of(k, head_dim), _strides_of(v, head_dim), n_local, heads,
-                                                    head_dim, n_ranks, _ptr_array(dst), dst_row0, _stream(stream)),
+                                                    head_dim, n_ranks, group_begin, group_heads, _ptr_array(dst), dst_row0,
+                                                    _stream(stream)),
            "sol_attn3d_exchange_pack_qkv_int8")
 
 
@@ -372,12 +376,14 @@ def sol_attn3d_exchange_dequantize_out_int8(records: torch.Tensor, out_rows: tor
                                                           _stream(stream)), "sol_attn3d_exchange_dequantize_out_int8")
 
 
-def sol_attn3d_exchange_merge_heads(recv: torch.Tensor, out: torch.Tensor, n_local: int, heads: int, record_bytes: int,
-                                    n_ranks: int, out_tok_stride_bytes: int = 0, stream=None) -> None:
-    if not recv.is_cuda or not out.is_cuda or not recv.is_contiguous():
-        raise ValueError("recv and out must be CUDA tensors, recv contiguous")
-    _check(_lib().sol_attn3d_exchange_merge_heads(_ptr(recv), _ptr(out), n_local, heads, record_bytes, n_ranks,
-                                                  out_tok_stride_bytes, _stream(stream)),
+def sol_attn3d_exchange_merge_heads(recv: torch.Tensor, out, n_local: int, heads: int, record_bytes: int,
+                                    n_ranks: int, out_tok_stride_bytes: int = 0, stream=None, out_rank_stride_bytes: int = 0) -> None:
+    """out: CUDA tensor, or a device address (int) when the rows start inside a larger tensor."""
+    if not recv.is_cuda or not recv.is_contiguous():
+        raise ValueError("recv must be a contiguous CUDA tensor")
+    out_ptr = ctypes.c_void_p(int(out)) if isinstance(out, int) else _ptr(out)
+    _check(_lib().sol_attn3d_exchange_merge_heads(_ptr(recv), out_ptr, n_local, heads, record_bytes, n_ranks,
+                                                  out_tok_stride_bytes, out_rank_stride_bytes, _stream(stream)),
            "sol_attn3d_exchange_merge_heads")
 
 

@@ -38,6 +38,8 @@ struct PackArgs {
   long long dst_row0;
   long long n_local;
   int heads, hl, n_ranks;
+  int h_begin, hg;            // of each rank's hl heads, heads [h_begin, h_begin + hg) are sent (a head group);
+                              // destination rows then hold hg heads: [row][3][hg][row_bytes]
   int chunks;                 // 16-byte chunks per head row
 };
 
@@ -47,21 +49,24 @@ __global__ void __launch_bounds__(256) exchange_pack_qkv_kernel(const PackArgs a
   // one item = up to kPackVec consecutive chunks of one head row; items ordered (token, which, head, piece):
   // a warp reads a contiguous stretch of one source row and writes contiguous stretches of hl * row_bytes
   const int pieces = (a.chunks + kPackVec - 1) / kPackVec;
-  const int per_tok = 3 * a.heads * pieces;
+  const int sent = a.n_ranks * a.hg;                            // heads sent per token
+  const int per_tok = 3 * sent * pieces;
   const long long items = a.n_local * per_tok;
   const bool small = items < (1ll << 32);
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < items; i += (long long)gridDim.x * blockDim.x) {
     long long t;
     int r;
     divmod(i, per_tok, small, t, r);
-    const int which = r / (a.heads * pieces);
-    r -= which * a.heads * pieces;
-    const int h = r / pieces;
-    const int c0 = (r - h * pieces) * kPackVec;
-    const int g = h / a.hl;
+    const int which = r / (sent * pieces);
+    r -= which * sent * pieces;
+    const int hs = r / pieces;                                  // index among the heads sent
+    const int c0 = (r - hs * pieces) * kPackVec;
+    const int g = hs / a.hg;
+    const int hj = hs - g * a.hg;                               // head within the group
+    const int h = g * a.hl + a.h_begin + hj;                    // head of the source tensor
     const uint4* src = reinterpret_cast<const uint4*>(a.src[which] + t * a.tok_stride_bytes[which] +
                                                       h * a.head_stride_bytes[which]) + c0;
-    uint4* dst = reinterpret_cast<uint4*>(a.dst[g]) + (((a.dst_row0 + t) * 3 + which) * a.hl + (h - g * a.hl)) * a.chunks + c0;
+    uint4* dst = reinterpret_cast<uint4*>(a.dst[g]) + (((a.dst_row0 + t) * 3 + which) * a.hg + hj) * a.chunks + c0;
     uint4 v[kPackVec];
 #pragma unroll
     for (int u = 0; u < kPackVec; ++u)
@@ -75,13 +80,15 @@ __global__ void __launch_bounds__(256) exchange_pack_qkv_kernel(const PackArgs a
 // Receiver's side of the output return: recv[g][t][hl][row_bytes] (what rank g computed for this rank's n
 // tokens) -> out[t][g*hl + h][row_bytes], the row-major input of the output projection.  row_bytes is
 // whatever one (token, head) record takes on the wire (2*head_dim for bf16, head_dim for raw E4M3, 144 for
-// block-INT8 records).  The hl records of one (rank, token) are contiguous on both sides: one run.
+// block-INT8 records).  The hl records of one (rank, token) are contiguous on both sides: one run.  Rank g's run
+// starts out_rank_chunks 16-byte chunks after rank g-1's in an output row (hl * chunks when recv holds all of a
+// rank's heads; larger when recv holds one head group of each rank and out is the full row).
 constexpr int kMergeUnroll = 4;  // independent 16-byte copies in flight per thread
 
 __global__ void __launch_bounds__(256) exchange_merge_heads_kernel(const uint8_t* __restrict__ recv,
                                                                    uint8_t* __restrict__ out, long long n, int hl,
                                                                    int n_ranks, int chunks,
-                                                                   long long out_tok_stride_bytes) {
+                                                                   long long out_tok_stride_bytes, int out_rank_chunks) {
   // one item = one 16-byte chunk, adjacent lanes take adjacent chunks (measured faster here than 64 bytes per lane)
   const int run = hl * chunks;                                  // chunks per (rank, token): contiguous on both sides
   const int per_tok = n_ranks * run;
@@ -102,7 +109,7 @@ __global__ void __launch_bounds__(256) exchange_merge_heads_kernel(const uint8_t
         const int g = r / run;
         r -= g * run;
         v[u] = __ldg(reinterpret_cast<const uint4*>(recv) + ((long long)g * n + t) * run + r);
-        dst[u] = reinterpret_cast<uint4*>(out + t * out_tok_stride_bytes) + (long long)g * run + r;
+        dst[u] = reinterpret_cast<uint4*>(out + t * out_tok_stride_bytes) + (long long)g * out_rank_chunks + r;
       }
     }
 #pragma unroll
@@ -149,6 +156,7 @@ struct QuantArgs {
   long long dst_row0;
   long long n_rows;
   int heads, hl, n_ranks;
+  int h_begin, hg;                      // head group, as in PackArgs
   int head_dim, rec_bytes;
 };
 
@@ -171,13 +179,17 @@ template <int NW>
 __global__ void __launch_bounds__(256) quantize_records_kernel(const QuantArgs a) {
   const int ng = a.head_dim >> 5;                               // groups (= scale codes) per tensor
   const int per_rec = NW * ng;                                  // threads per record
-  const long long n_items = a.n_rows * a.heads * per_rec;
+  const int sent = a.n_ranks * a.hg;                            // heads (records) written per token
+  const long long n_items = a.n_rows * sent * per_rec;
   const bool small = n_items < (1ll << 32);
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_items; i += (long long)gridDim.x * blockDim.x) {
     long long rec, t;
-    int rem, h;
+    int rem, hs;
     divmod(i, per_rec, small, rec, rem);
-    divmod(rec, a.heads, small, t, h);
+    divmod(rec, sent, small, t, hs);
+    const int g = hs / a.hg;
+    const int hj = hs - g * a.hg;
+    const int h = g * a.hl + a.h_begin + hj;                    // head of the source tensor
     const int which = rem / ng;
     const int grp = rem - which * ng;
     const uint4* src = reinterpret_cast<const uint4*>(a.src[which] + t * a.tok_stride_bytes[which] +
@@ -205,8 +217,7 @@ __global__ void __launch_bounds__(256) quantize_records_kernel(const QuantArgs a
     for (int j = 0; j < 8; ++j)
       o[j] = pack_low_bytes(rint_sat_s8(__fmul_rn(f[4 * j], inv)), rint_sat_s8(__fmul_rn(f[4 * j + 1], inv)),
                             rint_sat_s8(__fmul_rn(f[4 * j + 2], inv)), rint_sat_s8(__fmul_rn(f[4 * j + 3], inv)));
-    const int g = h / a.hl;
-    uint8_t* out = a.dst[g] + ((a.dst_row0 + t) * a.hl + (h - g * a.hl)) * a.rec_bytes;
+    uint8_t* out = a.dst[g] + ((a.dst_row0 + t) * a.hg + hj) * a.rec_bytes;
     uint4* dst = reinterpret_cast<uint4*>(out + which * a.head_dim + grp * 32);
     dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
     dst[1] = make_uint4(o[4], o[5], o[6], o[7]);

@@ -69,6 +69,7 @@ struct sol_attn3d_plan_s {
   // sol_attn3d_forward_host: copy streams and events, created on first use
   cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
   cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[8] = {}, ev_out[8] = {};
+  bool host_pipe_ready = false;
 };
 
 namespace {
@@ -77,6 +78,22 @@ int fail_cuda(sol_attn3d_plan_t p, cudaError_t e) {
   p->last_cuda = (int)e;
   (void)cudaGetLastError();
   return SOL_ATTN3D_ERR_CUDA;
+}
+
+// Streams and events of sol_attn3d_forward_host (host-side objects only).
+void release_host_pipe(sol_attn3d_plan_t p) {
+  if (p->s_h2d != nullptr) (void)cudaStreamDestroy(p->s_h2d);
+  if (p->s_d2h != nullptr) (void)cudaStreamDestroy(p->s_d2h);
+  if (p->ev_start != nullptr) (void)cudaEventDestroy(p->ev_start);
+  if (p->ev_done != nullptr) (void)cudaEventDestroy(p->ev_done);
+  for (int g = 0; g < 8; ++g) {
+    if (p->ev_in[g] != nullptr) (void)cudaEventDestroy(p->ev_in[g]);
+    if (p->ev_out[g] != nullptr) (void)cudaEventDestroy(p->ev_out[g]);
+    p->ev_in[g] = p->ev_out[g] = nullptr;
+  }
+  p->s_h2d = p->s_d2h = nullptr;
+  p->ev_start = p->ev_done = nullptr;
+  p->host_pipe_ready = false;
 }
 
 bool stride_ok(long long s) { return s > 0 && (s * 2) % 16 == 0 && (s * 2) < (1ll << 40); }
@@ -459,11 +476,13 @@ int sol_attn3d_forward_scatter(sol_attn3d_plan_t p, const void* q, const void* k
 
 int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, const int64_t q_strides[2],
                                  const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
-                                 int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
-                                 sol_attn3d_stream_t stream) {
+                                 int head_dim, int n_ranks, int group_begin, int group_heads, void* const* dst,
+                                 int64_t dst_row0, sol_attn3d_stream_t stream) {
   if (n_local < 0 || dst_row0 < 0 || heads < 1 || head_dim < 8 || (head_dim % 8) != 0 || n_ranks < 1 ||
       n_ranks > sol::kMaxRanks || (heads % n_ranks) != 0)
     return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (group_heads == 0) group_heads = heads / n_ranks - group_begin;
+  if (group_begin < 0 || group_heads < 1 || group_begin + group_heads > heads / n_ranks) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (n_local == 0) return SOL_ATTN3D_OK;            // a rank without tokens sends nothing (its pointers may be NULL)
   if (q == nullptr || k == nullptr || v == nullptr || dst == nullptr || q_strides == nullptr || k_strides == nullptr ||
       v_strides == nullptr)
@@ -488,8 +507,10 @@ int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, co
   a.heads = heads;
   a.hl = heads / n_ranks;
   a.n_ranks = n_ranks;
+  a.h_begin = group_begin;
+  a.hg = group_heads;
   a.chunks = head_dim * 2 / 16;
-  const long long items = n_local * 3ll * heads * ((a.chunks + sol::kPackVec - 1) / sol::kPackVec);
+  const long long items = n_local * 3ll * n_ranks * group_heads * ((a.chunks + sol::kPackVec - 1) / sol::kPackVec);
   const long long want = (items + 255) / 256;
   const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>(want, 148ll * 16));
   sol::exchange_pack_qkv_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
@@ -497,14 +518,18 @@ int sol_attn3d_exchange_pack_qkv(const void* q, const void* k, const void* v, co
 }
 
 int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local, int heads, int record_bytes,
-                                    int n_ranks, int64_t out_tok_stride_bytes, sol_attn3d_stream_t stream) {
+                                    int n_ranks, int64_t out_tok_stride_bytes, int64_t out_rank_stride_bytes,
+                                    sol_attn3d_stream_t stream) {
   if (n_local < 0 || heads < 1 || record_bytes < 16 || (record_bytes % 16) != 0 || n_ranks < 1 ||
       n_ranks > sol::kMaxRanks || (heads % n_ranks) != 0)
     return SOL_ATTN3D_ERR_INVALID_ARG;
   if (n_local == 0) return SOL_ATTN3D_OK;            // a rank without tokens receives nothing
   if (recv == nullptr || out == nullptr || recv == out || !aligned16(recv) || !aligned16(out))
     return SOL_ATTN3D_ERR_INVALID_ARG;
-  const long long dense = (long long)heads * record_bytes;
+  const long long run_bytes = (long long)(heads / n_ranks) * record_bytes;
+  const long long ors = out_rank_stride_bytes == 0 ? run_bytes : out_rank_stride_bytes;
+  if (ors < run_bytes || (ors % 16) != 0) return SOL_ATTN3D_ERR_INVALID_ARG;
+  const long long dense = ors * (n_ranks - 1) + run_bytes;
   const long long ots = out_tok_stride_bytes == 0 ? dense : out_tok_stride_bytes;
   if (ots < dense || (ots % 16) != 0) return SOL_ATTN3D_ERR_INVALID_ARG;
   const int chunks = record_bytes / 16;
@@ -512,7 +537,8 @@ int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local
   const long long want = (items + 256ll * sol::kMergeUnroll - 1) / (256ll * sol::kMergeUnroll);
   const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>(want, 148ll * 16));
   sol::exchange_merge_heads_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<const uint8_t*>(recv), static_cast<uint8_t*>(out), n_local, heads / n_ranks, n_ranks, chunks, ots);
+      static_cast<const uint8_t*>(recv), static_cast<uint8_t*>(out), n_local, heads / n_ranks, n_ranks, chunks, ots,
+      (int)(ors / 16));
   return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
 }
 
@@ -533,10 +559,13 @@ extern "C++" {
 namespace {
 template <int NW>
 int launch_quantize(const void* const src[3], const int64_t* const strides[3], int64_t n_rows, int heads, int head_dim,
-                    int n_ranks, void* const* dst, int64_t dst_row0, size_t rec_bytes, cudaStream_t st) {
+                    int n_ranks, int group_begin, int group_heads, void* const* dst, int64_t dst_row0, size_t rec_bytes,
+                    cudaStream_t st) {
   if (n_rows < 0 || dst_row0 < 0 || heads < 1 || (head_dim != 64 && head_dim != 128) || n_ranks < 1 ||
       n_ranks > sol::kMaxRanks || (heads % n_ranks) != 0)
     return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (group_heads == 0) group_heads = heads / n_ranks - group_begin;
+  if (group_begin < 0 || group_heads < 1 || group_begin + group_heads > heads / n_ranks) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (n_rows == 0) return SOL_ATTN3D_OK;
   if (dst == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   sol::QuantArgs a{};
@@ -558,9 +587,11 @@ int launch_quantize(const void* const src[3], const int64_t* const strides[3], i
   a.heads = heads;
   a.hl = heads / n_ranks;
   a.n_ranks = n_ranks;
+  a.h_begin = group_begin;
+  a.hg = group_heads;
   a.head_dim = head_dim;
   a.rec_bytes = (int)rec_bytes;
-  const long long n_items = n_rows * heads * (long long)(NW * head_dim / 32);      // one thread per group of 32 values
+  const long long n_items = n_rows * n_ranks * group_heads * (long long)(NW * head_dim / 32);   // one thread per group of 32 values
   const unsigned blocks = (unsigned)std::max<long long>(1, std::min<long long>((n_items + 255) / 256, 148ll * 16));
   sol::quantize_records_kernel<NW><<<blocks, 256, 0, st>>>(a);
   return cudaGetLastError() == cudaSuccess ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_CUDA;
@@ -570,11 +601,11 @@ int launch_quantize(const void* const src[3], const int64_t* const strides[3], i
 
 int sol_attn3d_exchange_pack_qkv_int8(const void* q, const void* k, const void* v, const int64_t q_strides[2],
                                       const int64_t k_strides[2], const int64_t v_strides[2], int64_t n_local, int heads,
-                                      int head_dim, int n_ranks, void* const* dst, int64_t dst_row0,
-                                      sol_attn3d_stream_t stream) {
+                                      int head_dim, int n_ranks, int group_begin, int group_heads, void* const* dst,
+                                      int64_t dst_row0, sol_attn3d_stream_t stream) {
   const void* const src[3] = {q, k, v};
   const int64_t* const strides[3] = {q_strides, k_strides, v_strides};
-  return launch_quantize<3>(src, strides, n_local, heads, head_dim, n_ranks, dst, dst_row0,
+  return launch_quantize<3>(src, strides, n_local, heads, head_dim, n_ranks, group_begin, group_heads, dst, dst_row0,
                             sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_QKV_INT8, head_dim),
                             static_cast<cudaStream_t>(stream));
 }
@@ -584,7 +615,7 @@ int sol_attn3d_exchange_quantize_out_int8(const void* out_rows, const int64_t ou
   const void* const src[3] = {out_rows, nullptr, nullptr};
   const int64_t* const strides[3] = {out_strides, nullptr, nullptr};
   void* const dst[1] = {records};
-  return launch_quantize<1>(src, strides, n_rows, heads, head_dim, 1, dst, 0,
+  return launch_quantize<1>(src, strides, n_rows, heads, head_dim, 1, 0, 0, dst, 0,
                             sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_OUT_INT8, head_dim),
                             static_cast<cudaStream_t>(stream));
 }
@@ -1065,15 +1096,20 @@ int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void*
   n_groups = std::min(std::min(n_groups, 8), p->heads);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
-  if (p->s_h2d == nullptr) {
-    if ((e = cudaStreamCreateWithFlags(&p->s_h2d, cudaStreamNonBlocking)) != cudaSuccess) return fail_cuda(p, e);
-    if ((e = cudaStreamCreateWithFlags(&p->s_d2h, cudaStreamNonBlocking)) != cudaSuccess) return fail_cuda(p, e);
-    if ((e = cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
-    if ((e = cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
-    for (int g = 0; g < 8; ++g) {
-      if ((e = cudaEventCreateWithFlags(&p->ev_in[g], cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
-      if ((e = cudaEventCreateWithFlags(&p->ev_out[g], cudaEventDisableTiming)) != cudaSuccess) return fail_cuda(p, e);
+  if (!p->host_pipe_ready) {
+    e = cudaStreamCreateWithFlags(&p->s_h2d, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->s_d2h, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming);
+    for (int g = 0; g < 8 && e == cudaSuccess; ++g) {
+      e = cudaEventCreateWithFlags(&p->ev_in[g], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_out[g], cudaEventDisableTiming);
     }
+    if (e != cudaSuccess) {
+      release_host_pipe(p);                          // whatever was created goes away again; the next call retries
+      return fail_cuda(p, e);
+    }
+    p->host_pipe_ready = true;
   }
   const size_t tensor = align_up((size_t)p->total_tokens * p->heads * p->head_dim * 2);
   unsigned char* base = static_cast<unsigned char*>(staging);
@@ -1161,16 +1197,7 @@ const char* sol_attn3d_strerror(int code) {
 
 int sol_attn3d_destroy(sol_attn3d_plan_t p) {
   if (p != nullptr && p->prof) (void)sol_attn3d_set_profiling(p, 0);
-  if (p != nullptr && p->s_h2d != nullptr) {
-    (void)cudaStreamDestroy(p->s_h2d);
-    (void)cudaStreamDestroy(p->s_d2h);
-    (void)cudaEventDestroy(p->ev_start);
-    (void)cudaEventDestroy(p->ev_done);
-    for (int g = 0; g < 8; ++g) {
-      (void)cudaEventDestroy(p->ev_in[g]);
-      (void)cudaEventDestroy(p->ev_out[g]);
-    }
-  }
+  if (p != nullptr) release_host_pipe(p);
   delete p;
   return SOL_ATTN3D_OK;
 }

@@ -45,26 +45,58 @@ class ExchangePlan:
         self.tok_begin = [a for a, _ in self.ranges] + [total_tokens]
         self.n_local = self.ranges[rank][1] - self.ranges[rank][0]
         self.first_token = self.ranges[rank][0]
-        qkv_row = self.hl * (qkv_record_elems or 3 * head_dim)  # elements per token in the QKV exchange
-        # split sizes are in ELEMENTS of the exchanged tensors
-        # QKV exchange: this rank sends n_local rows to everyone and receives n_s rows from rank s
-        self.qkv_send_splits = [self.n_local * qkv_row] * n_ranks
-        self.qkv_recv_splits = [(b - a) * qkv_row for a, b in self.ranges]
-        out_row = self.hl * (out_record_elems or head_dim)      # elements per token in the output return
+        self.qkv_record_elems = qkv_record_elems or 3 * head_dim
+        self.out_record_elems = out_record_elems or head_dim
         self.out_record_bytes = out_record_bytes               # bytes of one (token, head) record on the wire
-        # output return: this rank owes rows [a_g, b_g) to rank g and receives its own n_local rows from everyone
-        self.out_send_splits = [(b - a) * out_row for a, b in self.ranges]
-        self.out_recv_splits = [self.n_local * out_row] * n_ranks
+        (self.qkv_send_splits, self.qkv_recv_splits, self.out_send_splits, self.out_recv_splits) = self.splits(self.hl)
+
+    def splits(self, group_heads: int):
+        """Split sizes, in ELEMENTS of the exchanged tensors, when `group_heads` heads of every rank's shard travel:
+        (qkv send, qkv receive, output send, output receive).  QKV: this rank sends its n_local rows to everyone
+        and receives n_s rows from rank s.  Output: it owes rows [a_g, b_g) to rank g and receives its own
+        n_local rows from everyone."""
+        qkv_row = group_heads * self.qkv_record_elems
+        out_row = group_heads * self.out_record_elems
+        return ([self.n_local * qkv_row] * self.n_ranks, [(b - a) * qkv_row for a, b in self.ranges],
+                [(b - a) * out_row for a, b in self.ranges], [self.n_local * out_row] * self.n_ranks)
+
+
+class _HeadGroup:
+    """Buffers and plan of one head group of this rank's shard (collective transport)."""
+
+    def __init__(self, sp, seqs, begin: int, count: int, rope_dims, theta, device):
+        xp, D, G, n_local, total = sp.xp, sp.head_dim, sp.n_ranks, sp.xp.n_local, sp.xp.total
+        self.begin, self.count = begin, count
+        self.qkv_send_splits, self.qkv_recv_splits, self.out_send_splits, self.out_recv_splits = xp.splits(count)
+        st = (3 * count * D, D)
+        self.attn = B.Attn3d(seqs, count, D, rope_dims, theta, device, q_strides=st, k_strides=st, v_strides=st)
+        self.qkv = torch.empty((total, 3, count, D), dtype=torch.bfloat16, device=device)
+        if sp.qkv_int8:
+            self.send = torch.empty((G, n_local, count, sp.rb_in), dtype=torch.uint8, device=device)
+            self.qkv_records = torch.empty((total, count, sp.rb_in), dtype=torch.uint8, device=device)
+        else:
+            self.send = torch.empty((G, n_local, 3, count, D), dtype=torch.bfloat16, device=device)
+        self.out_shard = torch.empty((total, count, D), dtype=sp.out_dtype, device=device)
+        if sp.out_int8:
+            self.out_records = torch.empty((total, count, sp.rb_out), dtype=torch.uint8, device=device)
+            self.recv_out = torch.empty((G, n_local, count, sp.rb_out), dtype=torch.uint8, device=device)
+        else:
+            self.recv_out = torch.empty((G, n_local, count, D), dtype=sp.out_dtype, device=device)
+        self.ev_in = torch.cuda.Event()
+        self.ev_out = torch.cuda.Event()
 
 
 class SequenceParallelAttn3d:
     """One DiT-block attention over a sequence-sharded Q, K, V.  forward() returns this rank's token rows."""
 
     def __init__(self, seqs: Sequence[Tuple[int, int, int, int]], heads: int, head_dim: int, rope_dims, theta: float = 10000.0,
-                 group=None, device="cuda", out_format: str = "bf16", transport: str = "collective", qkv_wire: str = "bf16"):
+                 group=None, device="cuda", out_format: str = "bf16", transport: str = "collective", qkv_wire: str = "bf16",
+                 n_groups: int = 1):
         """out_format: what travels back and is returned -- "bf16", "e4m3" (raw bytes, returned as uint8) or "int8"
         (block-INT8 records on the wire, dequantised to bf16 on arrival).  qkv_wire: "bf16" or "int8" (block-INT8
-        records on the wire, dequantised to bf16 before the attention).  The quantised formats are approximate."""
+        records on the wire, dequantised to bf16 before the attention).  The quantised formats are approximate.
+        n_groups (collective transport): this rank's head shard is served in that many head groups; the exchanges
+        of one group run on side streams under the attention of another (heads are independent)."""
         import torch.distributed as dist
         self.dist = dist
         self.group = group
@@ -76,8 +108,8 @@ class SequenceParallelAttn3d:
             raise ValueError("qkv_wire: 'bf16' or 'int8'")
         if transport not in ("collective", "peer"):
             raise ValueError("transport: 'collective' or 'peer'")
-        if transport == "peer" and (qkv_wire != "bf16" or out_format == "int8"):
-            raise ValueError("transport 'peer' carries bf16 QKV and bf16 / e4m3 output")
+        if transport == "peer" and (qkv_wire != "bf16" or out_format == "int8" or n_groups != 1):
+            raise ValueError("transport 'peer' carries bf16 QKV and bf16 / e4m3 output, in one group")
         self.fp8 = out_format == "e4m3"
         self.out_int8 = out_format == "int8"
         self.qkv_int8 = qkv_wire == "int8"
@@ -92,26 +124,19 @@ class SequenceParallelAttn3d:
                                qkv_record_elems=self.rb_in if self.qkv_int8 else 0,
                                out_record_elems=self.rb_out if self.out_int8 else 0)
         hl = self.xp.hl
-        qkv_strides = (3 * hl * D, D)
-        self.attn = B.Attn3d(seqs, hl, D, rope_dims, theta, device, q_strides=qkv_strides, k_strides=qkv_strides,
-                             v_strides=qkv_strides)
         self.out_dtype = torch.uint8 if self.fp8 else torch.bfloat16
-        n_local = self.xp.n_local
         if transport == "collective":
-            self.qkv = torch.empty((total, 3, hl, D), dtype=torch.bfloat16, device=device)
-            if self.qkv_int8:
-                self.send = torch.empty((self.n_ranks, n_local, hl, self.rb_in), dtype=torch.uint8, device=device)
-                self.qkv_records = torch.empty((total, hl, self.rb_in), dtype=torch.uint8, device=device)
-            else:
-                self.send = torch.empty((self.n_ranks, n_local, 3, hl, D), dtype=torch.bfloat16, device=device)
-            self.out_shard = torch.empty((total, hl, D), dtype=self.out_dtype, device=device)
-            if self.out_int8:
-                self.out_records = torch.empty((total, hl, self.rb_out), dtype=torch.uint8, device=device)
-                self.recv_out = torch.empty((self.n_ranks, n_local, hl, self.rb_out), dtype=torch.uint8, device=device)
-            else:
-                self.recv_out = torch.empty((self.n_ranks, n_local, hl, D), dtype=self.out_dtype, device=device)
+            n_groups = max(1, min(int(n_groups), hl))
+            bounds = [hl * j // n_groups for j in range(n_groups + 1)]
+            self.groups = [_HeadGroup(self, seqs, bounds[j], bounds[j + 1] - bounds[j], rope_dims, theta, device)
+                           for j in range(n_groups)]
+            self.s_in = torch.cuda.Stream(device=device)       # QKV pack + exchange (+ dequantisation)
+            self.s_out = torch.cuda.Stream(device=device)      # output exchange + merge (+ dequantisation)
         else:
             import torch.distributed._symmetric_memory as symm
+            qkv_strides = (3 * hl * D, D)
+            self.attn = B.Attn3d(seqs, hl, D, rope_dims, theta, device, q_strides=qkv_strides, k_strides=qkv_strides,
+                                 v_strides=qkv_strides)
             per = self.xp.ranges[0][1] - self.xp.ranges[0][0]          # largest shard: same size on every rank
             self.qkv = symm.empty((total, 3, hl, D), dtype=torch.bfloat16, device=device)
             self.merged = symm.empty((max(per, 1), heads, D), dtype=self.out_dtype, device=device)
@@ -131,37 +156,10 @@ class SequenceParallelAttn3d:
         xp = self.xp
         if tuple(q.shape) != (xp.n_local, self.heads, self.head_dim):
             raise ValueError(f"expected [{xp.n_local}, {self.heads}, {self.head_dim}] on rank {self.rank}")
-        qv, kv, vv = self.qkv[:, 0], self.qkv[:, 1], self.qkv[:, 2]
         if self.transport == "collective":
-            dsts = [self.send[g].data_ptr() for g in range(self.n_ranks)]
-            if self.qkv_int8:
-                B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, self.n_ranks, dsts, 0)
-                self.dist.all_to_all_single(self.qkv_records.view(-1), self.send.view(-1), xp.qkv_recv_splits,
-                                            xp.qkv_send_splits, group=self.group)
-                B.sol_attn3d_exchange_unpack_qkv_int8(self.qkv_records, self.qkv, xp.total, xp.hl, self.head_dim)
-            else:
-                B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, dsts, 0)
-                self.dist.all_to_all_single(self.qkv.view(-1), self.send.view(-1), xp.qkv_recv_splits, xp.qkv_send_splits,
-                                            group=self.group)
-            if self.fp8:
-                B.sol_attn3d_forward_e4m3(self.attn.plan, qv, kv, vv, self.out_shard, key_mask)
-            else:
-                B.sol_attn3d_forward(self.attn.plan, qv, kv, vv, self.out_shard, key_mask)
-            wire = self.out_shard
-            if self.out_int8:
-                B.sol_attn3d_exchange_quantize_out_int8(self.out_shard, self.out_records)
-                wire = self.out_records
-            self.dist.all_to_all_single(self.recv_out.view(-1), wire.view(-1), xp.out_recv_splits, xp.out_send_splits,
-                                        group=self.group)
-            out = torch.empty((xp.n_local, self.heads, self.head_dim), dtype=self.out_dtype, device=q.device)
-            if self.out_int8:
-                merged = torch.empty((xp.n_local, self.heads, self.rb_out), dtype=torch.uint8, device=q.device)
-                B.sol_attn3d_exchange_merge_heads(self.recv_out, merged, xp.n_local, self.heads, self.rb_out, self.n_ranks)
-                B.sol_attn3d_exchange_dequantize_out_int8(merged, out)
-            else:
-                B.sol_attn3d_exchange_merge_heads(self.recv_out, out, xp.n_local, self.heads, self.rb_out, self.n_ranks)
-            return out
+            return self._forward_collective(q, k, v, key_mask)
         # peer transport: stores into the owners' buffers, barriers instead of payload collectives
+        qv, kv, vv = self.qkv[:, 0], self.qkv[:, 1], self.qkv[:, 2]
         self._barrier()                                       # everyone is done reading last call's buffers
         B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, self.qkv_peers, xp.first_token)
         self._barrier()
@@ -170,5 +168,62 @@ class SequenceParallelAttn3d:
         self._barrier()
         return self.merged[:xp.n_local]
 
+    def _forward_collective(self, q, k, v, key_mask):
+        xp, D, G = self.xp, self.head_dim, self.n_ranks
+        cur = torch.cuda.current_stream()
+        out = torch.empty((xp.n_local, self.heads, D), dtype=self.out_dtype, device=q.device)
+        out.record_stream(self.s_out)
+        merged = None
+        if self.out_int8:
+            merged = torch.empty((xp.n_local, self.heads, self.rb_out), dtype=torch.uint8, device=q.device)
+            merged.record_stream(self.s_out)
+        # (1) every group's QKV exchange is queued up front on the input stream: pack -> all-to-all (-> dequantise)
+        self.s_in.wait_stream(cur)                            # q, k, v are ready; last call's readers are done
+        self.s_out.wait_stream(cur)
+        with torch.cuda.stream(self.s_in):
+            for gr in self.groups:
+                dsts = [gr.send[r].data_ptr() for r in range(G)]
+                if self.qkv_int8:
+                    B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, G, dsts, 0, group_begin=gr.begin, group_heads=gr.count)
+                    self.dist.all_to_all_single(gr.qkv_records.view(-1), gr.send.view(-1), gr.qkv_recv_splits,
+                                                gr.qkv_send_splits, group=self.group)
+                    B.sol_attn3d_exchange_unpack_qkv_int8(gr.qkv_records, gr.qkv, xp.total, gr.count, D)
+                else:
+                    B.sol_attn3d_exchange_pack_qkv(q, k, v, G, dsts, 0, group_begin=gr.begin, group_heads=gr.count)
+                    self.dist.all_to_all_single(gr.qkv.view(-1), gr.send.view(-1), gr.qkv_recv_splits, gr.qkv_send_splits,
+                                                group=self.group)
+                gr.ev_in.record(self.s_in)
+        # (2) attention group by group on the caller's stream; (3) each group's output returns on the output stream
+        for gr in self.groups:
+            cur.wait_event(gr.ev_in)
+            qv, kv, vv = gr.qkv[:, 0], gr.qkv[:, 1], gr.qkv[:, 2]
+            if self.fp8:
+                B.sol_attn3d_forward_e4m3(gr.attn.plan, qv, kv, vv, gr.out_shard, key_mask)
+            else:
+                B.sol_attn3d_forward(gr.attn.plan, qv, kv, vv, gr.out_shard, key_mask)
+            wire = gr.out_shard
+            if self.out_int8:
+                B.sol_attn3d_exchange_quantize_out_int8(gr.out_shard, gr.out_records)
+                wire = gr.out_records
+            gr.ev_out.record(cur)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(gr.ev_out)
+                self.dist.all_to_all_single(gr.recv_out.view(-1), wire.view(-1), gr.out_recv_splits, gr.out_send_splits,
+                                            group=self.group)
+                # the group's heads land in their place in the full rows: rank stride = the whole shard
+                target = merged if self.out_int8 else out
+                rec = self.rb_out
+                B.sol_attn3d_exchange_merge_heads(gr.recv_out, target.data_ptr() + gr.begin * rec, xp.n_local, G * gr.count, rec, G,
+                                                  self.heads * rec, out_rank_stride_bytes=xp.hl * rec)
+        with torch.cuda.stream(self.s_out):
+            if self.out_int8:
+                B.sol_attn3d_exchange_dequantize_out_int8(merged, out)
+        cur.wait_stream(self.s_out)
+        return out
+
     def close(self):
-        self.attn.close()
+        if self.transport == "collective":
+            for gr in self.groups:
+                gr.attn.close()
+        else:
+            self.attn.close()

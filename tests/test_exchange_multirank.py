@@ -39,6 +39,15 @@ def _worker(rank, world, port, total, heads, D, out_dir):
         want = (full[0] + 2 * full[1] - full[2])[a:b]
         assert torch.equal(merged, want), f"rank {rank}: returned rows"
         assert xp.tok_begin[rank] == a and xp.tok_begin[-1] == total
+        # one head group of every shard (here: the last head of each): same routing with the group's split sizes
+        if hl > 1:
+            gs, gr, _, _ = xp.splits(1)
+            sel = torch.tensor([r * hl + hl - 1 for r in range(world)])
+            send_g = xo.pack_qkv_reference(full[0][a:b][:, sel], full[1][a:b][:, sel], full[2][a:b][:, sel], world)
+            recv_g = torch.empty((total, 3, 1, D), dtype=torch.int32)
+            dist.all_to_all_single(recv_g.view(-1), send_g.contiguous().view(-1), gr, gs)
+            for w in range(3):
+                assert torch.equal(recv_g[:, w, 0], full[w][:, rank * hl + hl - 1])
         open(os.path.join(out_dir, f"ok{rank}"), "w").write("ok")
     finally:
         dist.destroy_process_group()

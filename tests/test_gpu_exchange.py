@@ -148,6 +148,39 @@ def test_merge_heads_is_the_reference_permutation(B, G, n_local, heads, record):
     assert torch.equal(dense.cpu(), want)
 
 
+@pytest.mark.parametrize("G,heads,begin,count", [(2, 8, 1, 2), (4, 40, 7, 3), (1, 6, 0, 6), (8, 16, 1, 1)])
+def test_head_groups_pack_and_merge_in_place(B, G, heads, begin, count):
+    """A head group [begin, begin+count) of every rank's shard: the pack sends exactly those heads, the INT8 pack the
+    same records, and the merge drops the group into its place in the full output row."""
+    n_local, D = 53, 128
+    g = torch.Generator(device="cuda").manual_seed(500 + G)
+    q, k, v = (torch.randn((n_local, heads, D), generator=g, device="cuda").to(torch.bfloat16) for _ in range(3))
+    hl = heads // G
+    sel = torch.cat([torch.arange(r * hl + begin, r * hl + begin + count) for r in range(G)])
+    send = torch.empty((G, n_local, 3, count, D), dtype=torch.bfloat16, device="cuda")
+    B.sol_attn3d_exchange_pack_qkv(q, k, v, G, [send[r].data_ptr() for r in range(G)], 0, group_begin=begin, group_heads=count)
+    torch.cuda.synchronize()
+    want = xo.pack_qkv_reference(q.cpu()[:, sel], k.cpu()[:, sel], v.cpu()[:, sel], G)
+    assert torch.equal(send.cpu().view(torch.int16), want.view(torch.int16))
+    rb = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)
+    send8 = torch.empty((G, n_local, count, rb), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, G, [send8[r].data_ptr() for r in range(G)], 0, group_begin=begin, group_heads=count)
+    torch.cuda.synchronize()
+    rec = xo.qkv_records(q.cpu()[:, sel], k.cpu()[:, sel], v.cpu()[:, sel])
+    for r in range(G):
+        assert torch.equal(send8[r].cpu(), rec[:, r * count:(r + 1) * count])
+    # merge: what the ranks return for this group lands at heads r*hl + begin .. of the full rows; the rest stays
+    record = 2 * D
+    recv = torch.randint(0, 256, (G, n_local, count, record), generator=g, device="cuda", dtype=torch.uint8)
+    full = torch.full((n_local, heads, record), 0xAB, dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_merge_heads(recv, full.data_ptr() + begin * record, n_local, G * count, record, G, heads * record,
+                                      out_rank_stride_bytes=hl * record)
+    torch.cuda.synchronize()
+    exp = torch.full((n_local, heads, record), 0xAB, dtype=torch.uint8)
+    exp[:, sel] = xo.merge_heads_reference(recv.cpu())
+    assert torch.equal(full.cpu(), exp)
+
+
 def test_exchange_entry_points_reject_bad_arguments(B):
     x = torch.zeros((4, 6, 64), dtype=torch.bfloat16, device="cuda")
     dst = torch.zeros(4 * 3 * 6 * 64, dtype=torch.bfloat16, device="cuda")
@@ -279,7 +312,7 @@ def test_sequence_parallel_module_with_one_rank(B):
         dist.init_process_group("nccl", rank=0, world_size=1)
         created = True
     try:
-        w = wl.shrunk("cfg_batch")
+        w = replace(wl.shrunk("cfg_batch"), heads=4)
         inp = wl.make_inputs(w, "cuda")
         single = B.Attn3d.from_workload(w, "cuda")
         want = single.forward(inp.q, inp.k, inp.v, inp.key_mask)
@@ -311,6 +344,15 @@ def test_sequence_parallel_module_with_one_rank(B):
         assert torch.equal(gotq, wantq)
         rel = float(torch.linalg.vector_norm(gotq.double() - want.double()) / torch.linalg.vector_norm(want.double()))
         assert rel < 3e-2, rel
+        # head groups with the exchanges on side streams: same bytes as one group, for every wire format
+        for kw, ref_out in (({}, got), ({"out_format": "e4m3"}, got8), ({"out_format": "int8", "qkv_wire": "int8"}, gotq)):
+            for n_groups in (2, 4):
+                spg = SequenceParallelAttn3d(seq_tuples(w), w.heads, w.head_dim, w.rope_dims, w.theta, n_groups=n_groups, **kw)
+                for _ in range(2):
+                    gg = spg.forward(inp.q, inp.k, inp.v, inp.key_mask)
+                    torch.cuda.synchronize()
+                    assert torch.equal(gg, ref_out), (kw, n_groups)
+                spg.close()
         sp.close(); sp8.close(); spq.close(); a2.close(); single.close()
     finally:
         if created:
