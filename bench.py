@@ -411,7 +411,7 @@ def main():
         e_ms = ev0.elapsed_time(ev1) / e_steps
         h2d = 3 * inp.q.numel() * 2 + (0 if hmask is None else hmask.numel())
         e2e = {"ms": e_ms, "h2d": h2d, "d2h": out.numel() * 2, "steps": e_steps}
-        e2e["api"] = "sol_attn3d_forward_host (8 head groups, copies overlapped)" if plain else "copies + forward + copy on one stream"
+        e2e["api"] = "sol_attn3d_forward_host (head groups, copies overlapped)" if plain else "copies + forward + copy on one stream"
         if plain:
             torch.cuda.synchronize()
             e2e["max_abs_vs_device_forward"] = float((hout.to(dev).float() - out.float()).abs().max())

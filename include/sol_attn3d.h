@@ -308,7 +308,8 @@ int sol_attn3d_forward_scatter(sol_attn3d_plan_t plan, const void* q, const void
  *                  the default strides); key_mask_host HOST uint8 [total_tokens] or NULL.
  *   staging        DEVICE memory, 256-byte aligned, >= sol_attn3d_host_staging_bytes(plan) (four tensors and the
  *                  mask), caller-owned, must stay untouched until `stream` has passed this call.
- *   n_groups       1 .. 8; 0 = default (8); clamped to the number of heads.
+ *   n_groups       1 .. 8 equal groups (clamped to the number of heads); 0 = default: six groups of growing and then
+ *                  shrinking size (a small first group, whose inputs are exposed, and a small last one, whose outputs are).
  * The first call creates two streams and a few events (no device memory); sol_attn3d_destroy releases them.
  * Result: bit-identical to sol_attn3d_forward on device copies of the same tensors.
  * Errors: INVALID_ARG, NO_WORKSPACE (plan workspace or staging), UNSUPPORTED_SHAPE (strided plan), CUDA.

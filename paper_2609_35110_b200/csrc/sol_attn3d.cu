@@ -1092,8 +1092,20 @@ int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void*
   const long long dense_tok = (long long)p->heads * p->head_dim;
   for (const Strides* s : {&p->sq, &p->sk, &p->sv, &p->so})
     if (s->tok != dense_tok || s->head != p->head_dim) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;   // dense tensors only
-  if (n_groups <= 0) n_groups = 8;
-  n_groups = std::min(std::min(n_groups, 8), p->heads);
+  // head-group boundaries: equal groups when the caller names a count; by default a ramp (small first group:
+  // its host-to-device copy is exposed; small last group: its device-to-host copy is) with larger groups between
+  int bounds[9];
+  if (n_groups <= 0 && p->heads >= 12) {
+    static const int kRamp[7] = {0, 1, 4, 9, 14, 18, 20};       // cumulative weights 1, 3, 5, 5, 4, 2 (of 20)
+    n_groups = 6;
+    for (int g = 0; g <= 6; ++g) bounds[g] = (int)(((long long)p->heads * kRamp[g] + 10) / 20);
+    for (int g = 1; g <= 6; ++g) bounds[g] = std::max(bounds[g], bounds[g - 1] + 1);
+    bounds[6] = p->heads;
+  } else {
+    if (n_groups <= 0) n_groups = 8;
+    n_groups = std::min(std::min(n_groups, 8), p->heads);
+    for (int g = 0; g <= n_groups; ++g) bounds[g] = (int)((long long)p->heads * g / n_groups);
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
   if (!p->host_pipe_ready) {
@@ -1132,7 +1144,7 @@ int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void*
   p->prof = false;                                   // per-kernel events describe one launch set, not a pipeline
   int rc = SOL_ATTN3D_OK;
   for (int g = 0; g < n_groups && rc == SOL_ATTN3D_OK; ++g) {
-    const int h0 = (int)((long long)p->heads * g / n_groups), h1 = (int)((long long)p->heads * (g + 1) / n_groups);
+    const int h0 = bounds[g], h1 = bounds[g + 1];
     const size_t off = (size_t)h0 * p->head_dim * 2, width = (size_t)(h1 - h0) * p->head_dim * 2;
     // K and V first: the rotary producer and the attention of this group need all three
     const void* srcs[3] = {k_host, v_host, q_host};
