@@ -303,10 +303,13 @@ def sol_attn3d_forward_scatter(plan, q, k, v, key_mask, dst: Sequence[int], tok_
 
 
 def _strides_of(t: torch.Tensor, head_dim: int):
-    if t.dim() != 3 or t.stride(2) != 1 or t.shape[2] != head_dim:
+    """(token, head) element strides of a [tokens, heads, head_dim] tensor whose head_dim axis is contiguous."""
+    if t.dim() != 3 or t.shape[2] != head_dim or t.stride(2) != 1:
         raise ValueError("expected [tokens, heads, head_dim] with contiguous head_dim")
-    tok = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1] * head_dim)
-    return (ctypes.c_int64 * 2)(tok, t.stride(1) if t.shape[1] > 1 else head_dim)
+    # the stride torch reports for an axis of extent 0 or 1 is arbitrary: use the dense value there
+    tok = t.stride(0) if t.shape[0] > 1 else t.shape[1] * head_dim
+    head = t.stride(1) if t.shape[1] > 1 else head_dim
+    return (ctypes.c_int64 * 2)(tok, head)
 
 
 def sol_attn3d_exchange_pack_qkv(q, k, v, n_ranks: int, dst: Sequence[int], dst_row0: int = 0, stream=None,
