@@ -32,11 +32,12 @@ from paper_2609_35110_b200 import workloads as wl  # noqa: E402
 METRIC = "attention_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16 = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from the ncu summaries under
-# profiles/ (attn_fwd_kernel_lowres_ncu_full.md, bench_highres_launch_list.md).
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from the one-pass ncu captures
+# summarised under profiles/ (attn_fwd_kernel_dram_traffic.md).
 NCU_TRAFFIC = {
-    "lowres": (1020140288, "ncu capture of this workload"),
-    "highres": (int(1020140288 * 111856 / 25216), "scaled from the lowres capture by tokens x heads"),
+    "lowres": (779200000 + 236650000, "ncu capture of this workload (one pass, two DRAM counters)"),
+    "highres": (8160000000 + 1140000000, "ncu capture of this workload (one pass, two DRAM counters); K/V re-reads "
+                                         "that miss L2, see profiles/attn_fwd_kernel_dram_traffic.md"),
 }
 
 

@@ -149,6 +149,7 @@ __device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq
     }
   }
   __syncwarp();
+  const uint64_t pol_once = l2_policy_evict_first();            // output rows are written once, never read here
   const int ch = lane % kLanesPerRow;
 #pragma unroll 4
   for (int r0 = 0; r0 < 32; r0 += 32 / kLanesPerRow) {
@@ -157,7 +158,7 @@ __device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq
     bool store = qrow < sq.n_tokens;
     if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
     const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * kRowBytes + ((ch ^ (rr & (kLanesPerRow - 1))) << 4));
-    if (store) *reinterpret_cast<uint4*>(out_row_ptr(p, sq.tok_start + qrow, head, kFp8 ? 1 : 2) + ch * 16) = w;
+    if (store) st_global_evict_first(out_row_ptr(p, sq.tok_start + qrow, head, kFp8 ? 1 : 2) + ch * 16, w, pol_once);
   }
 }
 
@@ -361,13 +362,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // =========================================================== TMA producer
     if (lane == 0) {
       bool ok = true;
+      // Q tiles are read once: first to go from L2, so that they do not push out the head's K / V, which every
+      // CTA of the head streams (an evict-last hint on K / V was measured too: more DRAM reads, not fewer, because
+      // the previous heads' tiles then linger)
+      const uint64_t pol_once = l2_policy_evict_first();
       mbar_arrive_expect_tx(bar_q_full, 2 * L::kTile);
 #pragma unroll
       for (int t = 0; t < 2; ++t)
 #pragma unroll
         for (int hf = 0; hf < L::kHalves; ++hf)
-          tma_load_3d(sQ + t * L::kTile + hf * L::kHalfBytes, &tm_q, bar_q_full, hf * 64, head,
-                      tok0 + q_row0 + t * 128);
+          tma_load_3d_hint(sQ + t * L::kTile + hf * L::kHalfBytes, &tm_q, bar_q_full, hf * 64, head,
+                           tok0 + q_row0 + t * 128, pol_once);
       uint32_t it = 0, stage = 0, par = 0;
       for (int i = 0; i < n_proc && ok; ++i) {
         const int jt = __ldg(&ktiles[i]);
@@ -378,8 +383,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const CUtensorMap* tm = kv ? &tm_v : &tm_k;
 #pragma unroll
           for (int hf = 0; hf < L::kHalves; ++hf)
-            tma_load_3d(sKV + stage * L::kTile + hf * L::kHalfBytes, tm, bar_kv_full(stage), hf * 64, head,
-                        tok0 + jt * 128);
+            tma_load_3d(sKV + stage * L::kTile + hf * L::kHalfBytes, tm, bar_kv_full(stage), hf * 64, head, tok0 + jt * 128);
           ++it;
           if (++stage == (uint32_t)L::kStages) { stage = 0; par ^= 1u; }
         }
