@@ -36,7 +36,7 @@ NOMINAL_BF16 = 2250.0
 # summarised under profiles/ (attn_fwd_kernel_dram_traffic.md).
 NCU_TRAFFIC = {
     "lowres": (779200000 + 236650000, "ncu capture of this workload (one pass, two DRAM counters)"),
-    "highres": (8160000000 + 1140000000, "ncu capture of this workload (one pass, two DRAM counters); K/V re-reads "
+    "highres": (5650000000 + 1140000000, "ncu capture of this workload (one pass, two DRAM counters); K/V re-reads "
                                          "that miss L2, see profiles/attn_fwd_kernel_dram_traffic.md"),
 }
 

@@ -225,6 +225,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int* __restrict__ ktiles =
       sparse ? p.cta_list + sq.sparse_list_start + (long long)local * sq.n_ktiles : p.ktile_list + sq.ktile_start;
   const uint4* __restrict__ keybits = p.keybits + sq.ktile_start;
+  // Successive waves of CTAs walk the key tiles in opposite directions (the softmax does not care about the
+  // order): a wave then starts on the tiles its predecessor touched last, which are still in L2, instead of
+  // on the ones it touched first, which a long sequence has pushed out by then.
+  const bool backwards = ((cta / p.wave_ctas) & 1) != 0;
   const int q_row0 = pair * 256;                       // first local query row of the CTA
   const int tok0 = (int)sq.tok_start;                  // TMA token coordinate of the sequence start
   const unsigned long long limit = p.wait_limit_ns;
@@ -270,7 +274,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     bool ok = true;
 
     for (int i = 0; i < n_proc; ++i) {
-      const int jt = __ldg(&ktiles[i]);
+      const int jt = __ldg(&ktiles[backwards ? n_proc - 1 - i : i]);
       const uint4 kb = __ldg(&keybits[jt]);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full(t), i & 1, limit));
       if (!ok) break;
@@ -375,7 +379,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                            tok0 + q_row0 + t * 128, pol_once);
       uint32_t it = 0, stage = 0, par = 0;
       for (int i = 0; i < n_proc && ok; ++i) {
-        const int jt = __ldg(&ktiles[i]);
+        const int jt = __ldg(&ktiles[backwards ? n_proc - 1 - i : i]);
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
           if (!mbar_wait(bar_kv_empty(stage), par ^ 1u, limit)) { ok = false; break; }

@@ -46,6 +46,7 @@ struct AttnParams {
   int heads;
   int head_begin, head_end; // this launch serves heads [head_begin, head_end) (all heads: 0, heads)
   int cta_offset;           // work item of CTA 0 of this launch (a head range of one sequence is a contiguous range)
+  int wave_ctas;            // CTAs that run at the same time (one per SM): the key direction alternates per wave
   const uint4* keybits;     // [ktile] 128 validity bits (bit b of word w = key 32*w + b of the tile)
   const int* ktile_list;    // per sequence, tiles that hold at least one valid key, ascending
   const int* ktile_count;   // per sequence (schedule order)

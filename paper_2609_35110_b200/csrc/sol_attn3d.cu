@@ -70,6 +70,7 @@ struct sol_attn3d_plan_s {
   cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
   cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[8] = {}, ev_out[8] = {};
   bool host_pipe_ready = false;
+  int sm_count = 148;                 // of the device the workspace was bound on
 };
 
 namespace {
@@ -364,6 +365,8 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t p, void* device_ptr, size_t bytes
   int major = 0;
   if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess) return fail_cuda(p, e);
   if (major != 10) return SOL_ATTN3D_ERR_UNSUPPORTED_ARCH;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) p->sm_count = sms;
 
   if (p->encode == nullptr) {
     void* fn = nullptr;
@@ -854,6 +857,7 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.fault_inject = p->fault_inject;
   ap.head_begin = head_begin;
   ap.head_end = head_end;
+  ap.wave_ctas = p->sm_count;
   // one sequence: the CTAs of a head range are a contiguous range of work items; several sequences: launch
   // everything and let the CTAs of other heads leave at the door
   int grid = p->total_work;
@@ -1055,6 +1059,7 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
   ap.head_begin = 0;
   ap.head_end = p->heads;
   ap.cta_offset = 0;
+  ap.wave_ctas = p->sm_count;
   ap.o_tok_stride = p->so.tok;
   ap.o_head_stride = p->so.head;
   ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));

@@ -257,7 +257,8 @@ def test_exchange_returns_the_single_device_attention(B, name, heads, G, peer_st
     single.close()
     merged = virtual_ranks_forward(B, w, inp, G, B.OUT_BF16, peer_style)
     got = torch.cat(merged, dim=0)
-    # heads are independent and a CTA's arithmetic does not depend on the grid around it: bit-identical
+    # heads are independent and, at these sizes (one wave of CTAs), a CTA's arithmetic does not depend on the grid
+    # around it: bit-identical
     assert torch.equal(got.view(torch.int16), want.view(torch.int16))
     max_abs, rel_l2 = orc.compare(got.cpu(), oracle_dense(w, inp))
     assert max_abs <= TOL_MAX_ABS and rel_l2 <= TOL_REL_L2, (max_abs, rel_l2)
@@ -501,7 +502,7 @@ def test_full_size_lowres_e4m3_and_scatter_sampled_rows(B):
     assert not bool((out8 == 0x7F).any()), "an output byte was never written"
     attn.close()
     qc, kc, vc = inp.q.cpu(), inp.k.cpu(), inp.v.cpu()
-    select = [(0, h, torch.from_numpy(wl.sample_rows(w, 0, h, 1024))) for h in (0, w.heads - 1)]
+    select = [(0, h, torch.from_numpy(wl.sample_rows(w, 0, h, 1024))) for h in (0, 15, w.heads - 1)]
     refs = orc.attn3d_oracle(qc, kc, vc, seq_tuples(w), w.rope_dims, w.theta, None, select=select)
     for (_, h, rows), ref in zip(select, refs):
         idx = rows.cuda()
@@ -520,6 +521,14 @@ def test_full_size_lowres_e4m3_and_scatter_sampled_rows(B):
     assert shard.status() == 0
     shard.close()
     got = torch.cat(owners, dim=0)
-    assert torch.equal(got[:, r * hl:(r + 1) * hl].view(torch.int16), out16[:, r * hl:(r + 1) * hl].view(torch.int16))
+    # A 10-head plan puts the same (head, query block) in another wave of CTAs than the 40-head plan, and the order
+    # in which a CTA walks the key tiles alternates per wave: same sums in another order, equal to rounding.
+    a, b = got[:, r * hl:(r + 1) * hl].float(), out16[:, r * hl:(r + 1) * hl].float()
+    assert float((a - b).abs().max()) <= 2.0 ** -7 * float(b.abs().max())
+    assert float((a == b).float().mean()) > 0.4           # CTAs that walk in the same direction in both plans agree bit for bit
+    for (_, h, rows), ref in zip(select, refs):
+        if r * hl <= h < (r + 1) * hl:
+            max_abs, rel_l2 = orc.compare(got[rows.cuda(), h].cpu(), ref)
+            assert max_abs <= TOL_MAX_ABS and rel_l2 <= TOL_REL_L2
     assert bool(torch.isnan(got[:, :r * hl].float()).all()) and bool(torch.isnan(got[:, (r + 1) * hl:].float()).all()), \
         "the scatter epilogue wrote outside its head columns"
