@@ -35,7 +35,7 @@ NOMINAL_BF16 = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from the one-pass ncu captures
 # summarised under profiles/ (attn_fwd_kernel_dram_traffic.md).
 NCU_TRAFFIC = {
-    "lowres": (779200000 + 236650000, "ncu capture of this workload (one pass, two DRAM counters)"),
+    "lowres": (787700000 + 238820000, "ncu capture of this workload (one pass, two DRAM counters)"),
     "highres": (5650000000 + 1140000000, "ncu capture of this workload (one pass, two DRAM counters); K/V re-reads "
                                          "that miss L2, see profiles/attn_fwd_kernel_dram_traffic.md"),
 }
