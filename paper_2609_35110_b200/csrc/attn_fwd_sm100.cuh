@@ -162,6 +162,18 @@ __device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq
   }
 }
 
+// Half of softmax_pass: 64 columns -> 32 packed pairs, partial sums kept in acc.
+__device__ __forceinline__ void softmax_half(const uint32_t (&r)[64], float c, float mc, uint32_t (&pk)[32], float (&acc)[4]) {
+#pragma unroll
+  for (int cc = 0; cc < 32; ++cc) {
+    const float p_lo = ex2_approx(fmaf(__uint_as_float(r[2 * cc]), c, -mc));
+    const float p_hi = ex2_approx(fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc));
+    acc[(2 * cc) & 3] += p_lo;
+    acc[(2 * cc + 1) & 3] += p_hi;
+    pk[cc] = pack_bf16x2(p_lo, p_hi);
+  }
+}
+
 template <int D>
 struct AttnSmem {
   static constexpr int kTile = 128 * D * 2;               // bytes of one 128 x D bf16 tile
@@ -280,32 +292,51 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (!ok) break;
       tc_fence_after();
 
-      uint32_t r[128];
-#pragma unroll
-      for (int cch = 0; cch < 4; ++cch) tmem_ld32(tS + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[cch * 32]));
-      tmem_wait_ld();
-
-
       const bool mixed = (kb.x & kb.y & kb.z & kb.w) != 0xffffffffu;
-      if (mixed) {
-        // masked or out-of-range keys get -inf
+      uint32_t r[128];
+      uint32_t pk[64];
+      float tile_sum;
+      bool first_half_stored = false;
+      if (!mixed && i > 0) {
+        // Common case, in two halves: the second half of S is still on its way while the first is exponentiated, and
+        // the first half of P is on its way to tensor memory while the second is.
+        uint32_t (&r_lo)[64] = *reinterpret_cast<uint32_t(*)[64]>(&r[0]);
+        uint32_t (&r_hi)[64] = *reinterpret_cast<uint32_t(*)[64]>(&r[64]);
+        tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+        tmem_wait_ld_dep64(r_lo);
+        tmem_ld32(tS + 64, *reinterpret_cast<uint32_t(*)[32]>(&r[64]));
+        tmem_ld32(tS + 96, *reinterpret_cast<uint32_t(*)[32]>(&r[96]));
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const float mc = m_ref * c;
+        softmax_half(r_lo, c, mc, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]), acc);
+        tmem_wait_ld_dep64(r_hi);
+        tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));       // columns [0,32): their scores are in registers
+        first_half_stored = true;
+        softmax_half(r_hi, c, mc, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]), acc);
+        tile_sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+      } else {
 #pragma unroll
-        for (int cc = 0; cc < 128; ++cc) {
-          const uint32_t w = cc < 32 ? kb.x : cc < 64 ? kb.y : cc < 96 ? kb.z : kb.w;
-          if (((w >> (cc & 31)) & 1u) == 0) r[cc] = __float_as_uint(-CUDART_INF_F);
+        for (int cch = 0; cch < 4; ++cch) tmem_ld32(tS + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[cch * 32]));
+        tmem_wait_ld();
+        if (mixed) {
+          // masked or out-of-range keys get -inf
+#pragma unroll
+          for (int cc = 0; cc < 128; ++cc) {
+            const uint32_t w = cc < 32 ? kb.x : cc < 64 ? kb.y : cc < 96 ? kb.z : kb.w;
+            if (((w >> (cc & 31)) & 1u) == 0) r[cc] = __float_as_uint(-CUDART_INF_F);
+          }
         }
+        if (i == 0) m_ref = row_max128(r);
+        if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
+        else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum);
       }
-      if (i == 0) m_ref = row_max128(r);
-      // Speculative pass: exponentials against the current reference maximum, no row maximum taken.
+      // The pass ran against the current reference maximum, no row maximum taken.
       // All terms are positive, so a row sum <= 2^8 proves that every term is <= 2^8: the reference
       // is still good enough (the result does not depend on which reference is used, only overflow
       // does).  Only when the sum is larger (or not finite) is the row maximum computed; if it has grown
       // by more than 2^8 in the exp2 domain the reference moves, l and O are rescaled and the tile is
       // redone from the scores still held in registers, before any of its P is released.  Rare.
-      uint32_t pk[64];
-      float tile_sum;
-      if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
-      else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum);
       if (__any_sync(0xffffffffu, !(tile_sum <= 256.0f))) {
         const float mx = row_max128(r);
         const bool grow = (mx - m_ref) * c > 8.0f;
@@ -326,10 +357,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tmem_st32(tO + cch * 32, o);
           }
           softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
+          if (first_half_stored) tmem_wait_st();                         // the stale first half lands before its replacement
+          first_half_stored = false;
         }
       }
       l += tile_sum;
-      tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      if (!first_half_stored) tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
       tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
