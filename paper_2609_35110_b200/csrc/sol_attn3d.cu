@@ -813,9 +813,9 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
     unsigned long long* stats = reinterpret_cast<unsigned long long*>(sparse_ws + p->sp_off_stats);
     for (int s = 0; s < p->n_seqs; ++s) {
       const SeqDev& sq = p->sched[(size_t)s];
-      sol::pool_blocks_kernel<<<sq.n_qpairs * p->heads, p->head_dim, 0, st>>>(q_rot, d_seqs, p->heads, p->head_dim, 256, s,
+      sol::pool_blocks_kernel<<<sq.n_qpairs * p->heads, 256, 0, st>>>(q_rot, d_seqs, p->heads, p->head_dim, 256, s,
                                                                              sq.n_qpairs, 0, qbar + p->sp_qbar_seq[(size_t)s]);
-      sol::pool_blocks_kernel<<<sq.n_ktiles * p->heads, p->head_dim, 0, st>>>(k_rot, d_seqs, p->heads, p->head_dim, 128, s,
+      sol::pool_blocks_kernel<<<sq.n_ktiles * p->heads, 256, 0, st>>>(k_rot, d_seqs, p->heads, p->head_dim, 128, s,
                                                                              sq.n_ktiles, 1, kbar + p->sp_kbar_seq[(size_t)s]);
       const size_t smem = (size_t)sol::kSelectRows * ((size_t)p->head_dim + (size_t)sq.n_ktiles) * sizeof(float);
       if (smem > 48 * 1024) return SOL_ATTN3D_ERR_UNSUPPORTED_SHAPE;      // > ~1400 key tiles (180k tokens) per sequence

@@ -13,26 +13,49 @@ namespace sol {
 
 // ---------------------------------------------------------------------------------------------
 // Mean of the rotated operand over a block of tokens, per head (fp32).
-// x: rotated bf16 [token][head][D] contiguous.  One CTA per (sequence, head, block); thread d sums
-// column d over the block's tokens in order.  blockDim = D.
+// x: rotated bf16 [token][head][D] contiguous.  One CTA of 256 threads per (sequence, head, block): D/8 lanes
+// cover a token row with 16-byte loads, the other 256 / (D/8) lanes take every 16th (32nd) token; partial sums
+// meet in shared memory and are added in a fixed order.
 // Output layout: out[head][block][d], or transposed out[head][d][block] (so that the selection kernel
 // reads the pooled keys with consecutive threads on consecutive blocks).
 // ---------------------------------------------------------------------------------------------
-__global__ void pool_blocks_kernel(const __nv_bfloat16* __restrict__ x, const SeqDev* __restrict__ seqs, int heads,
-                                   int head_dim, int block_tokens, int seq_index, int n_blocks, int transposed,
-                                   float* __restrict__ out) {
+__global__ void __launch_bounds__(256) pool_blocks_kernel(const __nv_bfloat16* __restrict__ x,
+                                                          const SeqDev* __restrict__ seqs, int heads, int head_dim,
+                                                          int block_tokens, int seq_index, int n_blocks, int transposed,
+                                                          float* __restrict__ out) {
+  __shared__ float part[32][129];                  // [token lane][d], padded against bank conflicts
   const SeqDev sq = seqs[seq_index];
   const int blk = blockIdx.x % n_blocks;
   const int head = blockIdx.x / n_blocks;
-  const int d = threadIdx.x;
+  const int chunks = head_dim >> 3;
+  const int tlanes = blockDim.x / chunks;           // 16 for D = 128, 32 for D = 64
+  const int c = threadIdx.x % chunks, tl = threadIdx.x / chunks;
   const int t0 = blk * block_tokens;
   const int t1 = min(sq.n_tokens, t0 + block_tokens);
-  const __nv_bfloat16* src = x + ((sq.tok_start + t0) * heads + head) * (long long)head_dim + d;
-  float acc = 0.f;
-  for (int t = t0; t < t1; ++t, src += (long long)heads * head_dim) acc += __bfloat162float(*src);
-  const float mean = acc / (float)(t1 - t0);
-  if (transposed) out[((long long)head * head_dim + d) * n_blocks + blk] = mean;
-  else            out[((long long)head * n_blocks + blk) * head_dim + d] = mean;
+  const long long row = (long long)heads * head_dim;
+  const __nv_bfloat16* src = x + ((sq.tok_start + t0 + tl) * heads + head) * (long long)head_dim + c * 8;
+  float acc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+  for (int t = t0 + tl; t < t1; t += tlanes, src += row * tlanes) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      acc[2 * u] += __uint_as_float(w[u] << 16);
+      acc[2 * u + 1] += __uint_as_float(w[u] & 0xffff0000u);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) part[tl][c * 8 + e] = acc[e];
+  __syncthreads();
+  for (int d = threadIdx.x; d < head_dim; d += blockDim.x) {
+    float sum = 0.f;
+    for (int j = 0; j < tlanes; ++j) sum += part[j][d];
+    const float mean = sum / (float)(t1 - t0);
+    if (transposed) out[((long long)head * head_dim + d) * n_blocks + blk] = mean;
+    else            out[((long long)head * n_blocks + blk) * head_dim + d] = mean;
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
