@@ -126,6 +126,9 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t plan, void* device_ptr, size_t by
  *   K and V values at masked positions must be finite (0 * inf inside the tensor core is NaN).
  * The call only enqueues kernels (no allocation, no synchronisation, no host-device copy), so it may be
  * stream-captured into a CUDA graph and replayed (profiling off).
+ * Results are deterministic: the same plan on the same inputs gives the same bits, whichever entry point or head
+ * range is used.  Plans that differ in their number of heads walk the key tiles of a (head, query block) in
+ * possibly different order at sizes beyond one wave of CTAs, so their results agree to rounding, not to the bit.
  * Errors: INVALID_ARG (NULL / misaligned pointer), NO_WORKSPACE, CUDA.  Device-side time-outs are
  * reported by sol_attn3d_status after the caller has synchronised the stream.
  */
