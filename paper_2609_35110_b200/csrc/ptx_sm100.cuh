@@ -97,7 +97,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_
 #endif
 }
 
-// The same for a whole converged warp: every lane polls, the verdict is made uniform.
+// The same for a whole converged warp: every lane polls, the outcome is made uniform.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, limit_ns));
 }
