@@ -32,12 +32,12 @@ from paper_2609_35110_b200 import workloads as wl  # noqa: E402
 METRIC = "attention_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16 = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from the one-pass ncu captures
-# summarised under profiles/ (attn_fwd_kernel_dram_traffic.md).
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from one-pass ncu captures of these
+# very workloads (two DRAM counters, one launch).
 NCU_TRAFFIC = {
     "lowres": (787700000 + 238820000, "ncu capture of this workload (one pass, two DRAM counters)"),
-    "highres": (5650000000 + 1140000000, "ncu capture of this workload (one pass, two DRAM counters); K/V re-reads "
-                                         "that miss L2, see profiles/attn_fwd_kernel_dram_traffic.md"),
+    "highres": (5650000000 + 1140000000, "ncu capture of this workload (one pass, two DRAM counters); the excess over the "
+                                         "algorithmic bytes is K/V re-reads that miss L2 between waves of CTAs"),
 }
 
 
