@@ -377,9 +377,12 @@ int sol_attn3d_sparse_selection(sol_attn3d_plan_t plan, const void* sparse_ws, i
  * The function calls no cudaMalloc, cudaFree or other allocating routine, neither directly nor through
  * a library.  The first call on each device looks up the device address of the built-in array
  * (cudaGetSymbolAddress), raises the kernels' shared-memory limit and resolves one driver entry
- * point; do that first call with the device current and before any stream capture begins.  Later
- * calls only enqueue work: a 4-byte memset, two small host-to-device copies of the plan's tables, and
- * three kernels.  Nothing synchronises.
+ * point; do that first call with the device current and before any stream capture begins.  If the CUDA
+ * runtime loads modules lazily, that first call is also where the driver places the library's code and
+ * the 32 MiB array on the device; later calls find device memory unchanged.  Later calls only enqueue
+ * work: a 4-byte memset, two small host-to-device copies of the plan's tables (a few KB to a few hundred
+ * KB, read from ordinary pageable host memory owned by the plan), and three kernels.  Keep the plan alive
+ * until `stream` has passed the call.
  *
  * All calls on a device share the one array and it keeps the previous call's contents.  Everything a
  * call reads from it is rewritten by that call first (the status word is cleared, tables are copied
@@ -417,8 +420,24 @@ int sol_attn3d_status(sol_attn3d_plan_t plan);
 int sol_attn3d_set_profiling(sol_attn3d_plan_t plan, int enable);
 int sol_attn3d_last_forward_ms(sol_attn3d_plan_t plan, float ms[3]);
 
-/* Number of kernels one sol_attn3d_forward with / without a key mask enqueues (for launch accounting). */
-int sol_attn3d_launches_per_forward(sol_attn3d_plan_t plan, int with_mask);
+/*
+ * Number of kernels the most recent forward-type call on this plan enqueued (any sol_attn3d_forward* entry point,
+ * sol_attn3d_rope_qk, sol_attn3d_qknorm_rope), counted as they were launched: the dense forward launches 2 (rotary
+ * prologue, attention) plus 1 when the key-validity bits are rebuilt; the block-sparse forward adds 3 per sequence,
+ * the rectangular one 1, and sol_attn3d_forward_host launches one such set per head group.  Host-side counter, no
+ * device access.  For launch accounting in benchmarks (Section 3.2 counts launches around "SDPA").
+ */
+int sol_attn3d_last_launch_count(sol_attn3d_plan_t plan);
+
+/*
+ * Diagnostic for the online softmax (the running-maximum form of the softmax in Section 3.2's "SDPA"; the paper does
+ * not describe it): the attention kernel exponentiates each 128-key tile against a reference maximum per query
+ * row and moves that reference only when a tile's row maximum exceeds it by more than 2^8 (then the partial
+ * output and row sum are rescaled).  *count receives how often that happened, in (warp of 32 query rows, key
+ * tile) events, since the workspace was bound (sol_attn3d_set_workspace resets it).  Synchronous 4-byte copy;
+ * call after synchronising the stream.  Tests use it to prove that inputs built to move the maximum did so.
+ */
+int sol_attn3d_softmax_rescale_count(sol_attn3d_plan_t plan, unsigned long long* count);
 
 /* cudaError_t of the last failing CUDA call made on behalf of this plan (0 if none). */
 int sol_attn3d_last_cuda_error(sol_attn3d_plan_t plan);

@@ -255,11 +255,12 @@ def rope_oracle(x, seqs: Sequence[Tuple[int, int, int, int]], rope_dims: Sequenc
 # ---------------------------------------------------------------------------------------------
 # Block-sparse variant: the per-step dynamic sparsity of Section 3.4 ("Sparse Attention").
 # This is an approximation of dense attention, so the oracle follows the algorithm step by step.
-# Steps and notation (the paper gives the rule, not the block statistic; readings are marked):
-#   B1  query blocks of QBLK = 256 tokens, KV blocks of KBLK = 128 tokens, per sequence and head  [reading]
+# Steps and notation (the paper gives the rule, not the block statistic nor the block sizes; readings are
+# marked).  Nothing is rounded anywhere: the statistic is taken in fp64 on the un-rounded rotated operands.
+#   B1  query blocks of qblk tokens, KV blocks of kblk tokens, per sequence and head; both sizes are arguments
+#       of every function below                                                                    [reading]
 #   B2  block-level score  b_ij = < mean of q~ over block i , mean of k~ over block j > / sqrt(D)    [reading:
-#       mean-pooled, pre-softmax logits; q~, k~ are the rotated operands AS THE KERNEL SEES THEM, i.e.
-#       rounded to bf16, so that both sides take the selection decision on the same numbers]
+#       mean-pooled pre-softmax logits; by bilinearity this is the mean of the block's logits]
 #   B3  per query block: mu_i, sigma_i = mean and (population) standard deviation of b_ij over all KV
 #       blocks j; KV block j is selected iff b_ij > mu_i + tau * sigma_i                      [Section 3.4]
 #   B4  safety rails [Section 3.4]: KV blocks holding any prefix token are always selected (exact prefix
@@ -267,68 +268,87 @@ def rope_oracle(x, seqs: Sequence[Tuple[int, int, int, int]], rope_dims: Sequenc
 #       is always kept, so no query block is left without keys.                                [last: reading]
 #   B5  attention as O4-O5 restricted to the keys of the selected blocks (and to valid keys).
 # ---------------------------------------------------------------------------------------------
-QBLK = 256
-KBLK = 128
-
-
-def block_scores(q_rot: torch.Tensor, k_rot: torch.Tensor, head_dim: int) -> torch.Tensor:
-    """B2 for one (sequence, head): q_rot, k_rot [N, D] fp64 -> [ceil(N/256), ceil(N/128)]."""
+def block_scores(q_rot: torch.Tensor, k_rot: torch.Tensor, head_dim: int, qblk: int, kblk: int) -> torch.Tensor:
+    """B2 for one (sequence, head): q_rot, k_rot [N, D] fp64 -> [ceil(N/qblk), ceil(N/kblk)]."""
     n = q_rot.shape[0]
-    nq, nk = (n + QBLK - 1) // QBLK, (n + KBLK - 1) // KBLK
-    qbar = torch.stack([q_rot[i * QBLK: min(n, (i + 1) * QBLK)].mean(0) for i in range(nq)])
-    kbar = torch.stack([k_rot[j * KBLK: min(n, (j + 1) * KBLK)].mean(0) for j in range(nk)])
+    nq, nk = (n + qblk - 1) // qblk, (n + kblk - 1) // kblk
+    qbar = torch.stack([q_rot[i * qblk: min(n, (i + 1) * qblk)].mean(0) for i in range(nq)])
+    kbar = torch.stack([k_rot[j * kblk: min(n, (j + 1) * kblk)].mean(0) for j in range(nk)])
     return (qbar @ kbar.t()) / math.sqrt(head_dim)
 
 
-def block_select(scores: torch.Tensor, tau: float, text_len: int) -> torch.Tensor:
+def block_select(scores: torch.Tensor, tau: float, text_len: int, qblk: int, kblk: int) -> torch.Tensor:
     """B3-B4: bool [n_qblocks, n_kblocks], True = KV block attended."""
     mu = scores.mean(dim=1, keepdim=True)
     sigma = torch.sqrt(((scores - mu) ** 2).mean(dim=1, keepdim=True))
     sel = scores > mu + tau * sigma
     sel[torch.arange(scores.shape[0]), scores.argmax(dim=1)] = True
     if text_len > 0:
-        sel[:, : (text_len + KBLK - 1) // KBLK] = True           # exact prefix KV sink
-        sel[: (text_len + QBLK - 1) // QBLK, :] = True           # prefix queries stay dense
+        sel[:, : (text_len + kblk - 1) // kblk] = True           # exact prefix KV sink
+        sel[: (text_len + qblk - 1) // qblk, :] = True           # prefix queries stay dense
     return sel
 
 
+def sparse_rows(q_rot: torch.Tensor, k_rot: torch.Tensor, v: torch.Tensor, sel: torch.Tensor,
+                valid: Optional[torch.Tensor], rows: torch.Tensor, head_dim: int, qblk: int, kblk: int) -> torch.Tensor:
+    """B5 for one (sequence, head) and the given local query rows: q_rot, k_rot [N, D], v [N, Dv] fp64,
+    sel bool [n_qblocks, n_kblocks] -> fp64 [len(rows), Dv].  Rows of one query block share their key set."""
+    n = k_rot.shape[0]
+    rows = torch.as_tensor(rows, dtype=torch.int64)
+    out = torch.zeros(rows.shape[0], v.shape[1], dtype=F64)
+    blk = rows // qblk
+    for i in torch.unique(blk).tolist():
+        keys = sel[i].repeat_interleave(kblk)[:n]
+        if valid is not None:
+            keys = keys & valid
+        here = blk == i
+        out[here] = attention_rows(q_rot[rows[here]], k_rot, v, keys, head_dim)
+    return out
+
+
 def attn3d_sparse_oracle(q, k, v, seqs: Sequence[Tuple[int, int, int, int]], rope_dims: Sequence[int],
-                         theta: float, tau: float, key_mask: Optional[torch.Tensor] = None,
-                         selection: Optional[List[List[torch.Tensor]]] = None,
-                         operand_dtype: torch.dtype = torch.bfloat16):
-    """Block-sparse attention, all rows.  Returns (out fp64 [total, heads, D], selection, scores) where
-    selection[s][h] is the bool block mask used and scores[s][h] the block scores (None when a selection
-    was supplied).  ``selection`` overrides B2-B4 (used to check the attention arithmetic on a given
-    choice of blocks).  ``operand_dtype`` is the rounding applied to q~, k~ before the block statistic.
+                         theta: float, tau: float, qblk: int, kblk: int, key_mask: Optional[torch.Tensor] = None,
+                         selection=None, select: Optional[List[Tuple[int, int, torch.Tensor]]] = None):
+    """Block-sparse attention.  Returns (out, selection, scores).
+
+    With ``select`` = None every row is computed: out is fp64 [total, heads, D], selection[s][h] the bool block
+    mask used and scores[s][h] the block scores (None where a selection was supplied).  With ``select`` = a list
+    of (seq, head, local rows) only those rows are computed: out, selection and scores are lists in that order
+    (this is how full-size cases are sampled).  ``selection`` overrides B2-B4 (to check the attention
+    arithmetic on a given choice of blocks): indexed [s][h] in the first form, a list parallel to ``select`` in
+    the second.
     """
     cu, pos, has = layout_positions(seqs)
     total, heads, D = q.shape
-    out = torch.zeros(total, heads, v.shape[2], dtype=F64)
-    used, scs = [], []
-    for s, (L, T, H, W) in enumerate(seqs):
+    dense = select is None
+    if dense:
+        select = [(s, h, None) for s in range(len(seqs)) for h in range(heads)]
+        out_dense = torch.zeros(total, heads, v.shape[2], dtype=F64)
+        used = [[None] * heads for _ in seqs]
+        scs = [[None] * heads for _ in seqs]
+    outs, used_l, scs_l = [], [], []
+    for idx, (s, h, rows) in enumerate(select):
         a, b = cu[s], cu[s + 1]
         n = b - a
-        used.append([])
-        scs.append([])
+        L = seqs[s][0]
         valid = None if key_mask is None else (key_mask[a:b].to("cpu") != 0)
-        for h in range(heads):
-            q_rot = rope_rotate(widen(q[a:b, h]), pos[a:b], has[a:b], rope_dims, theta)
-            k_rot = rope_rotate(widen(k[a:b, h]), pos[a:b], has[a:b], rope_dims, theta)
-            if selection is None:
-                sc = block_scores(q_rot.to(operand_dtype).to(F64), k_rot.to(operand_dtype).to(F64), D)
-                sel = block_select(sc, tau, L)
-            else:
-                sc, sel = None, selection[s][h]
-            used[-1].append(sel)
-            scs[-1].append(sc)
-            vh = widen(v[a:b, h])
-            for i in range(sel.shape[0]):
-                keys = sel[i].repeat_interleave(KBLK)[:n]
-                if valid is not None:
-                    keys = keys & valid
-                r0, r1 = i * QBLK, min(n, (i + 1) * QBLK)
-                out[a + r0: a + r1, h] = attention_rows(q_rot[r0:r1], k_rot, vh, keys, D)
-    return out, used, scs
+        q_rot = rope_rotate(widen(q[a:b, h]), pos[a:b], has[a:b], rope_dims, theta)
+        k_rot = rope_rotate(widen(k[a:b, h]), pos[a:b], has[a:b], rope_dims, theta)
+        if selection is None:
+            sc = block_scores(q_rot, k_rot, D, qblk, kblk)
+            sel = block_select(sc, tau, L, qblk, kblk)
+        else:
+            sc, sel = None, (selection[s][h] if dense else selection[idx])
+        rows_t = torch.arange(n, dtype=torch.int64) if rows is None else torch.as_tensor(rows, dtype=torch.int64)
+        o = sparse_rows(q_rot, k_rot, widen(v[a:b, h]), sel, valid, rows_t, D, qblk, kblk)
+        if dense:
+            out_dense[a:b, h] = o
+            used[s][h], scs[s][h] = sel, sc
+        else:
+            outs.append(o)
+            used_l.append(sel)
+            scs_l.append(sc)
+    return (out_dense, used, scs) if dense else (outs, used_l, scs_l)
 
 
 def compare(gpu_rows: torch.Tensor, ref_rows: torch.Tensor) -> Tuple[float, float]:

@@ -127,8 +127,10 @@ def _lib():
     lib.sol_attn3d_set_profiling.restype = i32
     lib.sol_attn3d_last_forward_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.sol_attn3d_last_forward_ms.restype = i32
-    lib.sol_attn3d_launches_per_forward.argtypes = [vp, i32]
-    lib.sol_attn3d_launches_per_forward.restype = i32
+    lib.sol_attn3d_last_launch_count.argtypes = [vp]
+    lib.sol_attn3d_last_launch_count.restype = i32
+    lib.sol_attn3d_softmax_rescale_count.argtypes = [vp, ctypes.POINTER(ctypes.c_ulonglong)]
+    lib.sol_attn3d_softmax_rescale_count.restype = i32
     lib.sol_attn3d_last_cuda_error.argtypes = [vp]
     lib.sol_attn3d_last_cuda_error.restype = i32
     lib.sol_attn3d_strerror.argtypes = [i32]
@@ -461,8 +463,14 @@ def sol_attn3d_last_forward_ms(plan) -> Tuple[float, float, float]:
     return float(ms[0]), float(ms[1]), float(ms[2])
 
 
-def sol_attn3d_launches_per_forward(plan, with_mask: bool) -> int:
-    return int(_lib().sol_attn3d_launches_per_forward(plan, 1 if with_mask else 0))
+def sol_attn3d_last_launch_count(plan) -> int:
+    return int(_lib().sol_attn3d_last_launch_count(plan))
+
+
+def sol_attn3d_softmax_rescale_count(plan) -> int:
+    n = ctypes.c_ulonglong()
+    _check(_lib().sol_attn3d_softmax_rescale_count(plan, ctypes.byref(n)), "sol_attn3d_softmax_rescale_count")
+    return int(n.value)
 
 
 def sol_attn3d_last_cuda_error(plan) -> int:

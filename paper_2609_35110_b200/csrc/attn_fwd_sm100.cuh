@@ -45,6 +45,11 @@ constexpr int kAttnThreads = 384;   // 8 softmax warps + producer + MMA issuer +
 #ifndef SOL_EMU_CNT
 #define SOL_EMU_CNT 0
 #endif
+// P hand-over to the MMA issuer: 1 = one arrival per softmax warp (lane 0, after the warp has synchronised)
+// instead of one per thread.
+#ifndef SOL_PFULL_PER_WARP
+#define SOL_PFULL_PER_WARP 0
+#endif
 
 __device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
   float m0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
@@ -162,12 +167,21 @@ __device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq
   }
 }
 
-// Half of softmax_pass: 64 columns -> 32 packed pairs, partial sums kept in acc.
+// Half of softmax_pass: 64 columns -> 32 packed pairs, partial sums kept in acc.  Only called for tiles without
+// masked keys, so the share of exponentials that goes to the FMA pipes (see exp2_emulated) applies here too.
 __device__ __forceinline__ void softmax_half(const uint32_t (&r)[64], float c, float mc, uint32_t (&pk)[32], float (&acc)[4]) {
 #pragma unroll
   for (int cc = 0; cc < 32; ++cc) {
-    const float p_lo = ex2_approx(fmaf(__uint_as_float(r[2 * cc]), c, -mc));
-    const float p_hi = ex2_approx(fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc));
+    const float x_lo = fmaf(__uint_as_float(r[2 * cc]), c, -mc);
+    const float x_hi = fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc);
+    float p_lo, p_hi;
+    if ((cc % SOL_EMU_MOD) < SOL_EMU_CNT) {
+      p_lo = exp2_emulated(x_lo);
+      p_hi = exp2_emulated(x_hi);
+    } else {
+      p_lo = ex2_approx(x_lo);
+      p_hi = ex2_approx(x_hi);
+    }
     acc[(2 * cc) & 3] += p_lo;
     acc[(2 * cc + 1) & 3] += p_hi;
     pk[cc] = pack_bf16x2(p_lo, p_hi);
@@ -253,7 +267,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(bar_s_full(t), 1);
-      mbar_init(bar_p_full(t), 128);
+      mbar_init(bar_p_full(t), SOL_PFULL_PER_WARP ? 4 : 128);
       mbar_init(bar_o_done(t), 1);
     }
     mbar_init(bar_drain, 1);
@@ -341,6 +355,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const float mx = row_max128(r);
         const bool grow = (mx - m_ref) * c > 8.0f;
         if (__any_sync(0xffffffffu, grow)) {
+          if (lane == 0) atomicAdd(p.counters, 1u);                      // rare path: counted for the tests
           const float f = grow ? ex2_approx((m_ref - mx) * c) : 1.0f;
           if (grow) m_ref = mx;
           l *= f;
@@ -366,7 +381,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
+#if SOL_PFULL_PER_WARP
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p_full(t));
+#else
       mbar_arrive(bar_p_full(t));
+#endif
     }
 
     // ---- epilogue: O / l in the output format, staged through shared memory, coalesced 16-byte stores

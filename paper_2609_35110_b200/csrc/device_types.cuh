@@ -58,6 +58,7 @@ struct AttnParams {
   long long o_tok_stride, o_head_stride;  // in elements
   float scale_log2;         // log2(e) / sqrt(head_dim)
   unsigned int* status;     // 0 = fine; written once on a wait time-out
+  unsigned int* counters;   // [0]: (warp, key tile) events in which the softmax moved its reference maximum
   unsigned long long wait_limit_ns;
   unsigned int fault_inject;  // test hook: 1 = CTA 0 never publishes S of query tile 1 (exercises the bounded waits)
   unsigned int v_lbo, v_sbo;  // byte offsets of the V (MN-major) shared-memory descriptor

@@ -22,6 +22,7 @@ namespace {
 using sol::SeqDev;
 
 constexpr size_t kAlign = 256;
+constexpr size_t kCountersOffset = 64;   // diagnostic counters inside the 256-byte status block of a workspace
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 struct Strides {
@@ -71,6 +72,7 @@ struct sol_attn3d_plan_s {
   cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[8] = {}, ev_out[8] = {};
   bool host_pipe_ready = false;
   int sm_count = 148;                 // of the device the workspace was bound on
+  int launches = 0;                   // kernels enqueued by the most recent forward-type call
 };
 
 namespace {
@@ -261,14 +263,14 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
 }
 
 // [tokens][heads][D] bf16 tensor as a 3-D TMA map with 128 x 64-element boxes, 128-byte swizzle.
-int encode_map(sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides st) {
+int encode_map(EncodeTiledFn fn, sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides st) {
   const cuuint64_t dims[3] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->heads, (cuuint64_t)p->total_tokens};
   const cuuint64_t strides[2] = {(cuuint64_t)st.head * 2, (cuuint64_t)st.tok * 2};
   const cuuint32_t box[3] = {64, 1, 128};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = p->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     p->last_cuda = (int)r;
     return SOL_ATTN3D_ERR_CUDA;
@@ -278,8 +280,9 @@ int encode_map(sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides s
 
 bool aligned16(const void* x) { return (reinterpret_cast<uintptr_t>(x) & 15u) == 0; }
 
-int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, void* kr, const float* q_gain,
-                const float* k_gain, float eps, cudaStream_t st, int head_begin = 0, int head_end = 0) {
+int launch_rope(sol_attn3d_plan_t p, const unsigned char* ws, const void* q, const void* k, void* qr, void* kr,
+                const float* q_gain, const float* k_gain, float eps, cudaStream_t st, int head_begin = 0,
+                int head_end = 0) {
   sol::RopeArgs a{};
   a.gain[0] = q_gain;
   a.gain[1] = k_gain;
@@ -290,10 +293,10 @@ int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, voi
   a.y[1] = static_cast<__nv_bfloat16*>(kr);
   a.x_tok_stride[0] = p->sq.tok; a.x_head_stride[0] = p->sq.head;
   a.x_tok_stride[1] = p->sk.tok; a.x_head_stride[1] = p->sk.head;
-  a.seqs = reinterpret_cast<const SeqDev*>(p->ws + p->off_seqs);
+  a.seqs = reinterpret_cast<const SeqDev*>(ws + p->off_seqs);
   a.n_seqs = p->n_seqs;
   a.total_tokens = p->total_tokens;
-  a.tables = reinterpret_cast<const float2*>(p->ws + p->off_tables);
+  a.tables = reinterpret_cast<const float2*>(ws + p->off_tables);
   for (int i = 0; i < 3; ++i) { a.g.rope[i] = p->rope[i]; a.g.tab_off[i] = p->tab_off[i]; }
   a.g.head_dim = p->head_dim;
   a.g.heads = p->heads;
@@ -305,7 +308,9 @@ int launch_rope(sol_attn3d_plan_t p, const void* q, const void* k, void* qr, voi
   const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
   sol::rope_qk_kernel<<<(unsigned)blocks, threads, 0, st>>>(a);
   const cudaError_t e = cudaGetLastError();
-  return e == cudaSuccess ? SOL_ATTN3D_OK : fail_cuda(p, e);
+  if (e != cudaSuccess) return fail_cuda(p, e);
+  ++p->launches;
+  return SOL_ATTN3D_OK;
 }
 
 }  // namespace
@@ -372,7 +377,8 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t p, void* device_ptr, size_t bytes
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) return fail_cuda(p, e);
+    if (e != cudaSuccess) return fail_cuda(p, e);
+    if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return SOL_ATTN3D_ERR_CUDA;   // driver too old for TMA
     p->encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
   if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -393,8 +399,8 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t p, void* device_ptr, size_t bytes
                       cudaMemcpyHostToDevice)) != cudaSuccess)
     return fail_cuda(p, e);
   const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
-  int rc = encode_map(p, &p->tm_q, p->ws + p->off_qrot, dense);
-  if (rc == SOL_ATTN3D_OK) rc = encode_map(p, &p->tm_k, p->ws + p->off_krot, dense);
+  int rc = encode_map(p->encode, p, &p->tm_q, p->ws + p->off_qrot, dense);
+  if (rc == SOL_ATTN3D_OK) rc = encode_map(p->encode, p, &p->tm_k, p->ws + p->off_krot, dense);
   return rc;
 }
 
@@ -405,7 +411,8 @@ int sol_attn3d_rope_qk(sol_attn3d_plan_t p, const void* q, const void* k, void* 
   if ((q == nullptr) != (q_rot == nullptr) || (k == nullptr) != (k_rot == nullptr)) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (q == nullptr && k == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(q_rot) || !aligned16(k_rot)) return SOL_ATTN3D_ERR_INVALID_ARG;
-  return launch_rope(p, q, k, q_rot, k_rot, nullptr, nullptr, 0.f, static_cast<cudaStream_t>(stream));
+  p->launches = 0;
+  return launch_rope(p, p->ws, q, k, q_rot, k_rot, nullptr, nullptr, 0.f, static_cast<cudaStream_t>(stream));
 }
 
 namespace {
@@ -424,6 +431,13 @@ struct FwdOpts {
   int dst_heads = 0, head_offset = 0;
   int head_begin = 0, head_end = 0;   // serve heads [head_begin, head_end) only (0, 0 = all)
   bool skip_keybits = false;          // the key-validity bits of this mask were built by an earlier call
+  bool keep_launch_count = false;     // one of several launch sets of the same API call: keep counting
+  // Scratch other than the plan's bound workspace (sol_attn3d_forward_noalloc): the caller of forward_impl has put
+  // the tables and the sequence table there; nothing about it is cached in the plan.
+  unsigned char* ws = nullptr;
+  unsigned int* status = nullptr;     // status word to use instead of the one inside the scratch
+  EncodeTiledFn encode = nullptr;     // tensor-map encoder for such a call
+  int sm_count = 0;                   // SMs of the current device for such a call (the plan may never have been bound)
 };
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
                  sol_attn3d_stream_t stream, const FwdOpts& o);
@@ -716,7 +730,8 @@ int sol_attn3d_qknorm_rope(sol_attn3d_plan_t p, const void* q, const void* k, co
   if ((q != nullptr && q_gain == nullptr) || (k != nullptr && k_gain == nullptr) || !(eps >= 0.f))
     return SOL_ATTN3D_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(q_out) || !aligned16(k_out)) return SOL_ATTN3D_ERR_INVALID_ARG;
-  return launch_rope(p, q, k, q_out, k_out, q_gain, k_gain, eps, static_cast<cudaStream_t>(stream));
+  p->launches = 0;
+  return launch_rope(p, p->ws, q, k, q_out, k_out, q_gain, k_gain, eps, static_cast<cudaStream_t>(stream));
 }
 
 namespace {
@@ -759,14 +774,20 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   unsigned char* sparse_ws = o.sparse_ws;
   const float tau = o.tau;
   const uint8_t* query_mask = o.query_mask;
-  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  // the plan's bound workspace (tables uploaded, tensor maps of Q~ / K~ cached), or scratch handed in for this call
+  const bool own = o.ws == nullptr;
+  unsigned char* ws = own ? p->ws : o.ws;
+  if (ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  const EncodeTiledFn encode = own ? p->encode : o.encode;
+  if (encode == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
+  if (!o.keep_launch_count) p->launches = 0;
 
-  const SeqDev* d_seqs = reinterpret_cast<const SeqDev*>(p->ws + p->off_seqs);
-  uint32_t* d_bits = reinterpret_cast<uint32_t*>(p->ws + p->off_keybits);
-  int* d_list = reinterpret_cast<int*>(p->ws + p->off_list);
-  int* d_count = reinterpret_cast<int*>(p->ws + p->off_count);
+  const SeqDev* d_seqs = reinterpret_cast<const SeqDev*>(ws + p->off_seqs);
+  uint32_t* d_bits = reinterpret_cast<uint32_t*>(ws + p->off_keybits);
+  int* d_list = reinterpret_cast<int*>(ws + p->off_list);
+  int* d_count = reinterpret_cast<int*>(ws + p->off_count);
 
   const int head_begin = o.head_begin, head_end = o.head_end > 0 ? o.head_end : p->heads;
   if (head_begin < 0 || head_end > p->heads || head_begin >= head_end) return SOL_ATTN3D_ERR_INVALID_ARG;
@@ -774,28 +795,31 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
     p->prof_valid = false;
     if ((e = cudaEventRecord(p->ev[0], st)) != cudaSuccess) return fail_cuda(p, e);
   }
-  // (1) validity bits per key tile: rebuilt whenever a mask is given (its contents may have changed)
+  // (1) validity bits per key tile: rebuilt whenever a mask is given (its contents may have changed) and whenever
+  //     the scratch is not the plan's own (nothing is known about what it holds)
   p->prof_bits = false;
-  if (!o.skip_keybits && (key_mask != nullptr || p->keybits_state != 1)) {
+  if (!o.skip_keybits && (!own || key_mask != nullptr || p->keybits_state != 1)) {
     p->prof_bits = true;
     sol::keybits_kernel<<<p->n_seqs, 256, 0, st>>>(d_seqs, key_mask, d_bits, d_list, d_count);
     if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
-    p->keybits_state = key_mask ? 2 : 1;
+    ++p->launches;
+    if (own) p->keybits_state = key_mask ? 2 : 1;
   }
 
   if (p->prof && (e = cudaEventRecord(p->ev[1], st)) != cudaSuccess) return fail_cuda(p, e);
 
   // (2) rotary prologue: Q~, K~ into the workspace
-  int rc = launch_rope(p, q, k, p->ws + p->off_qrot, p->ws + p->off_krot, q_gain, k_gain, eps, st, head_begin, head_end);
+  int rc = launch_rope(p, ws, q, k, ws + p->off_qrot, ws + p->off_krot, q_gain, k_gain, eps, st, head_begin, head_end);
   if (rc != SOL_ATTN3D_OK) return rc;
   if (p->prof && (e = cudaEventRecord(p->ev[2], st)) != cudaSuccess) return fail_cuda(p, e);
 
   // (2a) rectangular mode: which query pairs hold a wanted row
   const uint8_t* d_pair_needed = nullptr;
   if (query_mask != nullptr) {
-    uint8_t* flags = p->ws + p->off_pairs;
+    uint8_t* flags = ws + p->off_pairs;
     sol::pair_needed_kernel<<<p->total_pairs, 32, 0, st>>>(d_seqs, p->n_seqs, query_mask, flags);
     if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+    ++p->launches;
     d_pair_needed = flags;
   }
 
@@ -804,8 +828,8 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   const int* d_cta_count = nullptr;
   if (sparse_ws != nullptr) {
     if ((e = cudaMemsetAsync(sparse_ws + p->sp_off_stats, 0, 256, st)) != cudaSuccess) return fail_cuda(p, e);
-    const __nv_bfloat16* q_rot = reinterpret_cast<const __nv_bfloat16*>(p->ws + p->off_qrot);
-    const __nv_bfloat16* k_rot = reinterpret_cast<const __nv_bfloat16*>(p->ws + p->off_krot);
+    const __nv_bfloat16* q_rot = reinterpret_cast<const __nv_bfloat16*>(ws + p->off_qrot);
+    const __nv_bfloat16* k_rot = reinterpret_cast<const __nv_bfloat16*>(ws + p->off_krot);
     float* qbar = reinterpret_cast<float*>(sparse_ws + p->sp_off_qbar);
     float* kbar = reinterpret_cast<float*>(sparse_ws + p->sp_off_kbar);
     int* lists = reinterpret_cast<int*>(sparse_ws + p->sp_off_list);
@@ -824,16 +848,27 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
           d_seqs, s, p->heads, p->head_dim, tau, qbar + p->sp_qbar_seq[(size_t)s], kbar + p->sp_kbar_seq[(size_t)s],
           reinterpret_cast<const uint4*>(d_bits), lists, counts, stats);
       if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+      p->launches += 3;
     }
     d_cta_list = lists;
     d_cta_count = counts;
   }
 
-  // (3) attention
-  if (p->v_cached != v) {
-    rc = encode_map(p, &p->tm_v, v, p->sv);
-    if (rc != SOL_ATTN3D_OK) return rc;
-    p->v_cached = v;
+  // (3) attention.  Tensor maps: the plan's cached ones for its own workspace, per-call ones otherwise.
+  CUtensorMap tm_q_call, tm_k_call, tm_v_call;
+  const CUtensorMap *tm_q = &p->tm_q, *tm_k = &p->tm_k, *tm_v = &p->tm_v;
+  if (own) {
+    if (p->v_cached != v) {
+      rc = encode_map(encode, p, &p->tm_v, v, p->sv);
+      if (rc != SOL_ATTN3D_OK) return rc;
+      p->v_cached = v;
+    }
+  } else {
+    const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
+    if ((rc = encode_map(encode, p, &tm_q_call, ws + p->off_qrot, dense)) != SOL_ATTN3D_OK) return rc;
+    if ((rc = encode_map(encode, p, &tm_k_call, ws + p->off_krot, dense)) != SOL_ATTN3D_OK) return rc;
+    if ((rc = encode_map(encode, p, &tm_v_call, v, p->sv)) != SOL_ATTN3D_OK) return rc;
+    tm_q = &tm_q_call; tm_k = &tm_k_call; tm_v = &tm_v_call;
   }
   sol::AttnParams ap{};
   ap.seqs = d_seqs;
@@ -850,14 +885,15 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.o_tok_stride = o_tok_stride;
   ap.o_head_stride = o_head_stride;
   ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));
-  ap.status = reinterpret_cast<unsigned int*>(p->ws + p->off_status);
+  ap.status = o.status != nullptr ? o.status : reinterpret_cast<unsigned int*>(ws + p->off_status);
+  ap.counters = reinterpret_cast<unsigned int*>(ws + p->off_status + kCountersOffset);
   ap.wait_limit_ns = p->wait_limit_ns;
   ap.v_lbo = p->v_lbo;
   ap.v_sbo = p->v_sbo;
-  ap.fault_inject = p->fault_inject;
+  ap.fault_inject = own ? p->fault_inject : 0u;
   ap.head_begin = head_begin;
   ap.head_end = head_end;
-  ap.wave_ctas = p->sm_count;
+  ap.wave_ctas = o.sm_count > 0 ? o.sm_count : p->sm_count;
   // one sequence: the CTAs of a head range are a contiguous range of work items; several sequences: launch
   // everything and let the CTAs of other heads leave at the door
   int grid = p->total_work;
@@ -867,11 +903,12 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
     grid = (head_end - head_begin) * p->sched[0].n_qpairs;
   }
   if (p->head_dim == 128) {
-    sol::attn_fwd_kernel<128><<<grid, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(p->tm_q, p->tm_k, p->tm_v, ap);
+    sol::attn_fwd_kernel<128><<<grid, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
   } else {
-    sol::attn_fwd_kernel<64><<<grid, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(p->tm_q, p->tm_k, p->tm_v, ap);
+    sol::attn_fwd_kernel<64><<<grid, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+  ++p->launches;
   if (p->prof) {
     if ((e = cudaEventRecord(p->ev[3], st)) != cudaSuccess) return fail_cuda(p, e);
     p->prof_valid = true;
@@ -927,9 +964,10 @@ constexpr int kMaxDevices = 64;
 // Device address of the array per device.  The array's name is only a host-side handle in host code;
 // the address a kernel can use comes from cudaGetSymbolAddress, asked once per device.
 unsigned char* g_static_scratch_addr[kMaxDevices] = {};
+int g_static_sm_count[kMaxDevices] = {};
 EncodeTiledFn g_static_encode = nullptr;
 
-int static_scratch_for_current_device(sol_attn3d_plan_t p, unsigned char** out) {
+int static_scratch_for_current_device(sol_attn3d_plan_t p, unsigned char** out, int* sm_count) {
   int dev = 0, n_dev = 0;
   cudaError_t e = cudaGetDeviceCount(&n_dev);
   if (e != cudaSuccess || n_dev == 0) {
@@ -943,6 +981,8 @@ int static_scratch_for_current_device(sol_attn3d_plan_t p, unsigned char** out) 
     if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
       return fail_cuda(p, e);
     if (major != 10) return SOL_ATTN3D_ERR_UNSUPPORTED_ARCH;
+    int sms = 0;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return fail_cuda(p, e);
     unsigned char* addr = nullptr;
     if ((e = cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), sol_attn3d_static_scratch)) != cudaSuccess)
       return fail_cuda(p, e);
@@ -957,40 +997,28 @@ int static_scratch_for_current_device(sol_attn3d_plan_t p, unsigned char** out) 
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
       e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-      if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) return fail_cuda(p, e);
+      if (e != cudaSuccess) return fail_cuda(p, e);
+      if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return SOL_ATTN3D_ERR_CUDA;   // driver too old for TMA
       g_static_encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
+    g_static_sm_count[dev] = sms;
     g_static_scratch_addr[dev] = addr;
   }
+  *sm_count = g_static_sm_count[dev];
   *out = g_static_scratch_addr[dev];
   return SOL_ATTN3D_OK;
 }
 
-int encode_map_with(EncodeTiledFn fn, sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides st) {
-  const cuuint64_t dims[3] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->heads, (cuuint64_t)p->total_tokens};
-  const cuuint64_t strides[2] = {(cuuint64_t)st.head * 2, (cuuint64_t)st.tok * 2};
-  const cuuint32_t box[3] = {64, 1, 128};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    p->last_cuda = (int)r;
-    return SOL_ATTN3D_ERR_CUDA;
-  }
-  return SOL_ATTN3D_OK;
-}
 }  // namespace
 
 int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out,
                                const uint8_t* key_mask, unsigned int* device_status, sol_attn3d_stream_t stream) {
   if (p == nullptr || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
-  if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(device_status) & 3u) != 0) return SOL_ATTN3D_ERR_INVALID_ARG;
   if (p->ws_bytes > kStaticScratchBytes) return SOL_ATTN3D_ERR_SCRATCH_LIMIT;
   unsigned char* ws = nullptr;
-  int rc = static_scratch_for_current_device(p, &ws);
+  int sm_count = 0;
+  const int rc = static_scratch_for_current_device(p, &ws, &sm_count);
   if (rc != SOL_ATTN3D_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
@@ -1006,77 +1034,13 @@ int sol_attn3d_forward_noalloc(sol_attn3d_plan_t p, const void* q, const void* k
   if ((e = cudaMemcpyAsync(ws + p->off_seqs, p->sched.data(), p->sched.size() * sizeof(SeqDev),
                            cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return fail_cuda(p, e);
-
-  const SeqDev* d_seqs = reinterpret_cast<const SeqDev*>(ws + p->off_seqs);
-  uint32_t* d_bits = reinterpret_cast<uint32_t*>(ws + p->off_keybits);
-  int* d_list = reinterpret_cast<int*>(ws + p->off_list);
-  int* d_count = reinterpret_cast<int*>(ws + p->off_count);
-  sol::keybits_kernel<<<p->n_seqs, 256, 0, st>>>(d_seqs, key_mask, d_bits, d_list, d_count);
-  if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
-
-  {
-    sol::RopeArgs a{};
-    a.x[0] = static_cast<const __nv_bfloat16*>(q);
-    a.x[1] = static_cast<const __nv_bfloat16*>(k);
-    a.y[0] = reinterpret_cast<__nv_bfloat16*>(ws + p->off_qrot);
-    a.y[1] = reinterpret_cast<__nv_bfloat16*>(ws + p->off_krot);
-    a.x_tok_stride[0] = p->sq.tok; a.x_head_stride[0] = p->sq.head;
-    a.x_tok_stride[1] = p->sk.tok; a.x_head_stride[1] = p->sk.head;
-    a.seqs = d_seqs;
-    a.n_seqs = p->n_seqs;
-    a.total_tokens = p->total_tokens;
-    a.tables = reinterpret_cast<const float2*>(ws + p->off_tables);
-    for (int i = 0; i < 3; ++i) { a.g.rope[i] = p->rope[i]; a.g.tab_off[i] = p->tab_off[i]; }
-    a.g.head_dim = p->head_dim;
-    a.g.heads = p->heads;
-    a.head_begin = 0;
-    a.head_end = p->heads;
-    const int chunks = p->head_dim / 8;
-    const int hpp = std::max(1, std::min(p->heads, 256 / chunks));
-    const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
-    sol::rope_qk_kernel<<<(unsigned)blocks, chunks * hpp, 0, st>>>(a);
-    if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
-  }
-
-  CUtensorMap tm_q, tm_k, tm_v;
-  const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
-  if ((rc = encode_map_with(g_static_encode, p, &tm_q, ws + p->off_qrot, dense)) != SOL_ATTN3D_OK) return rc;
-  if ((rc = encode_map_with(g_static_encode, p, &tm_k, ws + p->off_krot, dense)) != SOL_ATTN3D_OK) return rc;
-  if ((rc = encode_map_with(g_static_encode, p, &tm_v, v, p->sv)) != SOL_ATTN3D_OK) return rc;
-
-  sol::AttnParams ap{};
-  ap.seqs = d_seqs;
-  ap.n_seqs = p->n_seqs;
-  ap.heads = p->heads;
-  ap.keybits = reinterpret_cast<const uint4*>(d_bits);
-  ap.ktile_list = d_list;
-  ap.ktile_count = d_count;
-  ap.sink.base[0] = out;
-  ap.sink.tok_begin[0] = 0;
-  ap.sink.tok_begin[1] = p->total_tokens;
-  ap.sink.n_dst = 1;
-  ap.sink.fmt = sol::kOutBf16;
-  ap.head_begin = 0;
-  ap.head_end = p->heads;
-  ap.cta_offset = 0;
-  ap.wave_ctas = p->sm_count;
-  ap.o_tok_stride = p->so.tok;
-  ap.o_head_stride = p->so.head;
-  ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)p->head_dim));
-  ap.status = status;
-  ap.wait_limit_ns = p->wait_limit_ns;
-  ap.v_lbo = p->v_lbo;
-  ap.v_sbo = p->v_sbo;
-  ap.fault_inject = 0;
-  if (p->head_dim == 128) {
-    sol::attn_fwd_kernel<128><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(tm_q, tm_k, tm_v,
-                                                                                                      ap);
-  } else {
-    sol::attn_fwd_kernel<64><<<p->total_work, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(tm_q, tm_k, tm_v,
-                                                                                                    ap);
-  }
-  if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
-  return SOL_ATTN3D_OK;
+  // from here on the same code as every other forward, pointed at the built-in array
+  FwdOpts o;
+  o.ws = ws;
+  o.status = status;
+  o.encode = g_static_encode;
+  o.sm_count = sm_count;
+  return forward_impl(p, q, k, v, out, key_mask, stream, o);
 }
 
 size_t sol_attn3d_host_staging_bytes(sol_attn3d_plan_t p) {
@@ -1164,6 +1128,7 @@ int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void*
     o.head_begin = h0;
     o.head_end = h1;
     o.skip_keybits = g > 0;
+    o.keep_launch_count = g > 0;
     rc = forward_impl(p, dq, dk, dv, dout, dmask, stream, o);
     if (rc != SOL_ATTN3D_OK) break;
     if ((e = cudaEventRecord(p->ev_out[g], st)) != cudaSuccess) return fail_cuda(p, e);
@@ -1189,9 +1154,16 @@ int sol_attn3d_status(sol_attn3d_plan_t p) {
   return w == 0 ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_DEVICE_TIMEOUT;
 }
 
-int sol_attn3d_launches_per_forward(sol_attn3d_plan_t p, int with_mask) {
-  if (p == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
-  return with_mask ? 3 : 2;
+int sol_attn3d_last_launch_count(sol_attn3d_plan_t p) { return p == nullptr ? SOL_ATTN3D_ERR_INVALID_ARG : p->launches; }
+
+int sol_attn3d_softmax_rescale_count(sol_attn3d_plan_t p, unsigned long long* count) {
+  if (p == nullptr || count == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  unsigned int w = 0;
+  const cudaError_t e = cudaMemcpy(&w, p->ws + p->off_status + kCountersOffset, sizeof(w), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(p, e);
+  *count = w;
+  return SOL_ATTN3D_OK;
 }
 
 int sol_attn3d_last_cuda_error(sol_attn3d_plan_t p) { return p ? p->last_cuda : 0; }

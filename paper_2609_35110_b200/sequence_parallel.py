@@ -7,9 +7,12 @@ collective each way, as in the paper; the packed QKV receive buffer is consumed 
 and the attention's own output buffer is the send buffer of the return path, so neither side makes a layout copy
 beyond the pack and the merge.
 
-Transport "peer" (optional; needs `torch.distributed._symmetric_memory`, one node): the pack kernel stores
-straight into the owners' receive buffers and the attention epilogue stores each output row straight into its
-token owner's merged buffer, so the only collectives left are two barriers.
+Transport "peer" (optional, one node): the pack kernel stores straight into the owners' receive buffers and the
+attention epilogue stores each output row straight into its token owner's merged buffer, so the only
+collectives left are barriers.  Where the buffers come from is a separate object (`PeerBuffers`):
+`symmetric_memory_buffers` maps every rank's buffers into this process with
+`torch.distributed._symmetric_memory`; `local_peer_buffers` puts all ranks' buffers on one device, which is how
+the transport's own code runs in single-GPU tests (the ranks then take turns phase by phase).
 """
 from __future__ import annotations
 
@@ -61,6 +64,60 @@ class ExchangePlan:
                 [(b - a) * out_row for a, b in self.ranges], [self.n_local * out_row] * self.n_ranks)
 
 
+class PeerBuffers:
+    """Memory of the peer transport as one rank sees it: its own receive buffers and every rank's addresses.
+
+    qkv          this rank's packed QKV receive buffer [total, 3, heads/G, D] bf16
+    merged       this rank's output rows [largest shard, heads, D]
+    qkv_peers    device addresses of every rank's `qkv`, by rank (this rank's own included)
+    merged_peers the same for `merged`
+    barrier      callable: orders the phases across ranks (stream-ordered; a no-op where one stream runs all ranks)
+    """
+
+    def __init__(self, rank, n_ranks, qkv, merged, qkv_peers, merged_peers, barrier, keep=None):
+        self.rank, self.n_ranks = rank, n_ranks
+        self.qkv, self.merged = qkv, merged
+        self.qkv_peers, self.merged_peers = [int(x) for x in qkv_peers], [int(x) for x in merged_peers]
+        self.barrier = barrier
+        self.keep = keep                                   # whatever must stay alive with the buffers (handles)
+
+
+def peer_buffer_shapes(total: int, heads: int, head_dim: int, n_ranks: int):
+    """([total, 3, heads/G, D], [largest shard, heads, D]): the two buffers every rank of the peer transport owns."""
+    per = shard_ranges(total, n_ranks)[0]
+    return (total, 3, heads // n_ranks, head_dim), (max(per[1] - per[0], 1), heads, head_dim)
+
+
+def symmetric_memory_buffers(total, heads, head_dim, out_dtype, device, group=None) -> PeerBuffers:
+    """Buffers in symmetric memory, every rank's mapped into this process (plain peer addresses; no multicast is
+    used by the kernels that store through them).  Collective: every rank of `group` must call it."""
+    import torch.distributed as dist
+    import torch.distributed._symmetric_memory as symm
+    n_ranks, rank = dist.get_world_size(group), dist.get_rank(group)
+    qkv_shape, merged_shape = peer_buffer_shapes(total, heads, head_dim, n_ranks)
+    qkv = symm.empty(qkv_shape, dtype=torch.bfloat16, device=device)
+    merged = symm.empty(merged_shape, dtype=out_dtype, device=device)
+    gname = (group or dist.group.WORLD).group_name
+    hq, hm = symm.rendezvous(qkv, gname), symm.rendezvous(merged, gname)
+    token = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def barrier():
+        # stream-ordered: every rank's earlier kernels on this stream are complete when the reduction returns
+        dist.all_reduce(token, group=group)
+
+    return PeerBuffers(rank, n_ranks, qkv, merged, hq.buffer_ptrs, hm.buffer_ptrs, barrier, keep=(hq, hm, token))
+
+
+def local_peer_buffers(total, heads, head_dim, n_ranks, out_dtype, device) -> List[PeerBuffers]:
+    """All ranks' buffers on one device (one PeerBuffers per rank, sharing the address lists).  The ranks' phases
+    are then run one after another on one stream, which orders them: the barrier is a no-op."""
+    qkv_shape, merged_shape = peer_buffer_shapes(total, heads, head_dim, n_ranks)
+    qkvs = [torch.empty(qkv_shape, dtype=torch.bfloat16, device=device) for _ in range(n_ranks)]
+    mergeds = [torch.empty(merged_shape, dtype=out_dtype, device=device) for _ in range(n_ranks)]
+    qp, mp = [t.data_ptr() for t in qkvs], [t.data_ptr() for t in mergeds]
+    return [PeerBuffers(r, n_ranks, qkvs[r], mergeds[r], qp, mp, lambda: None) for r in range(n_ranks)]
+
+
 class _HeadGroup:
     """Buffers and plan of one head group of this rank's shard (collective transport)."""
 
@@ -91,17 +148,25 @@ class SequenceParallelAttn3d:
 
     def __init__(self, seqs: Sequence[Tuple[int, int, int, int]], heads: int, head_dim: int, rope_dims, theta: float = 10000.0,
                  group=None, device="cuda", out_format: str = "bf16", transport: str = "collective", qkv_wire: str = "bf16",
-                 n_groups: int = 1):
+                 n_groups: int = 1, peer_buffers: Optional[PeerBuffers] = None):
         """out_format: what travels back and is returned -- "bf16", "e4m3" (raw bytes, returned as uint8) or "int8"
         (block-INT8 records on the wire, dequantised to bf16 on arrival).  qkv_wire: "bf16" or "int8" (block-INT8
         records on the wire, dequantised to bf16 before the attention).  The quantised formats are approximate.
         n_groups (collective transport): this rank's head shard is served in that many head groups; the exchanges
-        of one group run on side streams under the attention of another (heads are independent)."""
-        import torch.distributed as dist
-        self.dist = dist
-        self.group = group
-        self.n_ranks = dist.get_world_size(group)
-        self.rank = dist.get_rank(group)
+        of one group run on side streams under the attention of another (heads are independent).
+        peer_buffers (peer transport): where the buffers live and who the ranks are; default: symmetric memory over
+        `group`.  With buffers from local_peer_buffers no process group is needed."""
+        if peer_buffers is not None:
+            if transport != "peer":
+                raise ValueError("peer_buffers belong to transport 'peer'")
+            self.dist, self.group = None, None
+            self.n_ranks, self.rank = peer_buffers.n_ranks, peer_buffers.rank
+        else:
+            import torch.distributed as dist
+            self.dist = dist
+            self.group = group
+            self.n_ranks = dist.get_world_size(group)
+            self.rank = dist.get_rank(group)
         if out_format not in ("bf16", "e4m3", "int8"):
             raise ValueError("out_format: 'bf16', 'e4m3' or 'int8'")
         if qkv_wire not in ("bf16", "int8"):
@@ -133,23 +198,33 @@ class SequenceParallelAttn3d:
             self.s_in = torch.cuda.Stream(device=device)       # QKV pack + exchange (+ dequantisation)
             self.s_out = torch.cuda.Stream(device=device)      # output exchange + merge (+ dequantisation)
         else:
-            import torch.distributed._symmetric_memory as symm
             qkv_strides = (3 * hl * D, D)
             self.attn = B.Attn3d(seqs, hl, D, rope_dims, theta, device, q_strides=qkv_strides, k_strides=qkv_strides,
                                  v_strides=qkv_strides)
-            per = self.xp.ranges[0][1] - self.xp.ranges[0][0]          # largest shard: same size on every rank
-            self.qkv = symm.empty((total, 3, hl, D), dtype=torch.bfloat16, device=device)
-            self.merged = symm.empty((max(per, 1), heads, D), dtype=self.out_dtype, device=device)
-            gname = (group or dist.group.WORLD).group_name
-            self.qkv_handle = symm.rendezvous(self.qkv, gname)
-            self.merged_handle = symm.rendezvous(self.merged, gname)
-            self.qkv_peers = [int(p) for p in self.qkv_handle.buffer_ptrs]
-            self.merged_peers = [int(p) for p in self.merged_handle.buffer_ptrs]
-            self._token = torch.zeros(1, dtype=torch.int32, device=device)
+            self.pb = peer_buffers if peer_buffers is not None else symmetric_memory_buffers(
+                total, heads, D, self.out_dtype, device, group)
+            qkv_shape, merged_shape = peer_buffer_shapes(total, heads, D, self.n_ranks)
+            if tuple(self.pb.qkv.shape) != qkv_shape or tuple(self.pb.merged.shape) != merged_shape or \
+                    self.pb.merged.dtype != self.out_dtype or len(self.pb.qkv_peers) != self.n_ranks or \
+                    len(self.pb.merged_peers) != self.n_ranks:
+                raise ValueError("peer buffers do not fit this problem")
 
-    def _barrier(self):
-        # stream-ordered: every rank's earlier kernels on this stream are complete when the reduction returns
-        self.dist.all_reduce(self._token, group=self.group)
+    # ---- peer transport, phase by phase (forward() runs them with barriers in between)
+    def peer_pack(self, q, k, v):
+        """Phase 1: this rank's Q, K, V rows go straight into every owner's receive buffer."""
+        B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, self.pb.qkv_peers, self.xp.first_token)
+
+    def peer_attend(self, key_mask=None):
+        """Phase 2 (after every rank's phase 1): attention over this rank's head shard; the epilogue stores each
+        output row into its token owner's merged buffer, at this shard's head offset."""
+        qkv = self.pb.qkv
+        B.sol_attn3d_forward_scatter(self.attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], key_mask, self.pb.merged_peers,
+                                     self.xp.tok_begin, self.heads, self.rank * self.xp.hl,
+                                     B.OUT_E4M3 if self.fp8 else B.OUT_BF16)
+
+    def peer_result(self):
+        """Phase 3 (after every rank's phase 2): this rank's token rows, all heads."""
+        return self.pb.merged[:self.xp.n_local]
 
     def forward(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, key_mask: Optional[torch.Tensor] = None) -> torch.Tensor:
         """q, k, v: [n_local, heads, D] bf16 (any strides, e.g. views into packed QKV); key_mask: uint8 [total] or None."""
@@ -159,14 +234,12 @@ class SequenceParallelAttn3d:
         if self.transport == "collective":
             return self._forward_collective(q, k, v, key_mask)
         # peer transport: stores into the owners' buffers, barriers instead of payload collectives
-        qv, kv, vv = self.qkv[:, 0], self.qkv[:, 1], self.qkv[:, 2]
-        self._barrier()                                       # everyone is done reading last call's buffers
-        B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, self.qkv_peers, xp.first_token)
-        self._barrier()
-        B.sol_attn3d_forward_scatter(self.attn.plan, qv, kv, vv, key_mask, self.merged_peers, xp.tok_begin, self.heads,
-                                     self.rank * xp.hl, B.OUT_E4M3 if self.fp8 else B.OUT_BF16)
-        self._barrier()
-        return self.merged[:xp.n_local]
+        self.pb.barrier()                                     # everyone is done reading last call's buffers
+        self.peer_pack(q, k, v)
+        self.pb.barrier()
+        self.peer_attend(key_mask)
+        self.pb.barrier()
+        return self.peer_result()
 
     def _forward_collective(self, q, k, v, key_mask):
         xp, D, G = self.xp, self.head_dim, self.n_ranks

@@ -532,3 +532,60 @@ def test_full_size_lowres_e4m3_and_scatter_sampled_rows(B):
             assert max_abs <= TOL_MAX_ABS and rel_l2 <= TOL_REL_L2
     assert bool(torch.isnan(got[:, :r * hl].float()).all()) and bool(torch.isnan(got[:, (r + 1) * hl:].float()).all()), \
         "the scatter epilogue wrote outside its head columns"
+
+
+# ------------------------------------------------------------------------------------------ peer transport, the module's own code
+@pytest.mark.parametrize("name,heads,G,fmt", [("lowres", 8, 4, "bf16"), ("varlen", 6, 3, "bf16"), ("cfg_batch", 8, 8, "bf16"),
+                                              ("lowres", 8, 2, "e4m3")])
+def test_peer_transport_of_the_module_with_virtual_ranks(B, name, heads, G, fmt):
+    """SequenceParallelAttn3d(transport="peer") with all ranks' buffers on this GPU (local_peer_buffers): every rank
+    is an instance of the module, and the ranks run its three phases in turn -- all pack, all attend, all read --
+    which is the order the barriers of a real run enforce.  Exercises the module's own pointer plumbing (token
+    offsets, head offsets, buffer sizes by the largest shard, the slice returned).  Result: each rank's token rows of
+    the single-device attention, bit for bit, and equal to the collective transport's kernels called by hand."""
+    from paper_2609_35110_b200.sequence_parallel import SequenceParallelAttn3d, local_peer_buffers, shard_ranges
+    w = replace(wl.shrunk(name), heads=heads)
+    inp = wl.make_inputs(w, "cuda")
+    out_dtype = torch.uint8 if fmt == "e4m3" else torch.bfloat16
+    bufs = local_peer_buffers(w.total_tokens, heads, w.head_dim, G, out_dtype, "cuda")
+    for pb in bufs:                                            # poison: an unwritten element shows
+        pb.qkv.fill_(float("nan"))
+        pb.merged.view(torch.uint8).fill_(0x7F)
+    ranks = [SequenceParallelAttn3d(seq_tuples(w), heads, w.head_dim, w.rope_dims, w.theta, transport="peer", out_format=fmt,
+                                    peer_buffers=bufs[r]) for r in range(G)]
+    ranges = shard_ranges(w.total_tokens, G)
+    for r, (a, b) in enumerate(ranges):
+        assert ranks[r].xp.n_local == b - a
+        if b > a:
+            ranks[r].peer_pack(inp.q[a:b], inp.k[a:b], inp.v[a:b])
+    for r in range(G):
+        ranks[r].peer_attend(inp.key_mask)
+    torch.cuda.synchronize()
+    for r in range(G):
+        assert ranks[r].attn.status() == 0
+    got = torch.cat([ranks[r].peer_result() for r in range(G)], dim=0)
+    assert got.shape[0] == w.total_tokens
+    single = B.Attn3d.from_workload(w, "cuda")
+    if fmt == "e4m3":
+        want = torch.empty((w.total_tokens, heads, w.head_dim), dtype=torch.uint8, device="cuda")
+        B.sol_attn3d_forward_e4m3(single.plan, inp.q, inp.k, inp.v, want, inp.key_mask)
+    else:
+        want = single.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    torch.cuda.synchronize()
+    single.close()
+    assert torch.equal(got.view(torch.uint8), want.view(torch.uint8))
+    by_hand = torch.cat(virtual_ranks_forward(B, w, inp, G, B.OUT_E4M3 if fmt == "e4m3" else B.OUT_BF16, False), dim=0)
+    assert torch.equal(got.view(torch.uint8), by_hand.view(torch.uint8))
+    if fmt == "bf16":
+        max_abs, rel_l2 = orc.compare(got.cpu(), oracle_dense(w, inp))
+        assert max_abs <= TOL_MAX_ABS and rel_l2 <= TOL_REL_L2
+    # forward() of one rank in a one-rank "job" runs the same phases with its (no-op) barriers
+    solo_buf = local_peer_buffers(w.total_tokens, heads, w.head_dim, 1, out_dtype, "cuda")[0]
+    solo = SequenceParallelAttn3d(seq_tuples(w), heads, w.head_dim, w.rope_dims, w.theta, transport="peer", out_format=fmt,
+                                  peer_buffers=solo_buf)
+    got1 = solo.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    torch.cuda.synchronize()
+    assert torch.equal(got1.view(torch.uint8), want.view(torch.uint8))
+    solo.close()
+    for r in ranks:
+        r.close()

@@ -42,3 +42,37 @@ def test_rect_forward_computes_only_wanted_rows(name):
     max_abs, rel_l2 = orc.compare(got, torch.cat(ref))
     assert max_abs <= 2e-2 and rel_l2 <= 5e-3
     attn.close()
+
+
+def test_rect_full_size_low_resolution_stage():
+    """The low-resolution-stage shape at full size (25,216 tokens, 40 heads): the first 60 % of the video are
+    reference tokens whose query rows are skipped (39 whole query blocks cost nothing, one is partial), plus a few
+    scattered skipped rows elsewhere.  Wanted rows equal the dense forward bit for bit, skipped rows are never
+    written, and sampled wanted rows match the oracle."""
+    from paper_2609_35110_b200 import binding as B
+    w = wl.CONFIGS["lowres"]
+    inp = wl.make_inputs(w, "cuda")
+    seqs = [(s.text_len, s.T, s.H, s.W) for s in w.seqs]
+    sq = w.seqs[0]
+    qmask = torch.ones(w.total_tokens, dtype=torch.uint8)
+    qmask[sq.text_len: sq.text_len + int(0.6 * sq.n_video)] = 0
+    qmask[torch.arange(20000, 25216, 97)] = 0
+    attn = B.Attn3d.from_workload(w, "cuda")
+    dense = attn.forward(inp.q, inp.k, inp.v, None)
+    out = torch.full_like(dense, 7.0)
+    B.sol_attn3d_forward_rect(attn.plan, inp.q, inp.k, inp.v, out, None, qmask.cuda())
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    want = qmask.bool().cuda()
+    assert torch.equal(out[want], dense[want])
+    assert bool((out[~want] == 7.0).all())
+    o, q, k, v = out.cpu(), inp.q.cpu(), inp.k.cpu(), inp.v.cpu()
+    sel = []
+    for h in (0, 21, w.heads - 1):
+        rows = torch.from_numpy(wl.sample_rows(w, 0, h, 512))
+        sel.append((0, h, rows[qmask[rows].bool()]))
+    ref = orc.attn3d_oracle(q, k, v, seqs, w.rope_dims, w.theta, None, sel)
+    got = torch.cat([o[rows, h] for (_, h, rows) in sel])
+    max_abs, rel_l2 = orc.compare(got, torch.cat(ref))
+    assert max_abs <= 2e-2 and rel_l2 <= 5e-3
+    attn.close()

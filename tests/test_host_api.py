@@ -116,8 +116,8 @@ def test_device_calls_fail_cleanly_without_workspace_or_device():
     if not torch.cuda.is_available():
         # a plausible pointer on a machine without a GPU: refused before anything is touched
         assert lib.sol_attn3d_set_workspace(p, 1 << 20, 1 << 30) in (B.ERR_NO_DEVICE, B.ERR_CUDA)
-    assert B.sol_attn3d_launches_per_forward(p, True) == 3
-    assert B.sol_attn3d_launches_per_forward(p, False) == 2
+    assert B.sol_attn3d_last_launch_count(p) == 0                                         # nothing was enqueued
+    assert lib.sol_attn3d_softmax_rescale_count(p, None) == B.ERR_INVALID_ARG
     assert B.sol_attn3d_strerror(B.ERR_DEVICE_TIMEOUT)
     assert lib.sol_attn3d_destroy(None) == 0
     B.sol_attn3d_destroy(p)

@@ -478,26 +478,30 @@ def test_qk_norm_inside_attention_matches_brute_force_and_order():
 def test_block_select_rule_on_hand_made_scores():
     # one query block, scores 0..7: mu = 3.5, sigma = sqrt(5.25) = 2.2913
     sc = torch.arange(8, dtype=F64)[None]
-    assert orc.block_select(sc, 1.0, 0).tolist() == [[False] * 6 + [True, True]]       # > 5.79
-    assert orc.block_select(sc, 1.5, 0).tolist() == [[False] * 7 + [True]]             # > 6.94
-    assert orc.block_select(sc, 0.0, 0).tolist() == [[False] * 4 + [True] * 4]         # > mean
+    assert orc.block_select(sc, 1.0, 0, 256, 128).tolist() == [[False] * 6 + [True, True]]       # > 5.79
+    assert orc.block_select(sc, 1.5, 0, 256, 128).tolist() == [[False] * 7 + [True]]             # > 6.94
+    assert orc.block_select(sc, 0.0, 0, 256, 128).tolist() == [[False] * 4 + [True] * 4]         # > mean
     # constant scores: sigma = 0, nothing is strictly above the mean; the arg-max block is kept
-    assert int(orc.block_select(torch.ones(1, 5, dtype=F64), 1.0, 0).sum()) == 1
+    assert int(orc.block_select(torch.ones(1, 5, dtype=F64), 1.0, 0, 256, 128).sum()) == 1
     # rails: prefix of 130 tokens = KV blocks 0 and 1 always on; query block 0 (holds prefix rows) dense
     sc = torch.tensor([[0.0, 0, 0, 0, 9.0], [0.0, 0, 0, 0, 9.0]], dtype=F64)
-    sel = orc.block_select(sc, 1.0, 130)
+    sel = orc.block_select(sc, 1.0, 130, 256, 128)
     assert sel.tolist() == [[True] * 5, [True, True, False, False, True]]
+    # the rails follow the block sizes: with 64-token KV blocks the same prefix covers three of them, and with
+    # 128-token query blocks both query blocks hold prefix rows
+    assert orc.block_select(sc, 1.0, 130, 256, 64).tolist() == [[True] * 5, [True, True, True, False, True]]
+    assert orc.block_select(sc, 1.0, 130, 128, 128).tolist() == [[True] * 5, [True] * 5]
     # a larger tau never selects more
     g = torch.Generator().manual_seed(5)
     sc = torch.randn(6, 40, generator=g, dtype=F64)
-    a, b, c = (orc.block_select(sc, t, 0) for t in (1.0, 1.25, 1.5))
+    a, b, c = (orc.block_select(sc, t, 0, 256, 128) for t in (1.0, 1.25, 1.5))
     assert bool((b <= a).all()) and bool((c <= b).all()) and int(c.sum()) < int(a.sum())
 
 
 def test_block_scores_are_pooled_logits():
     n, D = 300, 8
     q, k = rnd(n, D, seed=300).to(F64), rnd(n, D, seed=301).to(F64)
-    sc = orc.block_scores(q, k, D)
+    sc = orc.block_scores(q, k, D, 256, 128)
     assert sc.shape == (2, 3)
     # block (1, 2): query rows 256..299, keys 256..299 (ragged tails average over what is there)
     want = float(q[256:].mean(0) @ k[256:].mean(0)) / math.sqrt(D)
@@ -505,6 +509,11 @@ def test_block_scores_are_pooled_logits():
     # pooled logits = mean of the full logit block (bilinearity)
     full = (q[:256] @ k[128:256].t()) / math.sqrt(D)
     assert abs(float(sc[0, 1]) - float(full.mean())) < 1e-13
+    # other block sizes: 7 query blocks of 50 (no tail), 4 KV blocks of 96 (tail of 12)
+    sc = orc.block_scores(q, k, D, 50, 96)
+    assert sc.shape == (6, 4)
+    full = (q[100:150] @ k[288:].t()) / math.sqrt(D)
+    assert abs(float(sc[2, 3]) - float(full.mean())) < 1e-13
 
 
 def test_sparse_oracle_reduces_to_dense_and_respects_selection():
@@ -514,22 +523,34 @@ def test_sparse_oracle_reduces_to_dense_and_respects_selection():
     dense = orc.attn3d_oracle(q, k, v, seqs, (4, 6, 6), 10000.0)
     # everything selected = dense attention
     full = [[torch.ones(3, 6, dtype=torch.bool) for _ in range(2)]]
-    out, _, _ = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 1.0, selection=full)
+    out, _, _ = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 1.0, 256, 128, selection=full)
     assert torch.allclose(out, dense, atol=1e-13)
     # tau = -inf selects everything as well
-    out, used, sc = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, -1e30)
+    out, used, sc = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, -1e30, 256, 128)
     assert torch.allclose(out, dense, atol=1e-13) and all(bool(u.all()) for u in used[0])
     # a real tau: prefix rails hold, prefix query block equals dense, a dropped block's V does not matter
-    out, used, sc = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 0.5)
+    out, used, sc = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 0.5, 256, 128)
     sel = used[0][1]
     assert bool(sel[:, :2].all()) and bool(sel[0].all()) and not bool(sel.all())
     assert torch.allclose(out[:256], dense[:256], atol=1e-13)
     i, j = [(int(a), int(b)) for a, b in zip(*torch.nonzero(~sel, as_tuple=True))][0]
     v2 = v.clone()
     v2[j * 128: (j + 1) * 128, 1] = 50.0
-    out2, _, _ = orc.attn3d_sparse_oracle(q, k, v2, seqs, (4, 6, 6), 10000.0, 0.5, selection=used)
+    out2, _, _ = orc.attn3d_sparse_oracle(q, k, v2, seqs, (4, 6, 6), 10000.0, 0.5, 256, 128, selection=used)
     assert torch.equal(out2[i * 256: (i + 1) * 256, 1], out[i * 256: (i + 1) * 256, 1])
-    # the block statistic is taken on bf16-rounded rotated operands
-    qr = orc.rope_oracle(q, seqs, (4, 6, 6), 10000.0)[:, 1].to(torch.bfloat16).to(F64)
-    kr = orc.rope_oracle(k, seqs, (4, 6, 6), 10000.0)[:, 1].to(torch.bfloat16).to(F64)
-    assert torch.equal(sc[0][1], orc.block_scores(qr, kr, 16))
+    # the block statistic is taken on the rotated operands in fp64, nothing rounded
+    qr = orc.rope_oracle(q, seqs, (4, 6, 6), 10000.0)[:, 1]
+    kr = orc.rope_oracle(k, seqs, (4, 6, 6), 10000.0)[:, 1]
+    assert torch.equal(sc[0][1], orc.block_scores(qr, kr, 16, 256, 128))
+    # sampled rows of one (sequence, head) = the same rows of the all-rows result, with and without a given selection
+    rows = torch.tensor([0, 255, 256, 300, 511, 512, 649])
+    o_s, u_s, sc_s = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 0.5, 256, 128, select=[(0, 1, rows)])
+    # (the library matmul may block 7 rows differently from 256: equal to rounding of fp64, not to the bit)
+    assert torch.allclose(o_s[0], out[rows, 1], atol=1e-14) and torch.equal(u_s[0], used[0][1]) and torch.equal(sc_s[0], sc[0][1])
+    o_s, _, _ = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 0.5, 256, 128, selection=[used[0][1]],
+                                         select=[(0, 1, rows)])
+    assert torch.allclose(o_s[0], out[rows, 1], atol=1e-14)
+    # other block sizes give another (valid) approximation: 128-token query blocks select per 128 rows
+    out_b, used_b, _ = orc.attn3d_sparse_oracle(q, k, v, seqs, (4, 6, 6), 10000.0, 0.5, 128, 64)
+    assert used_b[0][0].shape == (6, 11) and bool(used_b[0][0][:, :3].all()) and bool(used_b[0][0][:2].all())
+    assert torch.allclose(out_b[:256], dense[:256], atol=1e-13)
