@@ -589,3 +589,46 @@ def test_peer_transport_of_the_module_with_virtual_ranks(B, name, heads, G, fmt)
     solo.close()
     for r in ranks:
         r.close()
+
+
+_PEER_ONE_RANK = r'''
+import os, sys
+sys.path.insert(0, os.getcwd())
+import torch, torch.distributed as dist
+from dataclasses import replace
+from paper_2609_35110_b200 import binding as B, workloads as wl
+from paper_2609_35110_b200.sequence_parallel import SequenceParallelAttn3d
+dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+w = replace(wl.shrunk("cfg_batch"), heads=4)
+inp = wl.make_inputs(w, "cuda")
+seqs = [(s.text_len, s.T, s.H, s.W) for s in w.seqs]
+single = B.Attn3d.from_workload(w, "cuda")
+want = single.forward(inp.q, inp.k, inp.v, inp.key_mask)
+want8 = torch.empty(want.shape, dtype=torch.uint8, device="cuda")
+B.sol_attn3d_forward_e4m3(single.plan, inp.q, inp.k, inp.v, want8, inp.key_mask)
+for fmt, ref in (("bf16", want), ("e4m3", want8)):
+    sp = SequenceParallelAttn3d(seqs, w.heads, w.head_dim, w.rope_dims, w.theta, transport="peer", out_format=fmt)
+    assert sp.pb.qkv_peers[0] == sp.pb.qkv.data_ptr() and sp.pb.merged_peers[0] == sp.pb.merged.data_ptr()
+    for _ in range(2):                                   # twice: the leading barrier protects the buffers of the last call
+        got = sp.forward(inp.q, inp.k, inp.v, inp.key_mask)
+        torch.cuda.synchronize()
+        assert torch.equal(got.view(torch.uint8), ref.view(torch.uint8)), fmt
+    assert sp.attn.status() == 0
+    sp.close()
+dist.destroy_process_group()
+print("PEER_ONE_RANK_OK")
+'''
+
+
+def test_peer_transport_with_symmetric_memory_one_rank(B):
+    """The real buffer provider of the peer transport: symmetric-memory allocation and rendezvous over an NCCL
+    group, peer addresses from the handles, the three stream-ordered barriers.  One rank (this run has one GPU), in a
+    child process so that multicast binding is switched off for NCCL and for the symmetric-memory allocator before
+    either initialises; the kernels use plain stores through the mapped addresses."""
+    import subprocess
+    import sys
+    env = dict(os.environ, NCCL_NVLS_ENABLE="0", TORCH_SYMM_MEM_DISABLE_MULTICAST="1", MASTER_ADDR="127.0.0.1",
+               MASTER_PORT=str(29900 + os.getpid() % 90))
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", _PEER_ONE_RANK], cwd=root, env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0 and "PEER_ONE_RANK_OK" in res.stdout, res.stdout[-2000:] + res.stderr[-4000:]
