@@ -1,7 +1,13 @@
 // Attention main kernel for sm_100a: S = Q~ K~^T and O += P V on tcgen05 tensor cores with the
 // accumulators in tensor memory, TMA-fed shared-memory ring, online softmax in registers.
 //
-// One CTA = one (sequence, head, pair of 128-row query tiles).  Warp roles:
+// One CTA = one (sequence, head, pair of 128-row query tiles).  With kCtas = 2 two such CTAs on neighbouring SMs
+// form a cluster that covers 512 consecutive query rows of one (sequence, head) and shares every K / V tile:
+// each CTA loads HALF of the tile (K: 64 of the 128 keys; V: 64 of the 128 head dims) with its own TMA loads and
+// one tcgen05.mma.cta_group::2 of M = 256 works on both CTAs' query rows, which halves the shared-memory reads of
+// the B operand and the L2 -> SM traffic per flop.  The even CTA (the leader) issues all MMAs; completion goes to
+// both CTAs with a multicast commit.  Nothing is loaded with multicast.
+// Warp roles (per CTA):
 //   warps 0-3   softmax / correction / epilogue of query tile 0 (thread = one query row)
 //   warps 4-7   the same for query tile 1
 //   warp  8     TMA producer (lane 0)
@@ -44,11 +50,6 @@ constexpr int kAttnThreads = 384;   // 8 softmax warps + producer + MMA issuer +
 #endif
 #ifndef SOL_EMU_CNT
 #define SOL_EMU_CNT 0
-#endif
-// P hand-over to the MMA issuer: 1 = one arrival per softmax warp (lane 0, after the warp has synchronised)
-// instead of one per thread.
-#ifndef SOL_PFULL_PER_WARP
-#define SOL_PFULL_PER_WARP 0
 #endif
 
 __device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
@@ -188,26 +189,30 @@ __device__ __forceinline__ void softmax_half(const uint32_t (&r)[64], float c, f
   }
 }
 
-template <int D>
+template <int D, int kCtas = 1>
 struct AttnSmem {
   static constexpr int kTile = 128 * D * 2;               // bytes of one 128 x D bf16 tile
   static constexpr int kHalves = D / 64;                  // 64-column (128-byte) swizzle boxes per row
   static constexpr int kHalfBytes = 128 * 128;            // one box: 128 rows x 128 bytes
-  static constexpr int kStages = (D == 128) ? 5 : 10;     // K/V ring (K and V tiles alternate)
+  static constexpr int kStageBytes = kTile / kCtas;       // what one CTA holds of a K or V tile
+  static constexpr int kKBoxBytes = kHalfBytes / kCtas;   // one K box: (128 / kCtas) keys x 128 bytes
+  static constexpr int kStages = ((D == 128) ? 5 : 10) * (kCtas == 2 ? 8 : 5) / 5;   // K/V ring (K and V tiles alternate)
   static constexpr int kOffQ = 0;
   static constexpr int kOffKV = 2 * kTile;
-  static constexpr int kOffBars = kOffKV + kStages * kTile;
+  static constexpr int kOffBars = kOffKV + kStages * kStageBytes;
   static constexpr int kNumBars = 1 + 2 * kStages + 7;  // q_full, kv_full/empty, s_full[2], p_full[2], o_done[2], drain
   static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
   static constexpr int kBytes = kOffTmemPtr + 16;
   static constexpr int kDynBytes = kBytes + 1024;         // slack to align the base to 1024 bytes
 };
 
-template <int D>
+template <int D, int kCtas>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
-  using L = AttnSmem<D>;
+  static_assert(kCtas == 1 || (kCtas == 2 && D == 128), "CTA pairs are built for head_dim 128");
+  using L = AttnSmem<D, kCtas>;
+  constexpr bool kPair = kCtas == 2;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t sbase = (raw_addr + 1023u) & ~1023u;
@@ -215,6 +220,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  // CTA pairs: rank 0 is the leader (issues the MMAs, owns the barriers the other CTA reports to)
+  const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+  const bool leader = rank == 0;
 
   const uint32_t sQ = sbase + L::kOffQ;
   const uint32_t sKV = sbase + L::kOffKV;
@@ -228,34 +236,36 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t bar_drain = bars + 8u * (7 + 2 * L::kStages);
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + L::kOffTmemPtr);
 
-  // A fault recorded by an earlier CTA stops later ones at the door (read once, CTA-uniform).
-  if (threadIdx.x == 0) tmem_ptr_smem[1] = *reinterpret_cast<volatile unsigned int*>(p.status);
-  __syncthreads();
-  if (tmem_ptr_smem[1] != 0) return;
-
-  // ---- which work item
-  const int cta = (int)blockIdx.x + p.cta_offset;
+  // ---- which work item (one per CTA, or one per CTA pair)
+  const int unit = (int)blockIdx.x / kCtas + p.cta_offset;
   int si = 0;
-  while (si + 1 < p.n_seqs && cta >= p.seqs[si + 1].work_start) ++si;
+  if (kPair) { while (si + 1 < p.n_seqs && unit >= p.seqs[si + 1].quad_work_start) ++si; }
+  else       { while (si + 1 < p.n_seqs && unit >= p.seqs[si + 1].work_start) ++si; }
   const SeqDev sq = p.seqs[si];
-  const int local = cta - sq.work_start;
-  const int head = local / sq.n_qpairs;
-  const int pair = local - head * sq.n_qpairs;
-  // a launch may serve a range of heads only (CTA-uniform, before any set-up)
+  const int units_per_head = kPair ? (sq.n_qpairs + 1) / 2 : sq.n_qpairs;
+  const int local = unit - (kPair ? sq.quad_work_start : sq.work_start);
+  const int head = local / units_per_head;
+  const int blk = local - head * units_per_head;        // query pair (256 rows) or query quad (512 rows)
+  // a launch may serve a range of heads only (uniform over the CTA / the pair, before any set-up)
   if (head < p.head_begin || head >= p.head_end) return;
-  // rectangular mode: a query pair without a wanted row has nothing to do (CTA-uniform, before any set-up)
-  if (p.pair_needed != nullptr && p.pair_needed[sq.pair_start + pair] == 0) return;
-  // dense: every CTA of a sequence walks the same list of key tiles; block-sparse: each CTA has its own
-  const bool sparse = p.cta_list != nullptr;
-  const int n_proc = sparse ? p.cta_count[cta] : p.ktile_count[si];
+  // rectangular mode: a query block without a wanted row has nothing to do (uniform, before any set-up)
+  if (p.pair_needed != nullptr) {
+    const uint8_t* need = p.pair_needed + sq.pair_start;
+    bool any = need[kCtas * blk] != 0;
+    if (kPair && 2 * blk + 1 < sq.n_qpairs) any = any || need[2 * blk + 1] != 0;
+    if (!any) return;
+  }
+  // dense: every CTA of a sequence walks the same list of key tiles; block-sparse (single CTAs only): each CTA has its own
+  const bool sparse = !kPair && p.cta_list != nullptr;
+  const int n_proc = sparse ? p.cta_count[unit] : p.ktile_count[si];
   const int* __restrict__ ktiles =
       sparse ? p.cta_list + sq.sparse_list_start + (long long)local * sq.n_ktiles : p.ktile_list + sq.ktile_start;
   const uint4* __restrict__ keybits = p.keybits + sq.ktile_start;
   // Successive waves of CTAs walk the key tiles in opposite directions (the softmax does not care about the
   // order): a wave then starts on the tiles its predecessor touched last, which are still in L2, instead of
   // on the ones it touched first, which a long sequence has pushed out by then.
-  const bool backwards = ((cta / p.wave_ctas) & 1) != 0;
-  const int q_row0 = pair * 256;                       // first local query row of the CTA
+  const bool backwards = ((unit / max(1, p.wave_ctas / kCtas)) & 1) != 0;
+  const int q_row0 = blk * (256 * kCtas) + (int)rank * 256;   // first local query row of this CTA
   const int tok0 = (int)sq.tok_start;                  // TMA token coordinate of the sequence start
   const unsigned long long limit = p.wait_limit_ns;
 
@@ -267,7 +277,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(bar_s_full(t), 1);
-      mbar_init(bar_p_full(t), SOL_PFULL_PER_WARP ? 4 : 128);
+      mbar_init(bar_p_full(t), 4 * kCtas);              // one arrival per softmax warp of the tile, from every CTA
       mbar_init(bar_o_done(t), 1);
     }
     mbar_init(bar_drain, 1);
@@ -276,14 +286,32 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     prefetch_tensormap(&tm_k);
     prefetch_tensormap(&tm_v);
   }
+  // A fault recorded by an earlier CTA stops later ones at the door (read once; made uniform over the pair below).
+  if (threadIdx.x == 0) tmem_ptr_smem[1] = *reinterpret_cast<volatile unsigned int*>(p.status);
   if (warp == 9) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 512);
-    tmem_relinquish();
+    if (kPair) { tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 512); tmem_relinquish_pair(); }
+    else       { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 512); tmem_relinquish(); }
   }
   tc_fence_before();
-  __syncthreads();
+  if (kPair) cluster_sync_all(); else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_ptr_smem[0];
+  {
+    uint32_t stop = tmem_ptr_smem[1];
+    if (kPair) {
+      // both CTAs must take the same decision: each looks at both flags, and nobody leaves before the other has looked
+      stop |= ld_shared_cluster_u32(mapa_shared(smem_u32(const_cast<uint32_t*>(&tmem_ptr_smem[1])), rank ^ 1u));
+      cluster_sync_all();
+    }
+    if (stop != 0) {
+      if (warp == 9) {
+        if (kPair) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
+      }
+      return;
+    }
+  }
+  // barriers of the leader that this CTA reports to (its own when it is the leader)
+  const uint32_t lead_q_full = kPair ? mapa_shared(bar_q_full, 0) : bar_q_full;
 
   if (warp < 8) {
     // =========================================================== softmax / correction / epilogue
@@ -294,6 +322,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t lane_off = static_cast<uint32_t>(wq * 32) << 16;
     const uint32_t tS = tmem_base + lane_off + t * 128;
     const uint32_t tO = tmem_base + lane_off + 256 + t * D;
+    const uint32_t lead_p_full = kPair ? mapa_shared(bar_p_full(t), 0) : bar_p_full(t);
     const float c = p.scale_log2;
     float m_ref = -CUDART_INF_F;
     float l = 0.f;
@@ -381,12 +410,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
-#if SOL_PFULL_PER_WARP
+      // one arrival per warp, on the leader's barrier (the MMA over both CTAs' rows starts when all eight have come)
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p_full(t));
-#else
-      mbar_arrive(bar_p_full(t));
-#endif
+      if (lane == 0) {
+        if (kPair) mbar_arrive_cluster(lead_p_full); else mbar_arrive(lead_p_full);
+      }
     }
 
     // ---- epilogue: O / l in the output format, staged through shared memory, coalesced 16-byte stores
@@ -423,43 +451,63 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // CTA of the head streams (an evict-last hint on K / V was measured too: more DRAM reads, not fewer, because
       // the previous heads' tiles then linger)
       const uint64_t pol_once = l2_policy_evict_first();
-      mbar_arrive_expect_tx(bar_q_full, 2 * L::kTile);
+      // the leader's barrier counts the bytes of both CTAs' loads
+      if (leader) mbar_arrive_expect_tx(bar_q_full, kCtas * 2 * L::kTile);
 #pragma unroll
       for (int t = 0; t < 2; ++t)
 #pragma unroll
-        for (int hf = 0; hf < L::kHalves; ++hf)
-          tma_load_3d_hint(sQ + t * L::kTile + hf * L::kHalfBytes, &tm_q, bar_q_full, hf * 64, head,
-                           tok0 + q_row0 + t * 128, pol_once);
+        for (int hf = 0; hf < L::kHalves; ++hf) {
+          const uint32_t dst = sQ + t * L::kTile + hf * L::kHalfBytes;
+          if (kPair) tma_load_3d_pair_hint(dst, &tm_q, lead_q_full, hf * 64, head, tok0 + q_row0 + t * 128, pol_once);
+          else       tma_load_3d_hint(dst, &tm_q, bar_q_full, hf * 64, head, tok0 + q_row0 + t * 128, pol_once);
+        }
       uint32_t it = 0, stage = 0, par = 0;
       for (int i = 0; i < n_proc && ok; ++i) {
         const int jt = __ldg(&ktiles[backwards ? n_proc - 1 - i : i]);
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
           if (!mbar_wait(bar_kv_empty(stage), par ^ 1u, limit)) { ok = false; break; }
-          mbar_arrive_expect_tx(bar_kv_full(stage), L::kTile);
-          const CUtensorMap* tm = kv ? &tm_v : &tm_k;
+          if (leader) mbar_arrive_expect_tx(bar_kv_full(stage), L::kTile);
+          const uint32_t dst = sKV + stage * L::kStageBytes;
+          if (kPair) {
+            // this CTA's half of the tile: K = its 64 keys (all head dims, two boxes), V = its 64 head dims (all keys)
+            const uint32_t full = mapa_shared(bar_kv_full(stage), 0);
+            if (kv == 0) {
 #pragma unroll
-          for (int hf = 0; hf < L::kHalves; ++hf)
-            tma_load_3d(sKV + stage * L::kTile + hf * L::kHalfBytes, tm, bar_kv_full(stage), hf * 64, head, tok0 + jt * 128);
+              for (int hf = 0; hf < L::kHalves; ++hf)
+                tma_load_3d_pair(dst + hf * L::kKBoxBytes, &tm_k, full, hf * 64, head, tok0 + jt * 128 + (int)rank * 64);
+            } else {
+              tma_load_3d_pair(dst, &tm_v, full, (int)rank * 64, head, tok0 + jt * 128);
+            }
+          } else {
+            const CUtensorMap* tm = kv ? &tm_v : &tm_k;
+#pragma unroll
+            for (int hf = 0; hf < L::kHalves; ++hf)
+              tma_load_3d(dst + hf * L::kHalfBytes, tm, bar_kv_full(stage), hf * 64, head, tok0 + jt * 128);
+          }
           ++it;
           if (++stage == (uint32_t)L::kStages) { stage = 0; par ^= 1u; }
         }
       }
       if (!ok) {
         atomicCAS(p.status, 0u, kStatusTimeoutProducer);
-        // let the copies already in flight land before the CTA gives its shared memory back
-        mbar_wait(bar_q_full, 0, limit);
-        const uint32_t first = it > (uint32_t)L::kStages ? it - L::kStages : 0u;
-        for (uint32_t j = first; j < it; ++j) mbar_wait(bar_kv_full(j % L::kStages), (j / L::kStages) & 1u, limit);
+        // Let the copies already in flight land before the CTA gives its shared memory back.  A single CTA (and the
+        // leader of a pair) can see them on its own barriers; the other CTA of a pair reports to the leader's
+        // barriers and cannot, but the wait that just ran out lasted `limit`, far longer than any copy takes.
+        if (leader) {
+          mbar_wait(bar_q_full, 0, limit);
+          const uint32_t first = it > (uint32_t)L::kStages ? it - L::kStages : 0u;
+          for (uint32_t j = first; j < it; ++j) mbar_wait(bar_kv_full(j % L::kStages), (j / L::kStages) & 1u, limit);
+        }
       }
     }
     __syncwarp();
-  } else if (warp == 9) {
+  } else if (warp == 9 && leader) {
     // =========================================================== MMA issuer
     {
       // The whole warp runs this loop (convergent); one elected lane issues each tcgen05 instruction.
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false);
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, true);
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(128 * kCtas, 128, false);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(128 * kCtas, D, true);
       bool ok = true;
       const uint32_t v_lbo = p.v_lbo, v_sbo = p.v_sbo;
       // descriptor words: only the low word (address) moves inside the loop
@@ -468,24 +516,39 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint32_t q_lo0 = smem_desc_lo(sQ, 16), q_lo1 = smem_desc_lo(sQ + L::kTile, 16);
       const uint32_t k_lo_base = smem_desc_lo(sKV, 16);
       const uint32_t v_lo_base = smem_desc_lo(sKV, v_lbo);
-      constexpr uint32_t kStageStep = L::kTile >> 4;
+      constexpr uint32_t kStageStep = L::kStageBytes >> 4;
       const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128;
       const uint32_t tO0 = tmem_base + 256, tO1 = tmem_base + 256 + D;
+      auto commit = [&](uint32_t bar) { if (kPair) tc_commit_elect_pair(bar); else tc_commit_elect(bar); };
+      auto wait_full = [&](uint32_t bar, uint32_t parity) {
+        return kPair ? mbar_wait_cluster_warp(bar, parity, limit) : mbar_wait_warp(bar, parity, limit);
+      };
       auto issue_qk = [&](uint32_t d_tmem, uint32_t q_lo, uint32_t stage) {
         const uint32_t k_lo = k_lo_base + stage * kStageStep;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = ((k >> 2) * L::kHalfBytes + (k & 3) * 32) >> 4;
-          if (k == 0) mma_ss_elect<false>(d_tmem, q_lo + off, k_lo + off, hi_k, idesc_qk, 0u);
-          else        mma_ss_elect<true>(d_tmem, q_lo + off, k_lo + off, hi_k, idesc_qk, 1u);
+          const uint32_t q_off = ((k >> 2) * L::kHalfBytes + (k & 3) * 32) >> 4;
+          const uint32_t k_off = ((k >> 2) * L::kKBoxBytes + (k & 3) * 32) >> 4;
+          if (kPair) {
+            if (k == 0) mma_ss_elect_pair<false>(d_tmem, q_lo + q_off, k_lo + k_off, hi_k, idesc_qk, 0u);
+            else        mma_ss_elect_pair<true>(d_tmem, q_lo + q_off, k_lo + k_off, hi_k, idesc_qk, 1u);
+          } else {
+            if (k == 0) mma_ss_elect<false>(d_tmem, q_lo + q_off, k_lo + k_off, hi_k, idesc_qk, 0u);
+            else        mma_ss_elect<true>(d_tmem, q_lo + q_off, k_lo + k_off, hi_k, idesc_qk, 1u);
+          }
         }
       };
       auto issue_pv = [&](uint32_t d_tmem, uint32_t p_tmem, uint32_t stage, bool acc) {
         const uint32_t v_lo = v_lo_base + stage * kStageStep;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          if (k == 0) mma_ts_elect<false>(d_tmem, p_tmem, v_lo, hi_v, idesc_pv, acc ? 1u : 0u);
-          else        mma_ts_elect<true>(d_tmem, p_tmem + k * 8, v_lo + k * (2048 >> 4), hi_v, idesc_pv, 1u);
+          if (kPair) {
+            if (k == 0) mma_ts_elect_pair<false>(d_tmem, p_tmem, v_lo, hi_v, idesc_pv, acc ? 1u : 0u);
+            else        mma_ts_elect_pair<true>(d_tmem, p_tmem + k * 8, v_lo + k * (2048 >> 4), hi_v, idesc_pv, 1u);
+          } else {
+            if (k == 0) mma_ts_elect<false>(d_tmem, p_tmem, v_lo, hi_v, idesc_pv, acc ? 1u : 0u);
+            else        mma_ts_elect<true>(d_tmem, p_tmem + k * 8, v_lo + k * (2048 >> 4), hi_v, idesc_pv, 1u);
+          }
         }
       };
       // consumer position in the K/V ring
@@ -493,15 +556,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       auto advance = [&]() { if (++st == (uint32_t)L::kStages) { st = 0; ph ^= 1u; } };
 
       if (n_proc > 0) {
-        ok = mbar_wait_warp(bar_q_full, 0, limit) && mbar_wait_warp(bar_kv_full(st), ph, limit);
+        ok = wait_full(bar_q_full, 0) && wait_full(bar_kv_full(st), ph);
         if (ok) {
           tc_fence_after();
           issue_qk(tS0, q_lo0, st);
-          tc_commit_elect(bar_s_full(0));
+          commit(bar_s_full(0));
           issue_qk(tS1, q_lo1, st);
-          // (test hook: CTA 0 withholds this signal so that the waits downstream run into their limit)
-          if (!(p.fault_inject == 1u && cta == 0)) tc_commit_elect(bar_s_full(1));
-          tc_commit_elect(bar_kv_empty(st));
+          // (test hook: work item 0 withholds this signal so that the waits downstream run into their limit)
+          if (!(p.fault_inject == 1u && unit == 0)) commit(bar_s_full(1));
+          commit(bar_kv_empty(st));
           advance();
         }
         for (int i = 0; i < n_proc && ok; ++i) {
@@ -510,45 +573,46 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const bool more = i + 1 < n_proc;
           const uint32_t k_st = st, k_ph = ph;
           if (more) advance();
-          if (!mbar_wait_warp(bar_kv_full(v_st), v_ph, limit)) { ok = false; break; }
-          if (!mbar_wait_warp(bar_p_full(0), i & 1, limit)) { ok = false; break; }
+          if (!wait_full(bar_kv_full(v_st), v_ph)) { ok = false; break; }
+          if (!wait_full(bar_p_full(0), i & 1)) { ok = false; break; }
           tc_fence_after();
           issue_pv(tO0, tS0, v_st, i > 0);
-          tc_commit_elect(bar_o_done(0));
+          commit(bar_o_done(0));
           if (more) {
-            if (!mbar_wait_warp(bar_kv_full(k_st), k_ph, limit)) { ok = false; break; }
+            if (!wait_full(bar_kv_full(k_st), k_ph)) { ok = false; break; }
             tc_fence_after();
             issue_qk(tS0, q_lo0, k_st);
-            tc_commit_elect(bar_s_full(0));
+            commit(bar_s_full(0));
           }
-          if (!mbar_wait_warp(bar_p_full(1), i & 1, limit)) { ok = false; break; }
+          if (!wait_full(bar_p_full(1), i & 1)) { ok = false; break; }
           tc_fence_after();
           issue_pv(tO1, tS1, v_st, i > 0);
-          tc_commit_elect(bar_o_done(1));
-          tc_commit_elect(bar_kv_empty(v_st));
+          commit(bar_o_done(1));
+          commit(bar_kv_empty(v_st));
           if (more) {
             issue_qk(tS1, q_lo1, k_st);
-            tc_commit_elect(bar_s_full(1));
-            tc_commit_elect(bar_kv_empty(k_st));
+            commit(bar_s_full(1));
+            commit(bar_kv_empty(k_st));
           }
         }
       }
       if (!ok) {
         if (lane == 0) atomicCAS(p.status, 0u, kStatusTimeoutMma);
-        // tensor-core work already issued must finish before tensor memory is released
-        tc_commit_elect(bar_drain);
+        // tensor-core work already issued must finish before tensor memory is released (in both CTAs of a pair:
+        // the other one learns of it at the cluster barrier below)
+        commit(bar_drain);
         mbar_wait_warp(bar_drain, 0, limit);
       }
     }
     __syncwarp();
   }
 
-  // ---- teardown: everyone is done with tensor memory before it is released
+  // ---- teardown: everyone (of both CTAs) is done with tensor memory and shared memory before they are released
   tc_fence_before();
-  __syncthreads();
+  if (kPair) cluster_sync_all(); else __syncthreads();
   if (warp == 9) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    if (kPair) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
   }
 }
 

@@ -16,7 +16,7 @@ struct SeqDev {
   int ktile_start;      // offset of this sequence in keybits / ktile_list
   int seq_id;           // index in the caller's order
   int pair_start;       // index of this sequence's first query pair in per-pair arrays
-  int pad1;
+  int quad_work_start;  // first work item of this sequence when CTA pairs serve 512-row query blocks (head-major)
   long long sparse_list_start;  // block-sparse mode: offset of this sequence's per-CTA key-tile lists
 };
 

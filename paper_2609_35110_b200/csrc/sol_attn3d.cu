@@ -44,6 +44,8 @@ struct sol_attn3d_plan_s {
   std::vector<SeqDev> sched;          // schedule order (longest first)
   long long total_tokens = 0;
   int total_work = 0;
+  int total_quad_work = 0;            // work items when CTA pairs serve 512-row query blocks
+  int pair_mode = 0;                  // 1: use CTA pairs (cta_group::2) where they apply: head_dim 128, not block-sparse
   int total_ktiles = 0;
   std::vector<float2> tables;
   int tab_off[3] = {0, 0, 0};
@@ -59,6 +61,7 @@ struct sol_attn3d_plan_s {
 
   EncodeTiledFn encode = nullptr;
   CUtensorMap tm_q{}, tm_k{}, tm_v{};
+  CUtensorMap tm_k64{};               // K~ with 64-token boxes: what one CTA of a pair loads of a key tile
   const void* v_cached = nullptr;
   int keybits_state = 0;              // 0 unknown, 1 built for "no mask", 2 built from a mask
   int last_cuda = 0;
@@ -97,6 +100,19 @@ void release_host_pipe(sol_attn3d_plan_t p) {
   p->s_h2d = p->s_d2h = nullptr;
   p->ev_start = p->ev_done = nullptr;
   p->host_pipe_ready = false;
+}
+
+// The attention kernels use more dynamic shared memory than the default limit (per device, idempotent).
+cudaError_t raise_shared_memory_limits() {
+  cudaError_t e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       sol::AttnSmem<128, 1>::kDynBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(sol::attn_fwd_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             sol::AttnSmem<64, 1>::kDynBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             sol::AttnSmem<128, 2>::kDynBytes);
+  return e;
 }
 
 bool stride_ok(long long s) { return s > 0 && (s * 2) % 16 == 0 && (s * 2) < (1ll << 40); }
@@ -175,10 +191,13 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     // so that CTAs running together stream the same head's K/V through L2
     std::stable_sort(seqs.begin(), seqs.end(), [](const SeqDev& a, const SeqDev& b) { return a.n_tokens > b.n_tokens; });
     long long work = 0;
+    long long quad_work = 0;
     long long ktiles = 0;
     long long pairs = 0;
     for (SeqDev& q : seqs) {
       q.work_start = (int)work;
+      q.quad_work_start = (int)quad_work;
+      quad_work += (long long)((q.n_qpairs + 1) / 2) * d->heads;
       q.ktile_start = (int)ktiles;
       q.pair_start = (int)pairs;
       pairs += q.n_qpairs;
@@ -212,6 +231,7 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     }
     p->sched = seqs;
     p->total_work = (int)work;
+    p->total_quad_work = (int)quad_work;
     p->total_ktiles = (int)ktiles;
     p->total_pairs = (int)pairs;
 
@@ -252,6 +272,9 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     }
     // Test hook for the failure-detection path: a wait inside the kernel is made to run out on purpose.
     if (const char* e = std::getenv("SOL_ATTN3D_FAULT_INJECT")) p->fault_inject = (unsigned)std::atol(e);
+    // SOL_ATTN3D_PAIR=1: CTA pairs share every K / V tile (one tcgen05.mma.cta_group::2 over 256 query rows).  Off by
+    // default: it lowers power and L2 traffic but lengthens the per-tile dependency chain, and measured slower.
+    if (const char* e = std::getenv("SOL_ATTN3D_PAIR")) p->pair_mode = std::atol(e) != 0;
     p->v_lbo = p->head_dim == 128 ? 16384u : 16u;
     p->v_sbo = 1024u;
   } catch (const std::bad_alloc&) {
@@ -263,10 +286,10 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
 }
 
 // [tokens][heads][D] bf16 tensor as a 3-D TMA map with 128 x 64-element boxes, 128-byte swizzle.
-int encode_map(EncodeTiledFn fn, sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides st) {
+int encode_map(EncodeTiledFn fn, sol_attn3d_plan_t p, CUtensorMap* tm, const void* base, Strides st, unsigned box_tokens = 128) {
   const cuuint64_t dims[3] = {(cuuint64_t)p->head_dim, (cuuint64_t)p->heads, (cuuint64_t)p->total_tokens};
   const cuuint64_t strides[2] = {(cuuint64_t)st.head * 2, (cuuint64_t)st.tok * 2};
-  const cuuint32_t box[3] = {64, 1, 128};
+  const cuuint32_t box[3] = {64, 1, box_tokens};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -381,12 +404,7 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t p, void* device_ptr, size_t bytes
     if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return SOL_ATTN3D_ERR_CUDA;   // driver too old for TMA
     p->encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                sol::AttnSmem<128>::kDynBytes)) != cudaSuccess)
-    return fail_cuda(p, e);
-  if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                sol::AttnSmem<64>::kDynBytes)) != cudaSuccess)
-    return fail_cuda(p, e);
+  if ((e = raise_shared_memory_limits()) != cudaSuccess) return fail_cuda(p, e);
 
   p->ws = static_cast<unsigned char*>(device_ptr);
   p->keybits_state = 0;
@@ -401,6 +419,7 @@ int sol_attn3d_set_workspace(sol_attn3d_plan_t p, void* device_ptr, size_t bytes
   const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
   int rc = encode_map(p->encode, p, &p->tm_q, p->ws + p->off_qrot, dense);
   if (rc == SOL_ATTN3D_OK) rc = encode_map(p->encode, p, &p->tm_k, p->ws + p->off_krot, dense);
+  if (rc == SOL_ATTN3D_OK) rc = encode_map(p->encode, p, &p->tm_k64, p->ws + p->off_krot, dense, 64);
   return rc;
 }
 
@@ -855,8 +874,10 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   }
 
   // (3) attention.  Tensor maps: the plan's cached ones for its own workspace, per-call ones otherwise.
+  // CTA pairs (two CTAs share every K / V tile) wherever they apply
+  const bool pair = p->pair_mode != 0 && p->head_dim == 128 && sparse_ws == nullptr;
   CUtensorMap tm_q_call, tm_k_call, tm_v_call;
-  const CUtensorMap *tm_q = &p->tm_q, *tm_k = &p->tm_k, *tm_v = &p->tm_v;
+  const CUtensorMap *tm_q = &p->tm_q, *tm_k = pair ? &p->tm_k64 : &p->tm_k, *tm_v = &p->tm_v;
   if (own) {
     if (p->v_cached != v) {
       rc = encode_map(encode, p, &p->tm_v, v, p->sv);
@@ -866,7 +887,7 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   } else {
     const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
     if ((rc = encode_map(encode, p, &tm_q_call, ws + p->off_qrot, dense)) != SOL_ATTN3D_OK) return rc;
-    if ((rc = encode_map(encode, p, &tm_k_call, ws + p->off_krot, dense)) != SOL_ATTN3D_OK) return rc;
+    if ((rc = encode_map(encode, p, &tm_k_call, ws + p->off_krot, dense, pair ? 64 : 128)) != SOL_ATTN3D_OK) return rc;
     if ((rc = encode_map(encode, p, &tm_v_call, v, p->sv)) != SOL_ATTN3D_OK) return rc;
     tm_q = &tm_q_call; tm_k = &tm_k_call; tm_v = &tm_v_call;
   }
@@ -896,16 +917,32 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.wave_ctas = o.sm_count > 0 ? o.sm_count : p->sm_count;
   // one sequence: the CTAs of a head range are a contiguous range of work items; several sequences: launch
   // everything and let the CTAs of other heads leave at the door
-  int grid = p->total_work;
+  int units = pair ? p->total_quad_work : p->total_work;
   ap.cta_offset = 0;
   if (p->n_seqs == 1) {
-    ap.cta_offset = head_begin * p->sched[0].n_qpairs;
-    grid = (head_end - head_begin) * p->sched[0].n_qpairs;
+    const int per_head = pair ? (p->sched[0].n_qpairs + 1) / 2 : p->sched[0].n_qpairs;
+    ap.cta_offset = head_begin * per_head;
+    units = (head_end - head_begin) * per_head;
   }
-  if (p->head_dim == 128) {
-    sol::attn_fwd_kernel<128><<<grid, sol::kAttnThreads, sol::AttnSmem<128>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
+  if (pair) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)units * 2u, 1, 1);
+    cfg.blockDim = dim3(sol::kAttnThreads, 1, 1);
+    cfg.dynamicSmemBytes = sol::AttnSmem<128, 2>::kDynBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, sol::attn_fwd_kernel<128, 2>, *tm_q, *tm_k, *tm_v, ap);
+    if (e != cudaSuccess) return fail_cuda(p, e);
+  } else if (p->head_dim == 128) {
+    sol::attn_fwd_kernel<128, 1><<<units, sol::kAttnThreads, sol::AttnSmem<128, 1>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
   } else {
-    sol::attn_fwd_kernel<64><<<grid, sol::kAttnThreads, sol::AttnSmem<64>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
+    sol::attn_fwd_kernel<64, 1><<<units, sol::kAttnThreads, sol::AttnSmem<64, 1>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
   ++p->launches;
@@ -987,12 +1024,7 @@ int static_scratch_for_current_device(sol_attn3d_plan_t p, unsigned char** out, 
     if ((e = cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), sol_attn3d_static_scratch)) != cudaSuccess)
       return fail_cuda(p, e);
     if (addr == nullptr || (reinterpret_cast<uintptr_t>(addr) % kAlign) != 0) return SOL_ATTN3D_ERR_NO_WORKSPACE;
-    if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  sol::AttnSmem<128>::kDynBytes)) != cudaSuccess)
-      return fail_cuda(p, e);
-    if ((e = cudaFuncSetAttribute(sol::attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  sol::AttnSmem<64>::kDynBytes)) != cudaSuccess)
-      return fail_cuda(p, e);
+    if ((e = raise_shared_memory_limits()) != cudaSuccess) return fail_cuda(p, e);
     if (g_static_encode == nullptr) {
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
