@@ -520,9 +520,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128;
       const uint32_t tO0 = tmem_base + 256, tO1 = tmem_base + 256 + D;
       auto commit = [&](uint32_t bar) { if (kPair) tc_commit_elect_pair(bar); else tc_commit_elect(bar); };
-      auto wait_full = [&](uint32_t bar, uint32_t parity) {
-        return kPair ? mbar_wait_cluster_warp(bar, parity, limit) : mbar_wait_warp(bar, parity, limit);
-      };
+      auto wait_full = [&](uint32_t bar, uint32_t parity) { return mbar_wait_warp(bar, parity, limit); };
       auto issue_qk = [&](uint32_t d_tmem, uint32_t q_lo, uint32_t stage) {
         const uint32_t k_lo = k_lo_base + stage * kStageStep;
 #pragma unroll

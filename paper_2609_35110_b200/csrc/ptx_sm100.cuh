@@ -355,33 +355,11 @@ __device__ __forceinline__ uint32_t ld_shared_cluster_u32(uint32_t cluster_addr)
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// arrive on an mbarrier that may live in another CTA of the cluster (address from mapa_shared)
+// Arrive on an mbarrier that may live in another CTA of the cluster (address from mapa_shared).  What is handed
+// over lives in tensor memory and is ordered by tcgen05.wait::st / tcgen05.fence, so the arrival itself carries the
+// default semantics; a release at cluster scope here cost the arriving warp about a thousand cycles per call.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-// try_wait whose acquire covers arrivals from the other CTA of the cluster
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"((uint32_t)SOL_TRYWAIT_HINT_NS)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
-  if (mbar_try_wait_cluster(bar, parity)) return true;
-  const uint64_t t0 = globaltimer_ns();
-  uint32_t spins = 0;
-  while (!mbar_try_wait_cluster(bar, parity)) {
-    if ((++spins & 0x3ffu) == 0 && globaltimer_ns() - t0 > limit_ns) return false;
-  }
-  return true;
-}
-__device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
-  return __all_sync(0xffffffffu, mbar_wait_cluster(bar, parity, limit_ns));
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 // TMA load of a CTA pair: the data lands in this CTA's shared memory, the completion bytes are counted on an
 // mbarrier that may belong to the other CTA of the pair (the leader's).  Not a multicast.
