@@ -1,9 +1,11 @@
-// Attention main kernel, "pipelined" form: ONE 128-row query tile per CTA and THREE score buffers in tensor memory.
+// Attention main kernel, "pipelined" form: ONE 128-row query tile per CTA, two score buffers and two P buffers in
+// tensor memory.
 //
-// The two-tile kernel (attn_fwd_sm100.cuh) keeps one score buffer per query tile, so the QK^T of a tile's next key
-// block can only start after the softmax of the current one has finished and its P has been consumed: every key
-// block pays the whole chain  S -> softmax -> P -> PV -> QK  in sequence.  Here the tensor core runs ahead instead:
-// S(j+1) and S(j+2) are computed while the softmax works on S(j), so the softmax warps never wait for the tensor core
+// The two-tile kernel (attn_fwd_sm100.cuh) keeps one score buffer per query tile and writes P over it, so the QK^T
+// of a tile's next key block can only start after the softmax of the current one has finished and its P has been
+// consumed: every key block pays the whole chain  S -> softmax -> P -> PV -> QK  in sequence.  Here P has buffers of
+// its own, so a score buffer is free again as soon as the softmax has read it into registers: the tensor core
+// computes S(j+2) while the softmax works on S(j) and S(j+1), the softmax warps do not wait for the tensor core
 // and the hand-over latencies are off the critical path.  The price is that a K / V tile serves 128 query rows
 // instead of 256; CTA pairs (kCtas = 2) buy that back: the two CTAs of a cluster take the two 128-row tiles of a
 // 256-row query block, each loads HALF of every K / V tile, and one tcgen05.mma.cta_group::2 of M = 256 works on
@@ -12,13 +14,24 @@
 // Work item = (sequence, head, 256-row query block), exactly as in the two-tile kernel; CTA 2u and 2u+1 of the
 // grid take its two tiles (as a cluster when kCtas = 2, independently otherwise).
 //
-// Warp roles (256 threads):
-//   warps 0-3  softmax / correction / epilogue (thread = one query row)
-//   warp  4    TMA producer (lane 0)
-//   warp  5    tcgen05.mma issuer (whole warp convergent, one elected lane issues); owns the TMEM allocation
-//   warps 6-7  idle
-// Tensor memory (512 columns): S0 | S1 | S2 (128 columns each, P of a block overwrites the first 64 columns of its
-// S) | O (D columns).
+// Warp roles (384 threads):
+//   warps 0-3  softmax of the EVEN key blocks of the tile (thread = one query row), and the epilogue
+//   warps 4-7  softmax of the ODD key blocks (warp w + 4 owns the same 32 rows as warp w and sits on the same
+//              scheduler: while one of the two waits for tensor memory or a barrier, the other keeps the
+//              special-function unit busy)
+//   warp  8    TMA producer (lane 0)
+//   warp  9    tcgen05.mma issuer (whole warp convergent, one elected lane issues); owns the TMEM allocation
+//   warps 10-11 idle (complete the third warpgroup)
+// Tensor memory (512 columns): S0 | S1 (128 columns each, fp32) | P0 | P1 (64 columns each, bf16 pairs) | O (D
+// columns).  Key block i uses S[i % 2] and P[i % 2].
+//
+// Online softmax over two warpgroups.  Both exponentiate against a per-row reference maximum that only ever grows
+// (lazily: by more than 2^8 or not at all, see the two-tile kernel).  The key blocks are FINALISED in order: the
+// warp that owns block i hands its P over only after its partner has finalised block i-1 and published the
+// reference it ended with.  If that reference differs from the one block i was exponentiated against (rare), the
+// block is redone from the scores still in registers; if block i itself needs a larger reference (rare), its
+// owner rescales O (after PV(i-1)) and publishes the new one.  Each warpgroup keeps the row sum of its own blocks;
+// the two are brought to the final reference and added in the epilogue.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -44,8 +57,8 @@ namespace sol {
 #define SOL_PROF_OUT(idx, v)
 #endif
 
-constexpr int kPipeThreads = 256;
-constexpr int kPipeBufs = 3;
+constexpr int kPipeThreads = 384;
+constexpr int kPipeBufs = 2;
 
 template <int D, int kCtas>
 struct PipeSmem {
@@ -58,9 +71,12 @@ struct PipeSmem {
   static constexpr int kOffQ = 0;
   static constexpr int kOffKV = kTile;
   static constexpr int kOffBars = kOffKV + kStages * kStageBytes;
-  static constexpr int kNumBars = 1 + 2 * kStages + 3 * kPipeBufs + 1;   // q_full, kv_full/empty, s_full[3], p_full[3], o_done[3], drain
+  // q_full, kv_full/empty, s_full[2], p_full[2], o_done[2], s_free[2], drain, fin[4 row groups][2 warpgroups]
+  static constexpr int kNumBars = 1 + 2 * kStages + 4 * kPipeBufs + 1 + 8;
   static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
-  static constexpr int kBytes = kOffTmemPtr + 16;
+  static constexpr int kOffRef = kOffTmemPtr + 16;        // float[128]: reference maximum per row as of the last finalised block
+  static constexpr int kOffSum = kOffRef + 128 * 4;       // float2[128]: (row sum, its reference) of the odd-block warpgroup
+  static constexpr int kBytes = kOffSum + 128 * 8;
   static constexpr int kDynBytes = kBytes + 1024;         // slack to align the base to 1024 bytes
 };
 
@@ -92,10 +108,17 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   auto bar_kv_empty = [&](int s) { return bars + 8u * (1 + L::kStages + s); };
   auto bar_s_full = [&](int b) { return bars + 8u * (1 + 2 * L::kStages + b); };
   auto bar_p_full = [&](int b) { return bars + 8u * (1 + 2 * L::kStages + kPipeBufs + b); };
-  // "PV of a key block in buffer b has completed".  One barrier per buffer, not one for all: a waiter may be up to
-  // three PVs behind the tensor core, and an mbarrier phase can only be told from its neighbour.
+  // "PV of a key block that used P buffer b has completed" (P[b] may be overwritten, O holds that block).  One
+  // barrier per buffer, not one for all: a waiter may be two PVs behind the tensor core, and an mbarrier phase can
+  // only be told from its neighbour.
   auto bar_o_done = [&](int b) { return bars + 8u * (1 + 2 * L::kStages + 2 * kPipeBufs + b); };
-  const uint32_t bar_drain = bars + 8u * (1 + 2 * L::kStages + 3 * kPipeBufs);
+  // "the softmax has read S[b] into registers": the tensor core may overwrite it
+  auto bar_s_free = [&](int b) { return bars + 8u * (1 + 2 * L::kStages + 3 * kPipeBufs + b); };
+  const uint32_t bar_drain = bars + 8u * (1 + 2 * L::kStages + 4 * kPipeBufs);
+  // "warp (g, q) has finalised its latest key block": waited on by its partner warp (1 - g, q)
+  auto bar_fin = [&](int q, int g) { return bars + 8u * (2 + 2 * L::kStages + 4 * kPipeBufs + 2 * q + g); };
+  volatile float* ref_smem = reinterpret_cast<volatile float*>(smem + L::kOffRef);
+  volatile float* sum_smem = reinterpret_cast<volatile float*>(smem + L::kOffSum);   // [2 * row] sum, [2 * row + 1] its reference
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + L::kOffTmemPtr);
 
   // ---- which work item
@@ -127,7 +150,7 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   const int tok0 = (int)sq.tok_start;                   // TMA token coordinate of the sequence start
   const unsigned long long limit = p.wait_limit_ns;
 
-  if (warp == 4 && lane == 0) {
+  if (warp == 8 && lane == 0) {
     mbar_init(bar_q_full, 1);
     for (int s = 0; s < L::kStages; ++s) {
       mbar_init(bar_kv_full(s), 1);
@@ -135,10 +158,13 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     }
     for (int b = 0; b < kPipeBufs; ++b) {
       mbar_init(bar_s_full(b), 1);
-      mbar_init(bar_p_full(b), 4 * kCtas);              // one arrival per softmax warp, from every CTA of the pair
+      mbar_init(bar_p_full(b), 4 * kCtas);              // one arrival per softmax warp of the block, from every CTA of the pair
+      mbar_init(bar_s_free(b), 4 * kCtas);
       mbar_init(bar_o_done(b), 1);
     }
     mbar_init(bar_drain, 1);
+    for (int q = 0; q < 4; ++q)
+      for (int g = 0; g < 2; ++g) mbar_init(bar_fin(q, g), 1);
     fence_mbar_init();
     prefetch_tensormap(&tm_q);
     prefetch_tensormap(&tm_k);
@@ -146,7 +172,7 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   }
   // A fault recorded by an earlier CTA stops later ones at the door (read once; made uniform over the pair below).
   if (threadIdx.x == 0) tmem_ptr_smem[1] = *reinterpret_cast<volatile unsigned int*>(p.status);
-  if (warp == 5) {
+  if (warp == 9) {
     if (kPair) { tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 512); tmem_relinquish_pair(); }
     else       { tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 512); tmem_relinquish(); }
   }
@@ -162,32 +188,48 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       cluster_sync_all();
     }
     if (stop != 0) {
-      if (warp == 5) {
+      if (warp == 9) {
         if (kPair) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
       }
       return;
     }
   }
-  const uint32_t tO_base = tmem_base + kPipeBufs * 128;
+  const uint32_t tP_base = tmem_base + kPipeBufs * 128;   // P0 | P1, 64 columns each
+  const uint32_t tO_base = tP_base + kPipeBufs * 64;
 
-  if (warp < 4) {
+  if (warp < 8) {
     // =========================================================== softmax / correction / epilogue
-    const int row = warp * 32 + lane;
-    const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
+    setmaxnreg_inc<SOL_REGS_SOFTMAX>();
+    const int g = warp >> 2;                             // warpgroup: key blocks g, g + 2, g + 4, ...
+    const int q = warp & 3;                              // row group: rows 32 q .. 32 q + 31 (tensor-memory lanes)
+    const int row = q * 32 + lane;
+    const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
     const uint32_t tO = tO_base + lane_off;
     const float c = p.scale_log2;
     float m_ref = -CUDART_INF_F;
     float l = 0.f;
     bool ok = true;
-    int b = 0;                                           // score buffer of key block i: i % 3
-    uint32_t use = 0;                                    // how often that buffer has been used before: i / 3
-    long long prof_wait = 0;
+    long long prof_wait = 0, prof_a = 0, prof_b = 0, prof_c = 0, prof_d = 0, prof_e = 0;
     SOL_PROF_T(prof_t0);
 
-    for (int i = 0; i < n_proc; ++i) {
-      const int jt = tile_at(i);
-      const uint4 kb = __ldg(&keybits[jt]);
+    // Validity bits of this warpgroup's blocks are fetched one block ahead and their tile numbers two blocks ahead,
+    // so that neither load (the second depends on the first) is waited for inside a block.
+    uint4 kb_next = g < n_proc ? __ldg(&keybits[tile_at(g)]) : make_uint4(0u, 0u, 0u, 0u);
+    int jt_next = g + 2 < n_proc ? tile_at(g + 2) : 0;
+    for (int i = g; i < n_proc; i += 2) {
+      const int b = i % kPipeBufs;                       // score buffer of key block i
+      const uint32_t use = (uint32_t)(i / kPipeBufs);    // how often that buffer has been used before
+      const uint4 kb = kb_next;
+      if (i + 2 < n_proc) kb_next = __ldg(&keybits[jt_next]);
+      if (i + 4 < n_proc) jt_next = tile_at(i + 4);
       const uint32_t tS = tmem_base + lane_off + b * 128;
+      const uint32_t tP = tP_base + lane_off + b * 64;
+      if (i == 1) {
+        // the odd warpgroup's first block: exponentiate against the reference that block 0 ended with
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_fin(q, 0), 0u, limit));
+        if (!ok) break;
+        m_ref = ref_smem[row];
+      }
       SOL_PROF_T(prof_w0);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full(b), use & 1u, limit));
       SOL_PROF_ADD(prof_wait, prof_w0);
@@ -199,28 +241,39 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       uint32_t pk[64];
       float tile_sum;
       bool first_half_stored = false;
+      SOL_PROF_T(prof_s1);
+      // the whole row of scores into registers, then S[b] goes back to the tensor core at once: S(i+2) is computed
+      // while this block is exponentiated (the partner warp on this scheduler covers the load latency)
+#pragma unroll
+      for (int cch = 0; cch < 4; ++cch) tmem_ld32(tS + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[cch * 32]));
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (kPair) mbar_arrive_cluster(mapa_shared(bar_s_free(b), 0)); else mbar_arrive(bar_s_free(b));
+      }
+      SOL_PROF_ADD(prof_a, prof_s1);
+      // P[b] still feeds PV(i-2) until that has completed: checked right before the first store into it
+      auto p_buffer_free = [&]() {
+        return i < 2 || __all_sync(0xffffffffu, mbar_wait(bar_o_done(b), (uint32_t)((i - 2) >> 1) & 1u, limit));
+      };
+      SOL_PROF_T(prof_s3);
       if (!mixed && i > 0) {
-        // Common case, in two halves: the second half of S is still on its way while the first is exponentiated, and
-        // the first half of P is on its way to tensor memory while the second is.
+        // Common case, in two halves: the first half of P is on its way to tensor memory while the second is computed
         uint32_t (&r_lo)[64] = *reinterpret_cast<uint32_t(*)[64]>(&r[0]);
         uint32_t (&r_hi)[64] = *reinterpret_cast<uint32_t(*)[64]>(&r[64]);
-        tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-        tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-        tmem_wait_ld_dep64(r_lo);
-        tmem_ld32(tS + 64, *reinterpret_cast<uint32_t(*)[32]>(&r[64]));
-        tmem_ld32(tS + 96, *reinterpret_cast<uint32_t(*)[32]>(&r[96]));
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         const float mc = m_ref * c;
         softmax_half(r_lo, c, mc, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]), acc);
-        tmem_wait_ld_dep64(r_hi);
-        tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));       // columns [0,32): their scores are in registers
+        SOL_PROF_T(prof_s2);
+        ok = p_buffer_free();
+        SOL_PROF_ADD(prof_b, prof_s2);
+        if (!ok) break;
+        tmem_st32(tP, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
         first_half_stored = true;
         softmax_half(r_hi, c, mc, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]), acc);
         tile_sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
       } else {
-#pragma unroll
-        for (int cch = 0; cch < 4; ++cch) tmem_ld32(tS + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[cch * 32]));
-        tmem_wait_ld();
         if (mixed) {
           // masked or out-of-range keys get -inf
 #pragma unroll
@@ -232,11 +285,30 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         if (i == 0) m_ref = row_max128(r);
         if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
         else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum);
+        ok = p_buffer_free();
+        if (!ok) break;
       }
-      // Lazy reference: the pass ran against the current reference maximum.  All terms are positive, so a row sum
+      SOL_PROF_ADD(prof_c, prof_s3);
+
+      // ---- finalise block i, in block order.  (1) The partner has finalised block i-1: adopt its reference.
+      if (i > 0) {
+        SOL_PROF_T(prof_s4);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_fin(q, 1 - g), (uint32_t)((i - 1) >> 1) & 1u, limit));
+        SOL_PROF_ADD(prof_d, prof_s4);
+        if (!ok) break;
+        const float r_prev = ref_smem[row];
+        const bool moved = r_prev != m_ref;              // it can only have grown
+        if (__any_sync(0xffffffffu, moved)) {
+          if (moved) { l *= ex2_approx((m_ref - r_prev) * c); m_ref = r_prev; }
+          softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
+          if (first_half_stored) tmem_wait_st();                         // the stale first half lands before its replacement
+          first_half_stored = false;
+        }
+      }
+      // (2) Lazy reference: the pass ran against the current reference.  All terms are positive, so a row sum
       // <= 2^8 proves every term <= 2^8 and the reference still good.  Otherwise the row maximum is taken; if it
-      // grew by more than 2^8 (exp2 domain) the reference moves, l and O are rescaled and the tile is redone from
-      // the scores still held in registers, before any of its P is released.  Rare.
+      // grew by more than 2^8 (exp2 domain) the reference moves, l and O are rescaled and the block is redone.
+      bool published = i == 0;
       if (__any_sync(0xffffffffu, !(tile_sum <= 256.0f))) {
         const float mx = row_max128(r);
         const bool grow = (mx - m_ref) * c > 8.0f;
@@ -246,10 +318,8 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           if (grow) m_ref = mx;
           l *= f;
           // O holds the sum over key blocks 0 .. i-1 once PV(i-1) has completed (PV(i) cannot start before this P).
-          // PV(i-4), the previous user of that buffer's barrier, completed before S(i) was even started.
-          const int bp = b == 0 ? kPipeBufs - 1 : b - 1;
-          const uint32_t up = b == 0 ? use - 1u : use;
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done(bp), up & 1u, limit));
+          // PV(i-3), the previous user of that barrier, completed before the partner stored P(i-1).
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done((i - 1) % kPipeBufs), (uint32_t)((i - 1) / kPipeBufs) & 1u, limit));
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
@@ -262,51 +332,72 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             tmem_st32(tO + cch * 32, o);
           }
           softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
-          if (first_half_stored) tmem_wait_st();                         // the stale first half lands before its replacement
+          if (first_half_stored) tmem_wait_st();
           first_half_stored = false;
+          published = true;
         }
       }
+      // (3) publish the reference this block ended with (only when it changed), then hand P over
+      if (published) ref_smem[row] = m_ref;
       l += tile_sum;
-      if (!first_half_stored) tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-      tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+      SOL_PROF_T(prof_s5);
+      if (!first_half_stored) tmem_st32(tP, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      tmem_st32(tP + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
-      // one arrival per warp, on the leader's barrier (the MMA over both CTAs' rows starts when all have come)
+      // one arrival per warp: on the leader's barrier for P (the MMA over both CTAs' rows starts when all have
+      // come), and on this warp's own "finalised" barrier for the partner
       __syncwarp();
       if (lane == 0) {
         if (kPair) mbar_arrive_cluster(mapa_shared(bar_p_full(b), 0)); else mbar_arrive(bar_p_full(b));
+        mbar_arrive(bar_fin(q, g));
       }
-      if (++b == kPipeBufs) { b = 0; ++use; }
+      SOL_PROF_ADD(prof_e, prof_s5);
     }
 #if SOL_PIPE_PROF
-    if (warp == 0 && lane == 0) { SOL_PROF_OUT(1, prof_wait); SOL_PROF_OUT(2, clock64() - prof_t0); SOL_PROF_OUT(9, 1); }
+    if (warp == 0 && lane == 0) {
+      SOL_PROF_OUT(1, prof_wait); SOL_PROF_OUT(2, clock64() - prof_t0); SOL_PROF_OUT(9, 1);
+      SOL_PROF_OUT(10, prof_a); SOL_PROF_OUT(11, prof_b); SOL_PROF_OUT(12, prof_c); SOL_PROF_OUT(13, prof_d); SOL_PROF_OUT(14, prof_e);
+    }
 #endif
-    (void)prof_wait;
+    (void)prof_wait; (void)prof_a; (void)prof_b; (void)prof_c; (void)prof_d; (void)prof_e;
 
-    // ---- epilogue: O / l in the output format, staged through shared memory, coalesced 16-byte stores
-    if (ok && n_proc > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done((n_proc - 1) % kPipeBufs), (uint32_t)((n_proc - 1) / kPipeBufs) & 1u, limit));
-      if (ok) tc_fence_after();
-    }
-    if (ok && n_proc > 0) {
-      const float inv = 1.0f / l;
-      uint8_t* stage = smem + L::kOffQ + warp * 32 * (D * 2);
-      if (p.sink.fmt == kOutE4M3) store_rows<D, true>(p, sq, head, q_row0 + warp * 32, lane, tO, inv, stage);
-      else                        store_rows<D, false>(p, sq, head, q_row0 + warp * 32, lane, tO, inv, stage);
-    } else if (ok) {
-      // no key tile at all (every key of the sequence masked): the row is defined as zero
-      const int qrow = q_row0 + row;
-      bool store = qrow < sq.n_tokens;
-      if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
-      if (store) {
-        const int row_bytes = p.sink.fmt == kOutE4M3 ? D : D * 2;
-        uint8_t* dst = out_row_ptr(p, sq.tok_start + qrow, head, row_bytes / D);
-        for (int c16 = 0; c16 < row_bytes / 16; ++c16) *reinterpret_cast<uint4*>(dst + c16 * 16) = make_uint4(0u, 0u, 0u, 0u);
+    // ---- the two warpgroups' row sums meet: the odd one leaves (sum, reference), the even one does the epilogue
+    if (g == 1) { sum_smem[2 * row] = l; sum_smem[2 * row + 1] = m_ref; }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (g == 0) {
+      // ---- epilogue: O / l in the output format, staged through shared memory, coalesced 16-byte stores
+      if (ok && n_proc > 0) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_o_done((n_proc - 1) % kPipeBufs), (uint32_t)((n_proc - 1) / kPipeBufs) & 1u, limit));
+        if (ok) tc_fence_after();
       }
-    } else if (lane == 0) {
-      atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);
+      if (ok && n_proc > 0) {
+        // both sums at the reference O ended with: that of the last block's owner
+        const float lo = sum_smem[2 * row], mo = sum_smem[2 * row + 1];
+        const float m_fin = fmaxf(m_ref, mo);            // references only grow: the later one is the larger one
+        float l_tot = l * ex2_approx((m_ref - m_fin) * c);
+        if (n_proc > 1) l_tot += lo * ex2_approx((mo - m_fin) * c);
+        const float inv = 1.0f / l_tot;
+        uint8_t* stage = smem + L::kOffQ + q * 32 * (D * 2);
+        if (p.sink.fmt == kOutE4M3) store_rows<D, true>(p, sq, head, q_row0 + q * 32, lane, tO, inv, stage);
+        else                        store_rows<D, false>(p, sq, head, q_row0 + q * 32, lane, tO, inv, stage);
+      } else if (ok) {
+        // no key tile at all (every key of the sequence masked): the row is defined as zero
+        const int qrow = q_row0 + row;
+        bool store = qrow < sq.n_tokens;
+        if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
+        if (store) {
+          const int row_bytes = p.sink.fmt == kOutE4M3 ? D : D * 2;
+          uint8_t* dst = out_row_ptr(p, sq.tok_start + qrow, head, row_bytes / D);
+          for (int c16 = 0; c16 < row_bytes / 16; ++c16) *reinterpret_cast<uint4*>(dst + c16 * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
     }
-  } else if (warp == 4) {
+    if (!ok && lane == 0) atomicCAS(p.status, 0u, kStatusTimeoutSoftmax);
+  } else {
+    setmaxnreg_dec<SOL_REGS_OTHER>();
+  }
+  if (warp == 8) {
     // =========================================================== TMA producer
     if (lane == 0) {
       bool ok = true;
@@ -352,12 +443,12 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         if (++stage == (uint32_t)L::kStages) { stage = 0; par ^= 1u; }
         return true;
       };
-      // in the order the MMA issuer consumes them: K(0), K(1), K(2), then V(i), K(i+3)
+      // in the order the MMA issuer consumes them: K(0), K(1), then K(i+2), V(i)
       const int pre = n_proc < kPipeBufs ? n_proc : kPipeBufs;
       for (int i = 0; i < pre && ok; ++i) ok = load(tile_at(i), false);
       for (int i = 0; i < n_proc && ok; ++i) {
-        ok = load(tile_at(i), true);
-        if (ok && i + kPipeBufs < n_proc) ok = load(tile_at(i + kPipeBufs), false);
+        if (i + kPipeBufs < n_proc) ok = load(tile_at(i + kPipeBufs), false);
+        if (ok) ok = load(tile_at(i), true);
       }
 #if SOL_PIPE_PROF
       SOL_PROF_OUT(7, prof_wait); SOL_PROF_OUT(8, clock64() - prof_t0);
@@ -376,7 +467,7 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       }
     }
     __syncwarp();
-  } else if (warp == 5 && leader) {
+  } else if (warp == 9 && leader) {
     // =========================================================== MMA issuer
     // The whole warp runs this loop (convergent); one elected lane issues each tcgen05 instruction.
     constexpr uint32_t idesc_qk = idesc_bf16_f32(128 * kCtas, 128, false);
@@ -426,7 +517,7 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
     if (n_proc > 0) {
       ok = wait_full(bar_q_full, 0);
-      // fill the score pipeline: S(0), S(1), S(2)
+      // fill the score pipeline: S(0), S(1)
       const int pre = n_proc < kPipeBufs ? n_proc : kPipeBufs;
       for (int b = 0; b < pre && ok; ++b) {
         if (!wait_full(bar_kv_full(st), ph)) { ok = false; break; }
@@ -437,11 +528,24 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         commit(bar_kv_empty(st));
         advance();
       }
-      int b = 0;
-      uint32_t use = 0;
       long long prof_v = 0, prof_p = 0, prof_k = 0;
       SOL_PROF_T(prof_t0);
       for (int i = 0; i < n_proc && ok; ++i) {
+        const int b = i & 1;
+        const uint32_t use = (uint32_t)(i >> 1);
+        if (i + kPipeBufs < n_proc) {
+          // S(i+2) goes into S[b] as soon as the softmax has read S(i) out of it
+          const uint32_t k_st = st, k_ph = ph;
+          advance();
+          SOL_PROF_T(prof_w2);
+          if (!wait_full(bar_kv_full(k_st), k_ph)) { ok = false; break; }
+          if (!wait_full(bar_s_free(b), use & 1u)) { ok = false; break; }
+          SOL_PROF_ADD(prof_k, prof_w2);
+          tc_fence_after();
+          issue_qk(tmem_base + b * 128, k_st);
+          commit(bar_s_full(b));
+          commit(bar_kv_empty(k_st));
+        }
         const uint32_t v_st = st, v_ph = ph;
         advance();
         SOL_PROF_T(prof_w0);
@@ -451,23 +555,9 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         if (!wait_full(bar_p_full(b), use & 1u)) { ok = false; break; }
         SOL_PROF_ADD(prof_p, prof_w1);
         tc_fence_after();
-        issue_pv(tO_base, tmem_base + b * 128, v_st, i > 0);
+        issue_pv(tO_base, tP_base + b * 64, v_st, i > 0);
         commit(bar_o_done(b));
         commit(bar_kv_empty(v_st));
-        if (i + kPipeBufs < n_proc) {
-          // the buffer whose P has just been handed to the tensor core takes S(i+3); the MMAs execute in issue
-          // order, so QK(i+3) overwrites it only after PV(i) has read it
-          const uint32_t k_st = st, k_ph = ph;
-          advance();
-          SOL_PROF_T(prof_w2);
-          if (!wait_full(bar_kv_full(k_st), k_ph)) { ok = false; break; }
-          SOL_PROF_ADD(prof_k, prof_w2);
-          tc_fence_after();
-          issue_qk(tmem_base + b * 128, k_st);
-          commit(bar_s_full(b));
-          commit(bar_kv_empty(k_st));
-        }
-        if (++b == kPipeBufs) { b = 0; ++use; }
       }
 #if SOL_PIPE_PROF
       if (lane == 0) { SOL_PROF_OUT(3, prof_v); SOL_PROF_OUT(4, prof_p); SOL_PROF_OUT(5, prof_k); SOL_PROF_OUT(6, clock64() - prof_t0); }
@@ -487,7 +577,7 @@ attn_fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   // ---- teardown: everyone (of both CTAs) is done with tensor memory and shared memory before they are released
   tc_fence_before();
   if (kPair) cluster_sync_all(); else __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after();
     if (kPair) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
   }
