@@ -32,13 +32,25 @@ from paper_2609_35110_b200 import workloads as wl  # noqa: E402
 METRIC = "attention_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16 = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_kernel launch, from one-pass ncu captures of these
-# very workloads (two DRAM counters, one launch).
-NCU_TRAFFIC = {
-    "lowres": (787700000 + 238820000, "ncu capture of this workload (one pass, two DRAM counters)"),
-    "highres": (5650000000 + 1140000000, "ncu capture of this workload (one pass, two DRAM counters); the excess over the "
-                                         "algorithmic bytes is K/V re-reads that miss L2 between waves of CTAs"),
-}
+TRAFFIC_SUMMARY = os.path.join(ROOT, "profiles", "attn_fwd_kernel_dram_traffic.md")
+SM_COUNT = 148
+TENSOR_FLOP_PER_CLK_PER_SM = 8192       # dense bf16 on one SM's tensor core
+
+
+def load_ncu_traffic(workload):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, as recorded in the tracked ncu
+    summary of that capture (lines `traffic <workload>: dram_read_bytes=R dram_write_bytes=W`).  None if absent."""
+    try:
+        with open(TRAFFIC_SUMMARY) as f:
+            for line in f:
+                parts = line.strip().strip("`").split()
+                if len(parts) >= 4 and parts[0] == "traffic" and parts[1].rstrip(":") == workload:
+                    kv = dict(x.split("=", 1) for x in parts[2:] if "=" in x)
+                    return int(kv["dram_read_bytes"]) + int(kv["dram_write_bytes"]), \
+                        "ncu capture of this workload (one pass, two DRAM counters), profiles/attn_fwd_kernel_dram_traffic.md"
+    except (OSError, KeyError, ValueError):
+        pass
+    return None, None
 
 
 def load_peaks():
@@ -272,12 +284,13 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return 0
-        warm = max(3, args.warmup) if args.warmup > 0 else 0
         inp = wl.make_inputs(w, "cpu")
         heads_s, rows = cpu_sample_spec(w, scale=0.34)
         sel = oracle_sample(w, inp, heads_s, rows)
         fl = sample_flops(w, sel)
-        for _ in range(min(warm, 1)):                        # one untimed pass warms the allocator / BLAS threads
+        # the oracle has no state to warm beyond the allocator and the BLAS threads: one untimed pass over one group
+        warm_done = 1 if args.warmup > 0 else 0
+        for _ in range(warm_done):
             run_oracle(w, inp, sel[:1])
         times = []
         for _ in range(args.steps):
@@ -288,7 +301,8 @@ def main():
         sample = f"{len(sel)} (seq, head) groups x {len(sel[0][2])} query rows against all keys"
         print(json.dumps({
             "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "steps": args.steps, "warmup": warm_done, "warmup_note": "one untimed oracle pass over one (seq, head) group",
+            "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                              "sample": sample},
@@ -444,11 +458,44 @@ def main():
     achieved = flops / (attn_ms * 1e-3) / 1e12
     long_step = total_ms > 1000.0
     peak = peaks["sustained"] if long_step else peaks["burst"]
-    traffic, traffic_note = NCU_TRAFFIC.get(w.name, (None, None))
+    traffic, traffic_note = load_ncu_traffic(w.name)
+    # cycles of one attention launch at the SM clock sampled during the timed region: separates gains in the
+    # dependency chain (fewer cycles) from gains in power (more MHz under the cap)
+    sm_mhz = clocks.get("sm_mhz") if clocks else None
+    attn_mcycles = attn_ms * 1e-3 * sm_mhz if sm_mhz else None
+    per_clock = flops / (attn_mcycles * 1e6 * SM_COUNT * TENSOR_FLOP_PER_CLK_PER_SM) if attn_mcycles else None
 
     # ------------------------------------------------------------------ CPU baseline (oracle, bounded sample)
     cpu = None
     parity = None
+    if not args.no_cpu_baseline and world == 1 and args.sparse_tau is not None:
+        # block-sparse leg: the oracle on a few sampled (head, rows) groups, over the blocks the GPU selected
+        from oracle import attn3d_oracle as orc
+        seqs = [(s.text_len, s.T, s.H, s.W) for s in w.seqs]
+        q_cpu, k_cpu, v_cpu = inp.q.cpu(), inp.k.cpu(), inp.v.cpu()
+        mask_cpu = None if inp.key_mask is None else inp.key_mask.cpu()
+        select, picked = [], []
+        for h in sorted({0, w.heads // 2, w.heads - 1}):
+            sq0 = w.seqs[0]
+            nq, nk = (sq0.n_tokens + 255) // 256, (sq0.n_tokens + 127) // 128
+            m = torch.zeros(nq, nk, dtype=torch.bool)
+            for i in range(nq):
+                m[i, B.sol_attn3d_sparse_selection(attn.plan, sparse_ws, 0, h, i, nk)] = True
+            picked.append(m)
+            select.append((0, h, torch.from_numpy(wl.sample_rows(w, 0, h, 256))))
+        t0 = time.perf_counter()
+        ref, _, _ = orc.attn3d_sparse_oracle(q_cpu, k_cpu, v_cpu, seqs, w.rope_dims, w.theta, args.sparse_tau, 256, 128,
+                                             mask_cpu, selection=picked, select=select)
+        dt = time.perf_counter() - t0
+        o_cpu = out.cpu()
+        got = torch.cat([o_cpu[rows_, h] for (_, h, rows_) in select])
+        ma, rl = orc.compare(got, torch.cat(ref))
+        kept = sum(float(m.float().mean()) for m in picked) / len(picked)
+        fl = sum(4.0 * len(r_) * w.seqs[0].n_tokens * w.head_dim for (_, _, r_) in select) * kept
+        cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "seconds": dt,
+               "sample": f"{len(select)} heads x 256 query rows of sequence 0 over the KV blocks the GPU selected (fp64)"}
+        parity = {"max_abs": ma, "rel_l2": rl, "rows": int(got.shape[0]), "tol_max_abs": 2e-2, "tol_rel_l2": 5e-3,
+                  "ok": bool(ma <= 2e-2 and rl <= 5e-3), "selection": "the GPU's own, read back per (head, query block)"}
     if not args.no_cpu_baseline and world == 1 and args.sparse_tau is None:
         from oracle import attn3d_oracle as orc
         inp_cpu = wl.Inputs(inp.q.cpu(), inp.k.cpu(), inp.v.cpu(), None if inp.key_mask is None else inp.key_mask.cpu())
@@ -475,6 +522,7 @@ def main():
                              "measured_sustained_%.1f" % peaks["sustained"]: 100 * value / world / peaks["sustained"],
                              "nominal_%.0f" % NOMINAL_BF16: 100 * value / world / NOMINAL_BF16},
         "kernel_ms": {"keybits": bits_ms, "rope_prologue": rope_ms, "attention": attn_ms},
+        "attention_mcycles": attn_mcycles, "tensor_pipe_busy_per_clock": per_clock,
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_kind": ("sustained" if long_step else "burst") + " bf16, " + peaks["source"],
                      "kernel": "attn_fwd_kernel<%d>" % w.head_dim, "traffic": traffic, "traffic_note": traffic_note,

@@ -94,18 +94,23 @@ struct RopeArgs {
   int head_begin, head_end;   // heads [head_begin, head_end) are produced by this launch
 };
 
-__global__ void __launch_bounds__(256, 4) rope_qk_kernel(const RopeArgs a) {
+__global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
   const int chunks = a.g.head_dim >> 3;          // 16-byte chunks per head row (8 or 16: divides the warp)
   const int heads_per_pass = blockDim.x / chunks;
   const int chunk = threadIdx.x % chunks;
   const int hsub = threadIdx.x / chunks;
   const int d1 = a.g.rope[0], d2 = d1 + a.g.rope[1], d3 = d2 + a.g.rope[2];
   const float inv_d = 1.0f / (float)a.g.head_dim;
-  float gn[2][8];
+  // which table entry each of the thread's four pairs uses (fixed per thread: it depends on the chunk only)
+  int axis[4], tab[4], step[4];                 // step: table entries per position of that axis
 #pragma unroll
-  for (int which = 0; which < 2; ++which)
-#pragma unroll
-    for (int e = 0; e < 8; ++e) gn[which][e] = a.gain[which] ? __ldg(a.gain[which] + chunk * 8 + e) : 1.0f;
+  for (int u = 0; u < 4; ++u) {
+    const int d = chunk * 8 + 2 * u;             // first head dim of the pair
+    if (d < d1)      { axis[u] = 0; tab[u] = a.g.tab_off[0] + (d >> 1);        step[u] = a.g.rope[0] >> 1; }
+    else if (d < d2) { axis[u] = 1; tab[u] = a.g.tab_off[1] + ((d - d1) >> 1); step[u] = a.g.rope[1] >> 1; }
+    else if (d < d3) { axis[u] = 2; tab[u] = a.g.tab_off[2] + ((d - d2) >> 1); step[u] = a.g.rope[2] >> 1; }
+    else             { axis[u] = -1; tab[u] = 0; step[u] = 0; }
+  }
 
   for (long long tok = blockIdx.x; tok < a.total_tokens; tok += gridDim.x) {
     // which sequence, which grid position
@@ -113,46 +118,45 @@ __global__ void __launch_bounds__(256, 4) rope_qk_kernel(const RopeArgs a) {
     while (s + 1 < a.n_seqs && !(tok >= a.seqs[s].tok_start && tok < a.seqs[s].tok_start + a.seqs[s].n_tokens)) ++s;
     const SeqDev sq = a.seqs[s];
     const int local = (int)(tok - sq.tok_start);
-    float2 cs[4];
-    bool rotate = local >= sq.text_len;
-    if (rotate) {
-      const int p = local - sq.text_len;
-      const int hw = sq.H * sq.W;
-      const int pos[3] = {p / hw, (p / sq.W) % sq.H, p % sq.W};
+    const bool rotate = local >= sq.text_len;
+    // heads in groups of kBatch per thread and tensor: the loads of Q AND K of a group are all issued before any is
+    // used, and the table lookups travel with them
+    constexpr int kBatch = 3;
+    for (int h0 = a.head_begin + hsub; h0 < a.head_end; h0 += kBatch * heads_per_pass) {
+      uint4 v[2][kBatch];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int d = chunk * 8 + 2 * u;          // first head dim of the pair
-        int axis, j;
-        if (d < d1) { axis = 0; j = d >> 1; }
-        else if (d < d2) { axis = 1; j = (d - d1) >> 1; }
-        else if (d < d3) { axis = 2; j = (d - d2) >> 1; }
-        else { axis = -1; j = 0; }
-        cs[u] = axis < 0 ? make_float2(1.f, 0.f)
-                         : __ldg(&a.tables[a.g.tab_off[axis] + pos[axis] * (a.g.rope[axis] >> 1) + j]);
-      }
-    }
-#pragma unroll
-    for (int which = 0; which < 2; ++which) {
-      if (a.x[which] == nullptr) continue;
-      const bool norm = a.gain[which] != nullptr;
-      const __nv_bfloat16* src = a.x[which] + tok * a.x_tok_stride[which] + chunk * 8;
-      __nv_bfloat16* dst = a.y[which] + (tok * a.g.heads) * (long long)a.g.head_dim + chunk * 8;
-      // heads in groups of kBatch per thread: all loads of a group are issued before any is used
-      constexpr int kBatch = 3;
-      for (int h0 = a.head_begin + hsub; h0 < a.head_end; h0 += kBatch * heads_per_pass) {
-        uint4 v[kBatch];
+      for (int which = 0; which < 2; ++which) {
+        if (a.x[which] == nullptr) continue;
+        const __nv_bfloat16* src = a.x[which] + tok * a.x_tok_stride[which] + chunk * 8;
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
           const int h = h0 + b * heads_per_pass;
-          if (h < a.head_end) v[b] = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
+          if (h < a.head_end) v[which][b] = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
         }
+      }
+      float2 cs[4];
+      if (rotate) {
+        const int p = local - sq.text_len;
+        const int hw = sq.H * sq.W;
+        const int pt = p / hw, ph = (p / sq.W) % sq.H, pw = p % sq.W;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int pos = axis[u] == 0 ? pt : axis[u] == 1 ? ph : pw;
+          cs[u] = axis[u] < 0 ? make_float2(1.f, 0.f) : __ldg(&a.tables[tab[u] + pos * step[u]]);
+        }
+      }
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        if (a.x[which] == nullptr) continue;
+        const bool norm = a.gain[which] != nullptr;
+        __nv_bfloat16* dst = a.y[which] + (tok * a.g.heads) * (long long)a.g.head_dim + chunk * 8;
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
           const int h = h0 + b * heads_per_pass;
           if (h >= a.head_end) break;
           // all lanes of a row enter together (the bound depends on hsub only)
           const unsigned lanes = __activemask();
-          const uint32_t w[4] = {v[b].x, v[b].y, v[b].z, v[b].w};
+          const uint32_t w[4] = {v[which][b].x, v[which][b].y, v[which][b].z, v[which][b].w};
           float f[8];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -166,8 +170,10 @@ __global__ void __launch_bounds__(256, 4) rope_qk_kernel(const RopeArgs a) {
             for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
             for (int off = chunks >> 1; off > 0; off >>= 1) ss += __shfl_xor_sync(lanes, ss, off);
             const float r = rsqrtf(ss * inv_d + a.eps);
+            // the gains of this thread's eight head dims: 32 bytes that stay in L1 (not kept in registers: the
+            // plain rotary path has no use for them)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] = f[e] * r * gn[which][e];
+            for (int e = 0; e < 8; ++e) f[e] = f[e] * r * __ldg(a.gain[which] + chunk * 8 + e);
           }
           uint32_t o[4];
 #pragma unroll

@@ -11,7 +11,6 @@
 #include <new>
 #include <vector>
 
-#include "attn_fwd_pipe_sm100.cuh"
 #include "attn_fwd_sm100.cuh"
 #include "device_types.cuh"
 #include "exchange_kernels.cuh"
@@ -46,8 +45,7 @@ struct sol_attn3d_plan_s {
   long long total_tokens = 0;
   int total_work = 0;
   int total_quad_work = 0;            // work items when CTA pairs serve 512-row query blocks
-  int pair_mode = 0;                  // 1: use CTA pairs (cta_group::2) where they apply (head_dim 128)
-  int pipe_kernel = 0;                // 1: the pipelined kernel (one query tile per CTA, three score buffers)
+  int pair_mode = 1;                  // CTA pairs (cta_group::2) where they apply: head_dim 128, not block-sparse
   int total_ktiles = 0;
   std::vector<float2> tables;
   int tab_off[3] = {0, 0, 0};
@@ -114,15 +112,6 @@ cudaError_t raise_shared_memory_limits() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(sol::attn_fwd_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              sol::AttnSmem<128, 2>::kDynBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(sol::attn_fwd_pipe_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             sol::PipeSmem<128, 1>::kDynBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(sol::attn_fwd_pipe_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             sol::PipeSmem<64, 1>::kDynBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(sol::attn_fwd_pipe_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             sol::PipeSmem<128, 2>::kDynBytes);
   return e;
 }
 
@@ -283,11 +272,10 @@ int build_plan(sol_attn3d_plan_t* out, const sol_attn3d_desc* d) {
     }
     // Test hook for the failure-detection path: a wait inside the kernel is made to run out on purpose.
     if (const char* e = std::getenv("SOL_ATTN3D_FAULT_INJECT")) p->fault_inject = (unsigned)std::atol(e);
-    // SOL_ATTN3D_PAIR=1: CTA pairs share every K / V tile (one tcgen05.mma.cta_group::2 over 256 query rows).  Off by
-    // default: it lowers power and L2 traffic but lengthens the per-tile dependency chain, and measured slower.
+    // SOL_ATTN3D_PAIR=0 keeps every launch of this plan on single CTAs (for comparisons and tests).  By default two
+    // CTAs on neighbouring SMs share every K / V tile (one tcgen05.mma.cta_group::2 over both CTAs' query rows):
+    // half the L2 -> SM traffic and B-operand reads, which buys SM clock under the power cap at the large sizes.
     if (const char* e = std::getenv("SOL_ATTN3D_PAIR")) p->pair_mode = std::atol(e) != 0;
-    // SOL_ATTN3D_KERNEL=pipe | pingpong: which form of the attention kernel serves this plan
-    if (const char* e = std::getenv("SOL_ATTN3D_KERNEL")) p->pipe_kernel = std::strcmp(e, "pipe") == 0;
     p->v_lbo = p->head_dim == 128 ? 16384u : 16u;
     p->v_sbo = 1024u;
   } catch (const std::bad_alloc&) {
@@ -888,8 +876,7 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
 
   // (3) attention.  Tensor maps: the plan's cached ones for its own workspace, per-call ones otherwise.
   // CTA pairs (two CTAs share every K / V tile) wherever they apply
-  const bool pipe = p->pipe_kernel != 0;
-  const bool pair = p->pair_mode != 0 && p->head_dim == 128 && (pipe || sparse_ws == nullptr);
+  const bool pair = p->pair_mode != 0 && p->head_dim == 128 && sparse_ws == nullptr;
   CUtensorMap tm_q_call, tm_k_call, tm_v_call;
   const CUtensorMap *tm_q = &p->tm_q, *tm_k = pair ? &p->tm_k64 : &p->tm_k, *tm_v = &p->tm_v;
   if (own) {
@@ -931,20 +918,19 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   ap.wave_ctas = o.sm_count > 0 ? o.sm_count : p->sm_count;
   // one sequence: the CTAs of a head range are a contiguous range of work items; several sequences: launch
   // everything and let the CTAs of other heads leave at the door
-  // work items: 256-row query blocks, except for pairs of the two-tile kernel, which take 512 rows
-  const bool quads = pair && !pipe;
-  int units = quads ? p->total_quad_work : p->total_work;
+  // work items: 256-row query blocks for single CTAs, 512-row blocks for pairs
+  int units = pair ? p->total_quad_work : p->total_work;
   ap.cta_offset = 0;
   if (p->n_seqs == 1) {
-    const int per_head = quads ? (p->sched[0].n_qpairs + 1) / 2 : p->sched[0].n_qpairs;
+    const int per_head = pair ? (p->sched[0].n_qpairs + 1) / 2 : p->sched[0].n_qpairs;
     ap.cta_offset = head_begin * per_head;
     units = (head_end - head_begin) * per_head;
   }
   if (pair) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)units * 2u, 1, 1);
-    cfg.blockDim = dim3(pipe ? sol::kPipeThreads : sol::kAttnThreads, 1, 1);
-    cfg.dynamicSmemBytes = pipe ? sol::PipeSmem<128, 2>::kDynBytes : sol::AttnSmem<128, 2>::kDynBytes;
+    cfg.blockDim = dim3(sol::kAttnThreads, 1, 1);
+    cfg.dynamicSmemBytes = sol::AttnSmem<128, 2>::kDynBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr{};
     attr.id = cudaLaunchAttributeClusterDimension;
@@ -953,15 +939,8 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if (pipe) e = cudaLaunchKernelEx(&cfg, sol::attn_fwd_pipe_kernel<128, 2>, *tm_q, *tm_k, *tm_v, ap);
-    else      e = cudaLaunchKernelEx(&cfg, sol::attn_fwd_kernel<128, 2>, *tm_q, *tm_k, *tm_v, ap);
+    e = cudaLaunchKernelEx(&cfg, sol::attn_fwd_kernel<128, 2>, *tm_q, *tm_k, *tm_v, ap);
     if (e != cudaSuccess) return fail_cuda(p, e);
-  } else if (pipe) {
-    // two independent CTAs per 256-row query block, one 128-row tile each
-    if (p->head_dim == 128)
-      sol::attn_fwd_pipe_kernel<128, 1><<<units * 2, sol::kPipeThreads, sol::PipeSmem<128, 1>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
-    else
-      sol::attn_fwd_pipe_kernel<64, 1><<<units * 2, sol::kPipeThreads, sol::PipeSmem<64, 1>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
   } else if (p->head_dim == 128) {
     sol::attn_fwd_kernel<128, 1><<<units, sol::kAttnThreads, sol::AttnSmem<128, 1>::kDynBytes, st>>>(*tm_q, *tm_k, *tm_v, ap);
   } else {

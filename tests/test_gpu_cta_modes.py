@@ -1,8 +1,9 @@
-"""The CTA-pair variant of the attention kernel (SOL_ATTN3D_PAIR=1 when the plan is built): two CTAs on neighbouring
-SMs cover 512 query rows, each loads half of every K / V tile, and one tcgen05.mma.cta_group::2 of M = 256 works on
-both.  It is off by default (measured slower than single CTAs), so these tests are what keeps it correct: the same
-parity bar as the default kernel, the paths that differ (odd number of 256-row blocks, head ranges, rectangular mode,
-key masks, the moving softmax reference, scatter and E4M3 epilogues), and the bounded-wait failure path."""
+"""The two launch modes of the attention kernel at head_dim 128.  By default two CTAs on neighbouring SMs form a pair
+that covers 512 query rows: each loads half of every K / V tile and one tcgen05.mma.cta_group::2 of M = 256 works on
+both.  SOL_ATTN3D_PAIR=0 (read when a plan is built) keeps the plan on single CTAs of 256 rows, which is also what
+the block-sparse variant and head_dim 64 always use.  Both modes get the same parity bar here, on the paths where
+they differ: odd and even numbers of 256-row blocks, head ranges, rectangular mode, key masks, the moving softmax
+reference, scatter and E4M3 epilogues, and the bounded-wait failure path."""
 from dataclasses import replace
 
 import pytest
@@ -17,11 +18,11 @@ TOL_MAX_ABS = 2e-2
 TOL_REL_L2 = 5e-3
 
 
-@pytest.fixture()
-def PB(monkeypatch):
+@pytest.fixture(params=["pair", "single"])
+def PB(request, monkeypatch):
     from paper_2609_35110_b200 import binding
     binding._lib()
-    monkeypatch.setenv("SOL_ATTN3D_PAIR", "1")           # read when a plan is built
+    monkeypatch.setenv("SOL_ATTN3D_PAIR", "1" if request.param == "pair" else "0")   # read when a plan is built
     return binding
 
 
@@ -35,7 +36,7 @@ def _oracle(w, inp):
 
 
 @pytest.mark.parametrize("name", ["lowres", "highres", "cfg_batch", "varlen"])
-def test_pair_mode_matches_oracle_all_rows(PB, name):
+def test_mode_matches_oracle_all_rows(PB, name):
     w = wl.shrunk(name)                                   # 620 / 1156 / 2 x 944 / ragged tokens: odd and even block counts
     inp = wl.make_inputs(w, "cuda")
     attn = PB.Attn3d.from_workload(w, "cuda")
@@ -55,9 +56,11 @@ def test_pair_mode_matches_oracle_all_rows(PB, name):
     attn.close()
 
 
-def test_pair_mode_equals_single_ctas_to_rounding_and_is_deterministic(PB, monkeypatch):
+def test_pair_mode_equals_single_ctas_to_rounding_and_is_deterministic(monkeypatch):
+    from paper_2609_35110_b200 import binding as PB
     w = wl.shrunk("highres")
     inp = wl.make_inputs(w, "cuda")
+    monkeypatch.setenv("SOL_ATTN3D_PAIR", "1")
     pair = PB.Attn3d.from_workload(w, "cuda")
     a = pair.forward(inp.q, inp.k, inp.v).clone()
     b = pair.forward(inp.q, inp.k, inp.v)
@@ -74,7 +77,7 @@ def test_pair_mode_equals_single_ctas_to_rounding_and_is_deterministic(PB, monke
 
 
 @pytest.mark.parametrize("direction", ["rising", "falling"])
-def test_pair_mode_moving_reference(PB, direction):
+def test_mode_moving_reference(PB, direction):
     """The logit ramp of the lazy-rescale tests: every tile moves the reference, in both CTAs of every pair."""
     w = wl.Workload(name="ramp_pair", seqs=(wl.SeqSpec(256, 5, 9, 20),), heads=40, head_dim=128, rope_dims=(32, 48, 32), seed=31)
     inp = wl.make_inputs(w, "cuda")
@@ -99,7 +102,7 @@ def test_pair_mode_moving_reference(PB, direction):
     attn.close()
 
 
-def test_pair_mode_rect_scatter_e4m3_and_host_groups(PB):
+def test_mode_rect_scatter_e4m3_and_host_groups(PB):
     w = replace(wl.shrunk("cfg_batch"), heads=4)
     inp = wl.make_inputs(w, "cuda")
     attn = PB.Attn3d.from_workload(w, "cuda")
@@ -142,9 +145,9 @@ def test_pair_mode_rect_scatter_e4m3_and_host_groups(PB):
     attn.close()
 
 
-def test_pair_mode_withheld_signal_times_out_and_context_survives(PB, monkeypatch):
-    """The failure path of the pair kernel: the leader of work item 0 withholds one "S is ready" signal; the waits of
-    BOTH CTAs that depend on it run out, everyone meets at the cluster barrier, the kernel returns and reports."""
+def test_mode_withheld_signal_times_out_and_context_survives(PB, monkeypatch):
+    """The failure path at head_dim 128: the MMA issuer of work item 0 withholds one "S is ready" signal; the waits that
+    depend on it (of BOTH CTAs of a pair) run out, everyone meets at the final barrier, the kernel returns and reports."""
     w = wl.shrunk("highres")
     inp = wl.make_inputs(w, "cuda")
     monkeypatch.setenv("SOL_ATTN3D_WAIT_LIMIT_MS", "20")
