@@ -78,7 +78,8 @@ __global__ void __launch_bounds__(32) pair_needed_kernel(const SeqDev* __restric
 // sum of squares is a shuffle reduction over them.  fp32 math throughout, one rounding to bf16 at the
 // end.  Prefix tokens are normalised but not rotated.
 // Layout in: [token][head][D] with element strides (tok, head); out: contiguous.
-// Block: (D/8) x HEADS_PER_PASS threads handle one token per iteration.
+// Block: (D/8) x HEADS_PER_PASS threads handle one token per iteration; the host picks HEADS_PER_PASS as a divisor of
+// the number of heads where it can, so that every thread has the same number of rows.
 // ---------------------------------------------------------------------------------------------
 struct RopeArgs {
   const __nv_bfloat16* x[2];
@@ -94,6 +95,7 @@ struct RopeArgs {
   int head_begin, head_end;   // heads [head_begin, head_end) are produced by this launch
 };
 
+template <bool kNorm>
 __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
   const int chunks = a.g.head_dim >> 3;          // 16-byte chunks per head row (8 or 16: divides the warp)
   const int heads_per_pass = blockDim.x / chunks;
@@ -101,6 +103,14 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
   const int hsub = threadIdx.x / chunks;
   const int d1 = a.g.rope[0], d2 = d1 + a.g.rope[1], d3 = d2 + a.g.rope[2];
   const float inv_d = 1.0f / (float)a.g.head_dim;
+  // the gains of this thread's eight head dims (the plain rotary instantiation carries none)
+  float gn[2][kNorm ? 8 : 1];
+  if (kNorm) {
+#pragma unroll
+    for (int which = 0; which < 2; ++which)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) gn[which][kNorm ? e : 0] = a.gain[which] ? __ldg(a.gain[which] + chunk * 8 + e) : 1.0f;
+  }
   // which table entry each of the thread's four pairs uses (fixed per thread: it depends on the chunk only)
   int axis[4], tab[4], step[4];                 // step: table entries per position of that axis
 #pragma unroll
@@ -121,7 +131,7 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
     const bool rotate = local >= sq.text_len;
     // heads in groups of kBatch per thread and tensor: the loads of Q AND K of a group are all issued before any is
     // used, and the table lookups travel with them
-    constexpr int kBatch = 3;
+    constexpr int kBatch = kNorm ? 3 : 4;         // (the normalising instantiation also holds sixteen gains)
     for (int h0 = a.head_begin + hsub; h0 < a.head_end; h0 += kBatch * heads_per_pass) {
       uint4 v[2][kBatch];
 #pragma unroll
@@ -148,7 +158,7 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
         if (a.x[which] == nullptr) continue;
-        const bool norm = a.gain[which] != nullptr;
+        const bool norm = kNorm && a.gain[which] != nullptr;
         __nv_bfloat16* dst = a.y[which] + (tok * a.g.heads) * (long long)a.g.head_dim + chunk * 8;
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
@@ -173,7 +183,7 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
             // the gains of this thread's eight head dims: 32 bytes that stay in L1 (not kept in registers: the
             // plain rotary path has no use for them)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] = f[e] * r * __ldg(a.gain[which] + chunk * 8 + e);
+            for (int e = 0; e < 8; ++e) f[e] = f[e] * r * gn[which][kNorm ? e : 0];
           }
           uint32_t o[4];
 #pragma unroll

@@ -327,10 +327,17 @@ int launch_rope(sol_attn3d_plan_t p, const unsigned char* ws, const void* q, con
   a.head_begin = head_begin;
   a.head_end = head_end > 0 ? head_end : p->heads;
   const int chunks = p->head_dim / 8;
-  const int hpp = std::max(1, std::min(a.head_end - a.head_begin, 256 / chunks));
+  // heads per pass: the largest divisor of the head count that fits a 256-thread block, so that all threads carry the
+  // same number of rows; a head count without a usable divisor (a large prime) takes what fits
+  const int n_heads = a.head_end - a.head_begin, cap = 256 / chunks;
+  const bool norm = q_gain != nullptr || k_gain != nullptr;
+  int hpp = std::max(1, std::min(n_heads, cap));
+  for (int d = std::min(n_heads, cap); !norm && d >= std::max(1, cap / 2); --d)   // (the normalising variant, bound by its
+    if (n_heads % d == 0) { hpp = d; break; }                                      //  reductions, measured better with full blocks)
   const int threads = chunks * hpp;
   const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
-  sol::rope_qk_kernel<<<(unsigned)blocks, threads, 0, st>>>(a);
+  if (norm) sol::rope_qk_kernel<true><<<(unsigned)blocks, threads, 0, st>>>(a);
+  else                                        sol::rope_qk_kernel<false><<<(unsigned)blocks, threads, 0, st>>>(a);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda(p, e);
   ++p->launches;
