@@ -53,7 +53,8 @@ typedef enum {
   SOL_ATTN3D_ERR_CUDA = -6,             /* a CUDA call failed; sol_attn3d_last_cuda_error() has the code */
   SOL_ATTN3D_ERR_DEVICE_TIMEOUT = -7,   /* a bounded wait inside a kernel ran out (status word) */
   SOL_ATTN3D_ERR_NO_MEMORY = -8,        /* host allocation failed */
-  SOL_ATTN3D_ERR_SCRATCH_LIMIT = -9     /* sol_attn3d_forward_noalloc: the plan needs more than the built-in scratch */
+  SOL_ATTN3D_ERR_SCRATCH_LIMIT = -9,    /* sol_attn3d_forward_noalloc: the plan needs more than the built-in scratch */
+  SOL_ATTN3D_ERR_DEVICE_ASSERT = -10    /* debug build: a device-side index check failed (status word) */
 } sol_attn3d_error;
 
 /*
@@ -408,6 +409,18 @@ int sol_attn3d_rope_qk(sol_attn3d_plan_t plan, const void* q, const void* k, voi
  * case `out` is undefined.  The word is cleared by the next sol_attn3d_set_workspace.
  */
 int sol_attn3d_status(sol_attn3d_plan_t plan);
+
+/*
+ * The raw status word behind sol_attn3d_status (same synchronous copy).  Low byte: 0 = fine, 1..3 = a bounded wait
+ * of the producer / MMA issuer / softmax warps ran out, 5 = a device-side index check failed; for 5 the upper 24
+ * bits name the check.  The checks exist only in the debug build of the library (compiled with
+ * -DSOL_ATTN3D_DEBUG=1; sol_attn3d_debug_build() returns 1 there): work-item decoding, key-tile numbers and counts
+ * taken from the lists, output-row addresses, the token -> sequence lookup of the rotary producer (the layout of
+ * Section 3.2 / 3.4 is where an indexing mistake would show).  A failing check records itself and execution goes
+ * on: nothing traps, the kernel returns.  SOL_ATTN3D_ERR_DEVICE_ASSERT is what sol_attn3d_status then returns.
+ */
+int sol_attn3d_status_word(sol_attn3d_plan_t plan, unsigned int* word);
+int sol_attn3d_debug_build(void);
 
 /*
  * Per-kernel timing for roofline accounting (Section 3.2 times "SDPA" apart from the layout work

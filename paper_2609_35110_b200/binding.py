@@ -53,6 +53,7 @@ ERR_CUDA = -6
 ERR_DEVICE_TIMEOUT = -7
 ERR_NO_MEMORY = -8
 ERR_SCRATCH_LIMIT = -9
+ERR_DEVICE_ASSERT = -10
 
 _LIB = None
 
@@ -123,6 +124,10 @@ def _lib():
     lib.sol_attn3d_rope_qk.restype = i32
     lib.sol_attn3d_status.argtypes = [vp]
     lib.sol_attn3d_status.restype = i32
+    lib.sol_attn3d_status_word.argtypes = [vp, ctypes.POINTER(ctypes.c_uint)]
+    lib.sol_attn3d_status_word.restype = i32
+    lib.sol_attn3d_debug_build.argtypes = []
+    lib.sol_attn3d_debug_build.restype = i32
     lib.sol_attn3d_set_profiling.argtypes = [vp, i32]
     lib.sol_attn3d_set_profiling.restype = i32
     lib.sol_attn3d_last_forward_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
@@ -451,6 +456,16 @@ def sol_attn3d_rope_qk(plan, q, k, q_rot, k_rot, stream=None) -> None:
 
 def sol_attn3d_status(plan) -> int:
     return int(_lib().sol_attn3d_status(plan))
+
+
+def sol_attn3d_status_word(plan) -> int:
+    w = ctypes.c_uint()
+    _check(_lib().sol_attn3d_status_word(plan, ctypes.byref(w)), "sol_attn3d_status_word")
+    return int(w.value)
+
+
+def sol_attn3d_debug_build() -> bool:
+    return bool(_lib().sol_attn3d_debug_build())
 
 
 def sol_attn3d_set_profiling(plan, enable: bool) -> None:

@@ -10,6 +10,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_NAME = "libsol_attn3d.so"
 LIB_PATH = os.path.join(HERE, LIB_NAME)
+# the same library with device-side index checks compiled in (see sol_attn3d_status_word in the header)
+DEBUG_LIB_PATH = os.path.join(HERE, "libsol_attn3d_debug.so")
+DEBUG_FLAGS = ("-DSOL_ATTN3D_DEBUG=1",)
 SOURCES = ["sol_attn3d.cu"]
 HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith(".cuh")) + [os.path.join("..", "..", "include", "sol_attn3d.h")]
 
@@ -43,5 +46,11 @@ def build_library(force: bool = False, verbose: bool = False, extra_flags=(), ou
     return out
 
 
+def build_debug_library(force: bool = False) -> str:
+    return build_library(force=force, extra_flags=DEBUG_FLAGS, out=DEBUG_LIB_PATH)
+
+
 if __name__ == "__main__":
     print(build_library(force=True, verbose="-v" in sys.argv))
+    if "--debug" in sys.argv:
+        print(build_debug_library(force=True))

@@ -42,16 +42,6 @@ namespace sol {
 #endif
 constexpr int kAttnThreads = 384;   // 8 softmax warps + producer + MMA issuer + 2 idle warps (a full third warpgroup)
 
-// Fraction of exponentials evaluated on the FMA pipes instead of the special-function unit: of every
-// kEmuMod adjacent pairs the first kEmuCnt use the polynomial (the MUFU and the tensor core would
-// otherwise need the same number of cycles per tile).
-#ifndef SOL_EMU_MOD
-#define SOL_EMU_MOD 4
-#endif
-#ifndef SOL_EMU_CNT
-#define SOL_EMU_CNT 0
-#endif
-
 __device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
   float m0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
   float m1 = max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
@@ -63,40 +53,18 @@ __device__ __forceinline__ float row_max128(const uint32_t (&r)[128]) {
   return max3(m0, m1, fmaxf(__uint_as_float(r[126]), __uint_as_float(r[127])));
 }
 
-// 2^x on the FMA / integer pipes: round-to-nearest split x = j + f, f in [-0.5, 0.5], cubic minimax
-// polynomial for 2^f (relative error 7.5e-5, far below the bf16 rounding of P), exponent bits added with
-// integer arithmetic.  Inputs are clamped at -125 (results below 2^-125 are noise).
-// Scalar fp32 on purpose: on this part a packed fma.f32x2 occupies the FMA pipe about four times as long
-// as one scalar FFMA (measured), so packing saves issue slots but costs pipe time.
-__device__ __forceinline__ float exp2_emulated(float x) {
-  x = fmaxf(x, -125.0f);
-  const float xf = x + 12582912.0f;                 // 1.5 * 2^23: integer part lands in the low mantissa bits
-  const float f = x - (xf - 12582912.0f);
-  float q = fmaf(f, 0.05517148971557617f, 0.2426111102104187f);
-  q = fmaf(q, f, 0.6932610273361206f);
-  q = fmaf(q, f, 0.9999280571937561f);
-  return __int_as_float(__float_as_int(q) + (__float_as_int(xf) << 23));
-}
-
 // One pass over a 128-column score row held in registers: p = 2^(s*c - mc) packed to bf16 and the fp32
-// row sum of the un-rounded p.  kEmu: evaluate a fixed share of the exponentials with exp2_emulated
-// (never on tiles with masked keys: exp2(-inf) must be exactly 0).
-template <bool kEmu>
+// row sum of the un-rounded p.  Every exponential goes to the special-function unit: evaluating a share of them
+// with a polynomial on the FMA pipes was measured more than once (scalar and packed fp32x2 arithmetic, 1/8 to 1/2
+// of the elements) and lost every time: the polynomial costs 12 to 16 issue cycles per element against 8
+// special-function cycles, and the thread-per-row layout has no registers left to interleave enough of them.
 __device__ __forceinline__ void softmax_pass(const uint32_t (&r)[128], float c, float mc, uint32_t (&pk)[64],
                                              float& sum) {
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int cc = 0; cc < 64; ++cc) {
-    const float x_lo = fmaf(__uint_as_float(r[2 * cc]), c, -mc);
-    const float x_hi = fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc);
-    float p_lo, p_hi;
-    if (kEmu && (cc % SOL_EMU_MOD) < SOL_EMU_CNT) {
-      p_lo = exp2_emulated(x_lo);
-      p_hi = exp2_emulated(x_hi);
-    } else {
-      p_lo = ex2_approx(x_lo);
-      p_hi = ex2_approx(x_hi);
-    }
+    const float p_lo = ex2_approx(fmaf(__uint_as_float(r[2 * cc]), c, -mc));
+    const float p_hi = ex2_approx(fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc));
     acc[(2 * cc) & 3] += p_lo;
     acc[(2 * cc + 1) & 3] += p_hi;
     pk[cc] = pack_bf16x2(p_lo, p_hi);
@@ -163,26 +131,19 @@ __device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq
     const int qrow = first_row + rr;
     bool store = qrow < sq.n_tokens;
     if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
+    SOL_DEVICE_CHECK(p.status, !store || (sq.tok_start + qrow >= 0 && sq.tok_start + qrow < p.sink.tok_begin[p.sink.n_dst]),
+                     kCheckOutputRow);
     const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * kRowBytes + ((ch ^ (rr & (kLanesPerRow - 1))) << 4));
     if (store) st_global_evict_first(out_row_ptr(p, sq.tok_start + qrow, head, kFp8 ? 1 : 2) + ch * 16, w, pol_once);
   }
 }
 
-// Half of softmax_pass: 64 columns -> 32 packed pairs, partial sums kept in acc.  Only called for tiles without
-// masked keys, so the share of exponentials that goes to the FMA pipes (see exp2_emulated) applies here too.
+// Half of softmax_pass: 64 columns -> 32 packed pairs, partial sums kept in acc.
 __device__ __forceinline__ void softmax_half(const uint32_t (&r)[64], float c, float mc, uint32_t (&pk)[32], float (&acc)[4]) {
 #pragma unroll
   for (int cc = 0; cc < 32; ++cc) {
-    const float x_lo = fmaf(__uint_as_float(r[2 * cc]), c, -mc);
-    const float x_hi = fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc);
-    float p_lo, p_hi;
-    if ((cc % SOL_EMU_MOD) < SOL_EMU_CNT) {
-      p_lo = exp2_emulated(x_lo);
-      p_hi = exp2_emulated(x_hi);
-    } else {
-      p_lo = ex2_approx(x_lo);
-      p_hi = ex2_approx(x_hi);
-    }
+    const float p_lo = ex2_approx(fmaf(__uint_as_float(r[2 * cc]), c, -mc));
+    const float p_hi = ex2_approx(fmaf(__uint_as_float(r[2 * cc + 1]), c, -mc));
     acc[(2 * cc) & 3] += p_lo;
     acc[(2 * cc + 1) & 3] += p_hi;
     pk[cc] = pack_bf16x2(p_lo, p_hi);
@@ -246,6 +207,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int local = unit - (kPair ? sq.quad_work_start : sq.work_start);
   const int head = local / units_per_head;
   const int blk = local - head * units_per_head;        // query pair (256 rows) or query quad (512 rows)
+  SOL_DEVICE_CHECK(p.status, si < p.n_seqs && local >= 0 && head < p.heads && blk >= 0 && blk < units_per_head, kCheckWorkItem);
+  SOL_DEVICE_CHECK(p.status, !(p.fault_inject == 2u && unit == 0), kCheckInjected);
   // a launch may serve a range of heads only (uniform over the CTA / the pair, before any set-up)
   if (head < p.head_begin || head >= p.head_end) return;
   // rectangular mode: a query block without a wanted row has nothing to do (uniform, before any set-up)
@@ -261,6 +224,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int* __restrict__ ktiles =
       sparse ? p.cta_list + sq.sparse_list_start + (long long)local * sq.n_ktiles : p.ktile_list + sq.ktile_start;
   const uint4* __restrict__ keybits = p.keybits + sq.ktile_start;
+  SOL_DEVICE_CHECK(p.status, n_proc >= 0 && n_proc <= sq.n_ktiles, kCheckTileCount);
   // Successive waves of CTAs walk the key tiles in opposite directions (the softmax does not care about the
   // order): a wave then starts on the tiles its predecessor touched last, which are still in L2, instead of
   // on the ones it touched first, which a long sequence has pushed out by then.
@@ -330,6 +294,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     for (int i = 0; i < n_proc; ++i) {
       const int jt = __ldg(&ktiles[backwards ? n_proc - 1 - i : i]);
+      SOL_DEVICE_CHECK(p.status, jt >= 0 && jt < sq.n_ktiles, kCheckKeyTile);
       const uint4 kb = __ldg(&keybits[jt]);
       ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full(t), i & 1, limit));
       if (!ok) break;
@@ -371,8 +336,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
         }
         if (i == 0) m_ref = row_max128(r);
-        if (mixed) softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
-        else       softmax_pass<true>(r, c, m_ref * c, pk, tile_sum);
+        softmax_pass(r, c, m_ref * c, pk, tile_sum);
       }
       // The pass ran against the current reference maximum, no row maximum taken.
       // All terms are positive, so a row sum <= 2^8 proves that every term is <= 2^8: the reference
@@ -400,7 +364,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int cc = 0; cc < 32; ++cc) o[cc] = __float_as_uint(__uint_as_float(o[cc]) * f);
             tmem_st32(tO + cch * 32, o);
           }
-          softmax_pass<false>(r, c, m_ref * c, pk, tile_sum);
+          softmax_pass(r, c, m_ref * c, pk, tile_sum);
           if (first_half_stored) tmem_wait_st();                         // the stale first half lands before its replacement
           first_half_stored = false;
         }

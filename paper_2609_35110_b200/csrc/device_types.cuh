@@ -60,15 +60,43 @@ struct AttnParams {
   unsigned int* status;     // 0 = fine; written once on a wait time-out
   unsigned int* counters;   // [0]: (warp, key tile) events in which the softmax moved its reference maximum
   unsigned long long wait_limit_ns;
-  unsigned int fault_inject;  // test hook: 1 = CTA 0 never publishes S of query tile 1 (exercises the bounded waits)
+  unsigned int fault_inject;  // test hooks: 1 = work item 0 never publishes S of query tile 1 (exercises the bounded
+                              // waits); 2 = work item 0 fails a device-side check on purpose (debug build)
   unsigned int v_lbo, v_sbo;  // byte offsets of the V (MN-major) shared-memory descriptor
 };
 
+// Status word: low byte = what happened (first event wins), upper bits = detail.
 enum : unsigned int {
   kStatusTimeoutProducer = 1,
   kStatusTimeoutMma = 2,
   kStatusTimeoutSoftmax = 3,
   kStatusBadAlignment = 4,
+  kStatusAssert = 5,          // debug build only: a device-side index check failed; bits [8,32) = which one
 };
+
+// Device-side index checks of the debug build (compile with -DSOL_ATTN3D_DEBUG=1).  A failing check records its
+// site in the status word and execution goes on (the checks guard nothing by themselves): nothing traps, the kernel
+// returns and the host reads the word.  In the release build the macro expands to nothing.
+enum : unsigned int {
+  kCheckWorkItem = 1,         // attention: (sequence, head, query block) decoded from the CTA index is in range
+  kCheckKeyTile = 2,          // attention: a key tile number taken from a list is inside the sequence
+  kCheckTileCount = 3,        // attention: the number of key tiles to walk does not exceed the sequence's
+  kCheckOutputRow = 4,        // attention epilogue: the token of a stored row is inside the packed tensor
+  kCheckTokenSequence = 5,    // rotary producer: the token lies inside the sequence found for it
+  kCheckInjected = 6,         // test hook: the host asked for a failing check
+};
+#ifndef SOL_ATTN3D_DEBUG
+#define SOL_ATTN3D_DEBUG 0
+#endif
+#if SOL_ATTN3D_DEBUG
+#define SOL_DEVICE_CHECK(status_ptr, cond, site)                                                       \
+  do {                                                                                                 \
+    if (!(cond)) atomicCAS((status_ptr), 0u, sol::kStatusAssert | (static_cast<unsigned int>(site) << 8)); \
+  } while (0)
+#else
+#define SOL_DEVICE_CHECK(status_ptr, cond, site) \
+  do {                                           \
+  } while (0)
+#endif
 
 }  // namespace sol

@@ -93,6 +93,7 @@ struct RopeArgs {
   const float2* tables;
   RopeGeom g;
   int head_begin, head_end;   // heads [head_begin, head_end) are produced by this launch
+  unsigned int* status;       // status word (written by the index checks of the debug build only)
 };
 
 template <bool kNorm>
@@ -128,6 +129,7 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
     while (s + 1 < a.n_seqs && !(tok >= a.seqs[s].tok_start && tok < a.seqs[s].tok_start + a.seqs[s].n_tokens)) ++s;
     const SeqDev sq = a.seqs[s];
     const int local = (int)(tok - sq.tok_start);
+    SOL_DEVICE_CHECK(a.status, local >= 0 && local < sq.n_tokens, kCheckTokenSequence);
     const bool rotate = local >= sq.text_len;
     // heads in groups of kBatch per thread and tensor: the loads of Q AND K of a group are all issued before any is
     // used, and the table lookups travel with them

@@ -326,6 +326,7 @@ int launch_rope(sol_attn3d_plan_t p, const unsigned char* ws, const void* q, con
   a.g.heads = p->heads;
   a.head_begin = head_begin;
   a.head_end = head_end > 0 ? head_end : p->heads;
+  a.status = const_cast<unsigned int*>(reinterpret_cast<const unsigned int*>(ws + p->off_status));
   const int chunks = p->head_dim / 8;
   // heads per pass: the largest divisor of the head count that fits a 256-thread block, so that all threads carry the
   // same number of rows; a head count without a usable divisor (a large prime) takes what fits
@@ -1192,8 +1193,18 @@ int sol_attn3d_status(sol_attn3d_plan_t p) {
   unsigned int w = 0;
   const cudaError_t e = cudaMemcpy(&w, p->ws + p->off_status, sizeof(w), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return fail_cuda(p, e);
-  return w == 0 ? SOL_ATTN3D_OK : SOL_ATTN3D_ERR_DEVICE_TIMEOUT;
+  if (w == 0) return SOL_ATTN3D_OK;
+  return (w & 0xffu) == sol::kStatusAssert ? SOL_ATTN3D_ERR_DEVICE_ASSERT : SOL_ATTN3D_ERR_DEVICE_TIMEOUT;
 }
+
+int sol_attn3d_status_word(sol_attn3d_plan_t p, unsigned int* word) {
+  if (p == nullptr || word == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p->ws == nullptr) return SOL_ATTN3D_ERR_NO_WORKSPACE;
+  const cudaError_t e = cudaMemcpy(word, p->ws + p->off_status, sizeof(*word), cudaMemcpyDeviceToHost);
+  return e == cudaSuccess ? SOL_ATTN3D_OK : fail_cuda(p, e);
+}
+
+int sol_attn3d_debug_build(void) { return SOL_ATTN3D_DEBUG; }
 
 int sol_attn3d_last_launch_count(sol_attn3d_plan_t p) { return p == nullptr ? SOL_ATTN3D_ERR_INVALID_ARG : p->launches; }
 
@@ -1221,6 +1232,7 @@ const char* sol_attn3d_strerror(int code) {
     case SOL_ATTN3D_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case SOL_ATTN3D_ERR_NO_MEMORY: return "out of host memory";
     case SOL_ATTN3D_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the built-in 32 MiB array holds";
+    case SOL_ATTN3D_ERR_DEVICE_ASSERT: return "a device-side index check of the debug build failed";
     default: return "unknown error";
   }
 }
