@@ -194,6 +194,7 @@ int sol_attn3d_forward_e4m3(sol_attn3d_plan_t plan, const void* q, const void* k
 #define SOL_ATTN3D_MAX_RANKS 8
 #define SOL_ATTN3D_OUT_BF16 0
 #define SOL_ATTN3D_OUT_E4M3 1
+#define SOL_ATTN3D_OUT_INT8 2
 
 /*
  * Sender's side, one pass: reads this rank's Q, K, V [n_local, heads, head_dim] (bf16, DEVICE) through their
@@ -282,6 +283,37 @@ int sol_attn3d_exchange_dequantize_out_int8(const void* records, void* out_rows,
                                             sol_attn3d_stream_t stream);
 
 /*
+ * sol_attn3d_forward with the block-INT8 output format of Section 3.3 ("Quantized communication": a 144-byte record
+ * per token and head at head_dim 128) written by the attention epilogue itself, the fusion that the paper's "Joint
+ * optimization with quantized communication" aims at: the bf16 rows are never written or re-read.  The values are
+ * rounded to bf16 and quantised by the rule stated above, so the records are byte for byte those of
+ * sol_attn3d_forward followed by sol_attn3d_exchange_quantize_out_int8.
+ *   out_records  DEVICE pointer, dense [total_tokens][heads][sol_attn3d_exchange_record_bytes(OUT_INT8, head_dim)]
+ *                bytes, 16-byte aligned (the plan's output strides, which describe bf16 rows, do not apply).
+ * Everything else as for sol_attn3d_forward.  Rows of a sequence without any valid key become records of zeros.
+ */
+int sol_attn3d_forward_int8(sol_attn3d_plan_t plan, const void* q, const void* k, const void* v, void* out_records,
+                            const uint8_t* key_mask, sol_attn3d_stream_t stream);
+
+/*
+ * sol_attn3d_forward fed by the block-INT8 QKV records of the exchange (Section 3.3, "Quantized communication"): the
+ * receiver's dequantisation is fused into the rotary producer ("Joint optimization with quantized communication"),
+ * so the packed bf16 QKV tensor is never written or re-read.  Each value is q * s rounded to bf16, exactly what
+ * sol_attn3d_exchange_unpack_qkv_int8 would have stored, and Q, K are rotated from there: the result is bit for bit
+ * that of unpack followed by sol_attn3d_forward on the unpacked views.
+ *   qkv_records  DEVICE pointer, dense [total_tokens][heads][record_bytes(QKV_INT8, head_dim)], 16-byte aligned
+ *                (heads = this plan's heads, e.g. a rank's shard after the all-to-all).
+ *   v_scratch    DEVICE pointer, caller-owned bf16 [total_tokens][heads][head_dim], 16-byte aligned: the producer
+ *                writes the dequantised V there and the attention kernel reads it (rotated Q and K go to the plan's
+ *                workspace as always).  Undefined afterwards.
+ *   out          as the output of sol_attn3d_forward (out_format BF16, plan's output strides),
+ *                sol_attn3d_forward_e4m3 (E4M3) or sol_attn3d_forward_int8 (INT8).
+ * The plan's q / k / v strides do not apply.  Everything else as for sol_attn3d_forward.
+ */
+int sol_attn3d_forward_qkv_int8(sol_attn3d_plan_t plan, const void* qkv_records, void* v_scratch, void* out,
+                                const uint8_t* key_mask, int out_format, sol_attn3d_stream_t stream);
+
+/*
  * sol_attn3d_forward whose epilogue delivers each output row to the owner of its token: the output return
  * of the exchange and the head merge fused into the attention kernel (no counterpart kernel in the paper,
  * which returns the output with a collective; same result).  The plan describes this rank's head shard
@@ -293,7 +325,9 @@ int sol_attn3d_exchange_dequantize_out_int8(const void* records, void* out_rows,
  *               owner without tokens.
  *   tok_begin   HOST array of n_dst+1 ascending token offsets, tok_begin[0] = 0, tok_begin[n_dst] = total.
  *   dst_heads   heads per row in the destinations (all ranks' shards); head_offset = this shard's first head.
- *   out_format  SOL_ATTN3D_OUT_BF16 or SOL_ATTN3D_OUT_E4M3 (see sol_attn3d_forward_e4m3).
+ *   out_format  SOL_ATTN3D_OUT_BF16, SOL_ATTN3D_OUT_E4M3 (see sol_attn3d_forward_e4m3) or SOL_ATTN3D_OUT_INT8 (see
+ *               sol_attn3d_forward_int8; a destination row then holds dst_heads records instead of dst_heads * head_dim
+ *               elements).
  * The arrays are read during the call only.  The caller needs a barrier across ranks before the owners
  * read their rows.  Everything else as for sol_attn3d_forward.
  */

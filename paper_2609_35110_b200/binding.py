@@ -90,6 +90,10 @@ def _lib():
     lib.sol_attn3d_forward_rect.restype = i32
     lib.sol_attn3d_forward_e4m3.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.sol_attn3d_forward_e4m3.restype = i32
+    lib.sol_attn3d_forward_int8.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.sol_attn3d_forward_int8.restype = i32
+    lib.sol_attn3d_forward_qkv_int8.argtypes = [vp, vp, vp, vp, vp, i32, vp]
+    lib.sol_attn3d_forward_qkv_int8.restype = i32
     lib.sol_attn3d_forward_scatter.argtypes = [vp, vp, vp, vp, vp, i32, ctypes.POINTER(vp), ctypes.POINTER(i64), i32, i32,
                                                i32, vp]
     lib.sol_attn3d_forward_scatter.restype = i32
@@ -276,7 +280,7 @@ def sol_attn3d_forward_host(plan, q_host: torch.Tensor, k_host: torch.Tensor, v_
            "sol_attn3d_forward_host")
 
 
-OUT_BF16, OUT_E4M3 = 0, 1
+OUT_BF16, OUT_E4M3, OUT_INT8 = 0, 1, 2
 MAX_RANKS = 8
 
 
@@ -289,6 +293,30 @@ def sol_attn3d_forward_e4m3(plan, q, k, v, out_e4m3: torch.Tensor, key_mask=None
         raise ValueError("out_e4m3 must be a CUDA tensor of one-byte elements")
     _check(_lib().sol_attn3d_forward_e4m3(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out_e4m3), _ptr(key_mask),
                                           _stream(stream)), "sol_attn3d_forward_e4m3")
+
+
+def sol_attn3d_forward_int8(plan, q, k, v, out_records: torch.Tensor, key_mask=None, stream=None) -> None:
+    """Forward whose epilogue writes block-INT8 output records [tokens, heads, record_bytes] (uint8)."""
+    for t in (q, k, v):
+        if not t.is_cuda or t.dtype != torch.bfloat16:
+            raise ValueError("q, k, v must be CUDA bf16 tensors")
+    if not out_records.is_cuda or out_records.element_size() != 1 or not out_records.is_contiguous():
+        raise ValueError("out_records must be a contiguous CUDA tensor of one-byte elements")
+    _check(_lib().sol_attn3d_forward_int8(plan, _ptr(q), _ptr(k), _ptr(v), _ptr(out_records), _ptr(key_mask),
+                                          _stream(stream)), "sol_attn3d_forward_int8")
+
+
+def sol_attn3d_forward_qkv_int8(plan, qkv_records: torch.Tensor, v_scratch: torch.Tensor, out: torch.Tensor, key_mask=None,
+                                out_format: int = OUT_BF16, stream=None) -> None:
+    """Forward fed by block-INT8 QKV records [tokens, heads, record_bytes]; v_scratch: bf16 [tokens, heads, D]."""
+    if not qkv_records.is_cuda or qkv_records.element_size() != 1 or not qkv_records.is_contiguous():
+        raise ValueError("qkv_records must be a contiguous CUDA tensor of one-byte elements")
+    if not v_scratch.is_cuda or v_scratch.dtype != torch.bfloat16 or not v_scratch.is_contiguous():
+        raise ValueError("v_scratch must be a contiguous CUDA bf16 tensor")
+    if not out.is_cuda:
+        raise ValueError("out must be a CUDA tensor")
+    _check(_lib().sol_attn3d_forward_qkv_int8(plan, _ptr(qkv_records), _ptr(v_scratch), _ptr(out), _ptr(key_mask), out_format,
+                                              _stream(stream)), "sol_attn3d_forward_qkv_int8")
 
 
 def _ptr_array(ptrs: Sequence[int]):

@@ -28,6 +28,7 @@
 #include <math_constants.h>
 
 #include "device_types.cuh"
+#include "exchange_kernels.cuh"
 #include "ptx_sm100.cuh"
 
 namespace sol {
@@ -135,6 +136,55 @@ __device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq
                      kCheckOutputRow);
     const uint4 w = *reinterpret_cast<const uint4*>(stage + rr * kRowBytes + ((ch ^ (rr & (kLanesPerRow - 1))) << 4));
     if (store) st_global_evict_first(out_row_ptr(p, sq.tok_start + qrow, head, kFp8 ? 1 : 2) + ch * 16, w, pol_once);
+  }
+}
+
+// Epilogue in the block-INT8 wire format of the exchange (Section 3.3, "Quantized communication"): the thread that owns
+// an accumulator row writes that row's record, [D int8 | D/32 scale codes | zeros to a multiple of 16 bytes], straight
+// from tensor memory.  A group of 32 values is exactly one 32-column load.  The values are first rounded to bf16 and
+// then quantised by the rule of quantize_records_kernel, so the bytes equal those of the bf16 epilogue followed by that
+// kernel; what is saved is a write and a read of the bf16 rows.  A record is contiguous (144 bytes at D = 128), so
+// every thread writes whole 16-byte chunks of its own record; nothing is staged.
+template <int D>
+__device__ __forceinline__ void store_rows_int8(const AttnParams& p, const SeqDev& sq, int head, int qrow, uint32_t tO, float inv) {
+  constexpr int kGroups = D / 32;
+  constexpr int kRecBytes = (D + kGroups + 15) / 16 * 16;
+  bool store = qrow < sq.n_tokens;
+  if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
+  SOL_DEVICE_CHECK(p.status, !store || sq.tok_start + qrow < p.sink.tok_begin[p.sink.n_dst], kCheckOutputRow);
+  uint8_t* rec = out_row_ptr(p, sq.tok_start + (store ? qrow : 0), head, 1);
+  uint32_t codes = 0;
+#pragma unroll
+  for (int grp = 0; grp < kGroups; ++grp) {
+    uint32_t o[32];
+    tmem_ld32(tO + grp * 32, o);                  // warp-collective: every lane loads, whether or not its row is stored
+    tmem_wait_ld();
+    float f[32];
+    float amax = 0.f;
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      f[e] = __bfloat162float(__float2bfloat16_rn(__uint_as_float(o[e]) * inv));
+      amax = fmaxf(amax, fabsf(f[e]));
+    }
+    const int code = ue5m3_smallest_cover(amax);
+    const float rs = __frcp_rn(ue5m3_value(code));
+    uint32_t w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      w[j] = pack_low_bytes(rint_sat_s8(__fmul_rn(f[4 * j], rs)), rint_sat_s8(__fmul_rn(f[4 * j + 1], rs)),
+                            rint_sat_s8(__fmul_rn(f[4 * j + 2], rs)), rint_sat_s8(__fmul_rn(f[4 * j + 3], rs)));
+    codes |= (uint32_t)code << (8 * grp);
+    if (store) {
+      uint4* dst = reinterpret_cast<uint4*>(rec + grp * 32);
+      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+  }
+  // tail: the scale codes, then zeros up to the record size (D = 128: one chunk; D = 64: 2 codes + 14 zeros)
+  if (store) {
+#pragma unroll
+    for (int b = D; b < kRecBytes; b += 16)
+      *reinterpret_cast<uint4*>(rec + b) = make_uint4(b == D ? codes : 0u, 0u, 0u, 0u);
   }
 }
 
@@ -389,14 +439,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (ok && n_proc > 0) {
       const float inv = 1.0f / l;
       uint8_t* stage = smem + L::kOffQ + t * L::kTile + wq * 32 * (D * 2);
-      if (p.sink.fmt == kOutE4M3) store_rows<D, true>(p, sq, head, q_row0 + t * 128 + wq * 32, lane, tO, inv, stage);
-      else                        store_rows<D, false>(p, sq, head, q_row0 + t * 128 + wq * 32, lane, tO, inv, stage);
+      if (p.sink.fmt == kOutInt8)      store_rows_int8<D>(p, sq, head, q_row0 + t * 128 + row, tO, inv);
+      else if (p.sink.fmt == kOutE4M3) store_rows<D, true>(p, sq, head, q_row0 + t * 128 + wq * 32, lane, tO, inv, stage);
+      else                             store_rows<D, false>(p, sq, head, q_row0 + t * 128 + wq * 32, lane, tO, inv, stage);
     } else if (ok) {
       // no key tile at all (every key of the sequence masked): the row is defined as zero
       const int qrow = q_row0 + t * 128 + row;
       bool store = qrow < sq.n_tokens;
       if (store && p.query_mask != nullptr) store = p.query_mask[sq.tok_start + qrow] != 0;
-      if (store) {
+      if (store && p.sink.fmt == kOutInt8) {
+        // a record of zeros: every group's scale code is the smallest one (0x01), as the quantiser writes it
+        constexpr int kRecBytes = (D + D / 32 + 15) / 16 * 16;
+        uint8_t* dst = out_row_ptr(p, sq.tok_start + qrow, head, 1);
+        for (int b = 0; b < kRecBytes; b += 16)
+          *reinterpret_cast<uint4*>(dst + b) = make_uint4(b == D ? (D == 128 ? 0x01010101u : 0x00000101u) : 0u, 0u, 0u, 0u);
+      } else if (store) {
         const int row_bytes = p.sink.fmt == kOutE4M3 ? D : D * 2;
         uint8_t* dst = out_row_ptr(p, sq.tok_start + qrow, head, row_bytes / D);
         for (int c16 = 0; c16 < row_bytes / 16; ++c16) *reinterpret_cast<uint4*>(dst + c16 * 16) = make_uint4(0u, 0u, 0u, 0u);

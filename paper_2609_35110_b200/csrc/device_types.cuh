@@ -32,12 +32,13 @@ struct RopeGeom {
 // base[g] addresses row tok_begin[g] (head 0 of this launch) in that destination, which may be this GPU's
 // memory or a peer's mapped into this process.  Plain forward: one destination starting at token 0.
 constexpr int kMaxOutDst = 8;
-enum : int { kOutBf16 = 0, kOutE4M3 = 1 };
+enum : int { kOutBf16 = 0, kOutE4M3 = 1, kOutInt8 = 2 };
 struct OutSink {
   void* base[kMaxOutDst];
   long long tok_begin[kMaxOutDst + 1];
   int n_dst;
-  int fmt;                  // kOutBf16: 2-byte elements; kOutE4M3: one raw E4M3 byte per element (unit scale)
+  int fmt;                  // kOutBf16: 2-byte elements; kOutE4M3: one raw E4M3 byte per element (unit scale);
+                            // kOutInt8: one block-INT8 record per (token, head), strides counted in bytes
 };
 
 struct AttnParams {

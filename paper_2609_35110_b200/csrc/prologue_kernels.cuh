@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include "device_types.cuh"
+#include "exchange_kernels.cuh"
 
 namespace sol {
 
@@ -200,6 +201,100 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
           }
           *reinterpret_cast<uint4*>(dst + (long long)h * a.g.head_dim) = make_uint4(o[0], o[1], o[2], o[3]);
         }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same producer fed by the block-INT8 QKV records of the exchange (Section 3.3, "Quantized communication"; the
+// fusion of the receiver's dequantisation into the consumer is what "Joint optimization with quantized
+// communication" asks for): records [token][head][q int8 x D | k | v | 3 D/32 scale codes | pad] -> rotated Q~, K~
+// and plain V, all bf16 [token][head][D].  value = q * s is rounded to bf16 first and rotated then, so Q~ and K~ are
+// bit for bit what dequantize_records_kernel followed by rope_qk_kernel produce; the packed bf16 QKV tensor in
+// between (a write and a read of the whole shard) is never made.  Thread mapping as in rope_qk_kernel: a thread owns
+// 8 head dims of a token (8 record bytes in, 16 bytes out), fetches its four (cos, sin) once per token and walks
+// over the heads.
+// ---------------------------------------------------------------------------------------------
+struct RopeRecordArgs {
+  const uint8_t* records;     // [total_tokens][heads][rec_bytes]
+  __nv_bfloat16* y[3];        // Q~, K~, V outputs, contiguous [token][head][D]
+  int rec_bytes;
+  const SeqDev* seqs;
+  int n_seqs;
+  long long total_tokens;
+  const float2* tables;
+  RopeGeom g;
+  unsigned int* status;
+};
+
+__global__ void __launch_bounds__(256, 3) rope_records_kernel(const RopeRecordArgs a) {
+  const int D = a.g.head_dim;
+  const int chunks = D >> 3;
+  const int heads_per_pass = blockDim.x / chunks;
+  const int chunk = threadIdx.x % chunks;
+  const int hsub = threadIdx.x / chunks;
+  const int d1 = a.g.rope[0], d2 = d1 + a.g.rope[1], d3 = d2 + a.g.rope[2];
+  int axis[4], tab[4], step[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int d = chunk * 8 + 2 * u;
+    if (d < d1)      { axis[u] = 0; tab[u] = a.g.tab_off[0] + (d >> 1);        step[u] = a.g.rope[0] >> 1; }
+    else if (d < d2) { axis[u] = 1; tab[u] = a.g.tab_off[1] + ((d - d1) >> 1); step[u] = a.g.rope[1] >> 1; }
+    else if (d < d3) { axis[u] = 2; tab[u] = a.g.tab_off[2] + ((d - d2) >> 1); step[u] = a.g.rope[2] >> 1; }
+    else             { axis[u] = -1; tab[u] = 0; step[u] = 0; }
+  }
+  const int code_off = 3 * D + (chunk >> 2);      // this chunk's scale code inside a tensor's D/32 codes
+  const int n_codes = D >> 5;
+
+  for (long long tok = blockIdx.x; tok < a.total_tokens; tok += gridDim.x) {
+    int s = 0;
+    while (s + 1 < a.n_seqs && !(tok >= a.seqs[s].tok_start && tok < a.seqs[s].tok_start + a.seqs[s].n_tokens)) ++s;
+    const SeqDev sq = a.seqs[s];
+    const int local = (int)(tok - sq.tok_start);
+    SOL_DEVICE_CHECK(a.status, local >= 0 && local < sq.n_tokens, kCheckTokenSequence);
+    const bool rotate = local >= sq.text_len;
+    float2 cs[4];
+    if (rotate) {
+      const int p = local - sq.text_len;
+      const int hw = sq.H * sq.W;
+      const int pt = p / hw, ph = (p / sq.W) % sq.H, pw = p % sq.W;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int pos = axis[u] == 0 ? pt : axis[u] == 1 ? ph : pw;
+        cs[u] = axis[u] < 0 ? make_float2(1.f, 0.f) : __ldg(&a.tables[tab[u] + pos * step[u]]);
+      }
+    }
+    for (int h = hsub; h < a.g.heads; h += heads_per_pass) {
+      const uint8_t* rec = a.records + (tok * a.g.heads + h) * (long long)a.rec_bytes;
+      uint2 v[3];
+      float sc[3];
+#pragma unroll
+      for (int which = 0; which < 3; ++which) {
+        v[which] = __ldg(reinterpret_cast<const uint2*>(rec + which * D + chunk * 8));
+        sc[which] = ue5m3_value(__ldg(rec + code_off + which * n_codes));
+      }
+#pragma unroll
+      for (int which = 0; which < 3; ++which) {
+        const uint32_t w[2] = {v[which].x, v[which].y};
+        float f[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float qv = (float)(int)(int8_t)((w[e >> 2] >> (8 * (e & 3))) & 0xffu);
+          f[e] = __bfloat162float(__float2bfloat16_rn(qv * sc[which]));     // the value the bf16 wire tensor would hold
+        }
+        uint32_t o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          float re = f[2 * u], ro = f[2 * u + 1];
+          if (which < 2 && rotate) {
+            re = f[2 * u] * cs[u].x - f[2 * u + 1] * cs[u].y;
+            ro = f[2 * u] * cs[u].y + f[2 * u + 1] * cs[u].x;
+          }
+          const __nv_bfloat162 r2 = __floats2bfloat162_rn(re, ro);
+          o[u] = *reinterpret_cast<const uint32_t*>(&r2);
+        }
+        *reinterpret_cast<uint4*>(a.y[which] + (tok * a.g.heads + h) * (long long)D + chunk * 8) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   }

@@ -13,7 +13,6 @@
 
 #include "attn_fwd_sm100.cuh"
 #include "device_types.cuh"
-#include "exchange_kernels.cuh"
 #include "prologue_kernels.cuh"
 #include "sparse_kernels.cuh"
 
@@ -63,6 +62,7 @@ struct sol_attn3d_plan_s {
   CUtensorMap tm_q{}, tm_k{}, tm_v{};
   CUtensorMap tm_k64{};               // K~ with 64-token boxes: what one CTA of a pair loads of a key tile
   const void* v_cached = nullptr;
+  bool v_cached_dense = false;        // the cached V map was encoded with dense strides (inputs were records)
   int keybits_state = 0;              // 0 unknown, 1 built for "no mask", 2 built from a mask
   int last_cuda = 0;
   unsigned long long wait_limit_ns = 2000000000ull;
@@ -458,6 +458,7 @@ struct FwdOpts {
   const int64_t* tok_begin = nullptr;
   int dst_heads = 0, head_offset = 0;
   int head_begin = 0, head_end = 0;   // serve heads [head_begin, head_end) only (0, 0 = all)
+  const void* qkv_records = nullptr;  // Q, K, V arrive as block-INT8 records (q and k are then NULL, v is a bf16 scratch)
   bool skip_keybits = false;          // the key-validity bits of this mask were built by an earlier call
   bool keep_launch_count = false;     // one of several launch sets of the same API call: keep counting
   // Scratch other than the plan's bound workspace (sol_attn3d_forward_noalloc): the caller of forward_impl has put
@@ -504,13 +505,32 @@ int sol_attn3d_forward_e4m3(sol_attn3d_plan_t p, const void* q, const void* k, c
   return forward_impl(p, q, k, v, out_e4m3, key_mask, stream, o);
 }
 
+int sol_attn3d_forward_qkv_int8(sol_attn3d_plan_t p, const void* qkv_records, void* v_scratch, void* out,
+                                const uint8_t* key_mask, int out_format, sol_attn3d_stream_t stream) {
+  if (qkv_records == nullptr || v_scratch == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (out_format != SOL_ATTN3D_OUT_BF16 && out_format != SOL_ATTN3D_OUT_E4M3 && out_format != SOL_ATTN3D_OUT_INT8)
+    return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (out == qkv_records) return SOL_ATTN3D_ERR_INVALID_ARG;
+  FwdOpts o;
+  o.qkv_records = qkv_records;
+  o.out_fmt = out_format == SOL_ATTN3D_OUT_E4M3 ? sol::kOutE4M3 : out_format == SOL_ATTN3D_OUT_INT8 ? sol::kOutInt8 : sol::kOutBf16;
+  return forward_impl(p, nullptr, nullptr, v_scratch, out, key_mask, stream, o);
+}
+
+int sol_attn3d_forward_int8(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out_records,
+                            const uint8_t* key_mask, sol_attn3d_stream_t stream) {
+  FwdOpts o;
+  o.out_fmt = sol::kOutInt8;
+  return forward_impl(p, q, k, v, out_records, key_mask, stream, o);
+}
+
 int sol_attn3d_forward_scatter(sol_attn3d_plan_t p, const void* q, const void* k, const void* v,
                                const uint8_t* key_mask, int n_dst, void* const* dst, const int64_t* tok_begin,
                                int dst_heads, int head_offset, int out_format, sol_attn3d_stream_t stream) {
-  if (n_dst < 1 || (out_format != SOL_ATTN3D_OUT_BF16 && out_format != SOL_ATTN3D_OUT_E4M3))
+  if (n_dst < 1 || (out_format != SOL_ATTN3D_OUT_BF16 && out_format != SOL_ATTN3D_OUT_E4M3 && out_format != SOL_ATTN3D_OUT_INT8))
     return SOL_ATTN3D_ERR_INVALID_ARG;
   FwdOpts o;
-  o.out_fmt = out_format == SOL_ATTN3D_OUT_E4M3 ? sol::kOutE4M3 : sol::kOutBf16;
+  o.out_fmt = out_format == SOL_ATTN3D_OUT_E4M3 ? sol::kOutE4M3 : out_format == SOL_ATTN3D_OUT_INT8 ? sol::kOutInt8 : sol::kOutBf16;
   o.n_dst = n_dst;
   o.dst = dst;
   o.tok_begin = tok_begin;
@@ -765,29 +785,34 @@ int sol_attn3d_qknorm_rope(sol_attn3d_plan_t p, const void* q, const void* k, co
 namespace {
 int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* v, void* out, const uint8_t* key_mask,
                  sol_attn3d_stream_t stream, const FwdOpts& o) {
-  if (p == nullptr || q == nullptr || k == nullptr || v == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (p == nullptr || v == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (o.qkv_records == nullptr && (q == nullptr || k == nullptr)) return SOL_ATTN3D_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o.qkv_records)) return SOL_ATTN3D_ERR_INVALID_ARG;
   sol::OutSink sink{};
   sink.fmt = o.out_fmt;
   long long o_tok_stride = p->so.tok, o_head_stride = p->so.head;
+  // block-INT8 records: dense [token][head][record], strides in bytes (the plan's output strides describe bf16 rows)
+  const long long rec_bytes = (long long)sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_OUT_INT8, p->head_dim);
+  if (o.out_fmt == sol::kOutInt8) { o_tok_stride = (long long)p->heads * rec_bytes; o_head_stride = rec_bytes; }
   if (o.n_dst > 0) {
     // scatter: destination g owns flat tokens [tok_begin[g], tok_begin[g+1]) as rows [n_g][dst_heads][head_dim]
     if (o.n_dst > sol::kMaxOutDst || o.dst == nullptr || o.tok_begin == nullptr) return SOL_ATTN3D_ERR_INVALID_ARG;
     if (o.head_offset < 0 || o.dst_heads < o.head_offset + p->heads) return SOL_ATTN3D_ERR_INVALID_ARG;
     if (o.tok_begin[0] != 0 || o.tok_begin[o.n_dst] != p->total_tokens) return SOL_ATTN3D_ERR_INVALID_ARG;
-    const size_t esize = o.out_fmt == sol::kOutE4M3 ? 1 : 2;
+    // bytes of one head's slot in a destination row
+    const size_t slot = o.out_fmt == sol::kOutInt8 ? (size_t)rec_bytes : (size_t)p->head_dim * (o.out_fmt == sol::kOutE4M3 ? 1 : 2);
     for (int g = 0; g < o.n_dst; ++g) {
       if (o.tok_begin[g + 1] < o.tok_begin[g]) return SOL_ATTN3D_ERR_INVALID_ARG;
       const bool empty = o.tok_begin[g + 1] == o.tok_begin[g];
       if (!empty && (o.dst[g] == nullptr || !aligned16(o.dst[g]))) return SOL_ATTN3D_ERR_INVALID_ARG;
       if (o.dst[g] == q || o.dst[g] == k || o.dst[g] == v) return SOL_ATTN3D_ERR_INVALID_ARG;
-      sink.base[g] = static_cast<unsigned char*>(o.dst[g]) + (size_t)o.head_offset * p->head_dim * esize;
+      sink.base[g] = static_cast<unsigned char*>(o.dst[g]) + (size_t)o.head_offset * slot;
       sink.tok_begin[g] = o.tok_begin[g];
     }
     sink.tok_begin[o.n_dst] = o.tok_begin[o.n_dst];
     sink.n_dst = o.n_dst;
-    o_tok_stride = (long long)o.dst_heads * p->head_dim;
-    o_head_stride = p->head_dim;
+    o_tok_stride = (long long)o.dst_heads * (o.out_fmt == sol::kOutInt8 ? rec_bytes : p->head_dim);
+    o_head_stride = o.out_fmt == sol::kOutInt8 ? rec_bytes : p->head_dim;
   } else {
     if (out == nullptr || !aligned16(out)) return SOL_ATTN3D_ERR_INVALID_ARG;
     if (out == q || out == k || out == v) return SOL_ATTN3D_ERR_INVALID_ARG;
@@ -836,8 +861,35 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
 
   if (p->prof && (e = cudaEventRecord(p->ev[1], st)) != cudaSuccess) return fail_cuda(p, e);
 
-  // (2) rotary prologue: Q~, K~ into the workspace
-  int rc = launch_rope(p, ws, q, k, ws + p->off_qrot, ws + p->off_krot, q_gain, k_gain, eps, st, head_begin, head_end);
+  // (2) rotary prologue: Q~, K~ into the workspace (and V out of the records, when the inputs are records)
+  int rc = SOL_ATTN3D_OK;
+  const Strides dense_v{(long long)p->heads * p->head_dim, (long long)p->head_dim};
+  if (o.qkv_records != nullptr) {
+    sol::RopeRecordArgs ra{};
+    ra.records = static_cast<const uint8_t*>(o.qkv_records);
+    ra.y[0] = reinterpret_cast<__nv_bfloat16*>(ws + p->off_qrot);
+    ra.y[1] = reinterpret_cast<__nv_bfloat16*>(ws + p->off_krot);
+    ra.y[2] = static_cast<__nv_bfloat16*>(const_cast<void*>(v));
+    ra.rec_bytes = (int)sol_attn3d_exchange_record_bytes(SOL_ATTN3D_WIRE_QKV_INT8, p->head_dim);
+    ra.seqs = d_seqs;
+    ra.n_seqs = p->n_seqs;
+    ra.total_tokens = p->total_tokens;
+    ra.tables = reinterpret_cast<const float2*>(ws + p->off_tables);
+    for (int i = 0; i < 3; ++i) { ra.g.rope[i] = p->rope[i]; ra.g.tab_off[i] = p->tab_off[i]; }
+    ra.g.head_dim = p->head_dim;
+    ra.g.heads = p->heads;
+    ra.status = reinterpret_cast<unsigned int*>(ws + p->off_status);
+    const int chunks = p->head_dim / 8, cap = 256 / chunks;
+    int hpp = std::max(1, std::min(p->heads, cap));
+    for (int d = std::min(p->heads, cap); d >= std::max(1, cap / 2); --d)
+      if (p->heads % d == 0) { hpp = d; break; }
+    const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
+    sol::rope_records_kernel<<<(unsigned)blocks, chunks * hpp, 0, st>>>(ra);
+    if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
+    ++p->launches;
+  } else {
+    rc = launch_rope(p, ws, q, k, ws + p->off_qrot, ws + p->off_krot, q_gain, k_gain, eps, st, head_begin, head_end);
+  }
   if (rc != SOL_ATTN3D_OK) return rc;
   if (p->prof && (e = cudaEventRecord(p->ev[2], st)) != cudaSuccess) return fail_cuda(p, e);
 
@@ -888,16 +940,18 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
   CUtensorMap tm_q_call, tm_k_call, tm_v_call;
   const CUtensorMap *tm_q = &p->tm_q, *tm_k = pair ? &p->tm_k64 : &p->tm_k, *tm_v = &p->tm_v;
   if (own) {
-    if (p->v_cached != v) {
-      rc = encode_map(encode, p, &p->tm_v, v, p->sv);
+    const bool v_dense = o.qkv_records != nullptr;
+    if (p->v_cached != v || p->v_cached_dense != v_dense) {
+      rc = encode_map(encode, p, &p->tm_v, v, v_dense ? dense_v : p->sv);
       if (rc != SOL_ATTN3D_OK) return rc;
       p->v_cached = v;
+      p->v_cached_dense = v_dense;
     }
   } else {
     const Strides dense{(long long)p->heads * p->head_dim, (long long)p->head_dim};
     if ((rc = encode_map(encode, p, &tm_q_call, ws + p->off_qrot, dense)) != SOL_ATTN3D_OK) return rc;
     if ((rc = encode_map(encode, p, &tm_k_call, ws + p->off_krot, dense, pair ? 64 : 128)) != SOL_ATTN3D_OK) return rc;
-    if ((rc = encode_map(encode, p, &tm_v_call, v, p->sv)) != SOL_ATTN3D_OK) return rc;
+    if ((rc = encode_map(encode, p, &tm_v_call, v, o.qkv_records != nullptr ? dense_v : p->sv)) != SOL_ATTN3D_OK) return rc;
     tm_q = &tm_q_call; tm_k = &tm_k_call; tm_v = &tm_v_call;
   }
   sol::AttnParams ap{};

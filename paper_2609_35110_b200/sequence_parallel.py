@@ -82,21 +82,28 @@ class PeerBuffers:
         self.keep = keep                                   # whatever must stay alive with the buffers (handles)
 
 
-def peer_buffer_shapes(total: int, heads: int, head_dim: int, n_ranks: int):
-    """([total, 3, heads/G, D], [largest shard, heads, D]): the two buffers every rank of the peer transport owns."""
+def peer_buffer_shapes(total: int, heads: int, head_dim: int, n_ranks: int, qkv_record_bytes: int = 0,
+                       out_record_bytes: int = 0):
+    """Shapes of the two buffers every rank of the peer transport owns: the QKV receive buffer, [total, 3, heads/G, D]
+    bf16 or [total, heads/G, record] bytes for the block-INT8 wire format, and the output rows, [largest shard, heads,
+    D] or [largest shard, heads, record] bytes."""
     per = shard_ranges(total, n_ranks)[0]
-    return (total, 3, heads // n_ranks, head_dim), (max(per[1] - per[0], 1), heads, head_dim)
+    n_max, hl = max(per[1] - per[0], 1), heads // n_ranks
+    qkv = (total, hl, qkv_record_bytes) if qkv_record_bytes else (total, 3, hl, head_dim)
+    merged = (n_max, heads, out_record_bytes) if out_record_bytes else (n_max, heads, head_dim)
+    return qkv, merged
 
 
-def symmetric_memory_buffers(total, heads, head_dim, out_dtype, device, group=None) -> PeerBuffers:
+def symmetric_memory_buffers(total, heads, head_dim, out_dtype, device, group=None, qkv_record_bytes: int = 0,
+                             out_record_bytes: int = 0) -> PeerBuffers:
     """Buffers in symmetric memory, every rank's mapped into this process (plain peer addresses; no multicast is
     used by the kernels that store through them).  Collective: every rank of `group` must call it."""
     import torch.distributed as dist
     import torch.distributed._symmetric_memory as symm
     n_ranks, rank = dist.get_world_size(group), dist.get_rank(group)
-    qkv_shape, merged_shape = peer_buffer_shapes(total, heads, head_dim, n_ranks)
-    qkv = symm.empty(qkv_shape, dtype=torch.bfloat16, device=device)
-    merged = symm.empty(merged_shape, dtype=out_dtype, device=device)
+    qkv_shape, merged_shape = peer_buffer_shapes(total, heads, head_dim, n_ranks, qkv_record_bytes, out_record_bytes)
+    qkv = symm.empty(qkv_shape, dtype=torch.uint8 if qkv_record_bytes else torch.bfloat16, device=device)
+    merged = symm.empty(merged_shape, dtype=torch.uint8 if out_record_bytes else out_dtype, device=device)
     gname = (group or dist.group.WORLD).group_name
     hq, hm = symm.rendezvous(qkv, gname), symm.rendezvous(merged, gname)
     token = torch.zeros(1, dtype=torch.int32, device=device)
@@ -108,12 +115,15 @@ def symmetric_memory_buffers(total, heads, head_dim, out_dtype, device, group=No
     return PeerBuffers(rank, n_ranks, qkv, merged, hq.buffer_ptrs, hm.buffer_ptrs, barrier, keep=(hq, hm, token))
 
 
-def local_peer_buffers(total, heads, head_dim, n_ranks, out_dtype, device) -> List[PeerBuffers]:
+def local_peer_buffers(total, heads, head_dim, n_ranks, out_dtype, device, qkv_record_bytes: int = 0,
+                       out_record_bytes: int = 0) -> List[PeerBuffers]:
     """All ranks' buffers on one device (one PeerBuffers per rank, sharing the address lists).  The ranks' phases
     are then run one after another on one stream, which orders them: the barrier is a no-op."""
-    qkv_shape, merged_shape = peer_buffer_shapes(total, heads, head_dim, n_ranks)
-    qkvs = [torch.empty(qkv_shape, dtype=torch.bfloat16, device=device) for _ in range(n_ranks)]
-    mergeds = [torch.empty(merged_shape, dtype=out_dtype, device=device) for _ in range(n_ranks)]
+    qkv_shape, merged_shape = peer_buffer_shapes(total, heads, head_dim, n_ranks, qkv_record_bytes, out_record_bytes)
+    qkvs = [torch.empty(qkv_shape, dtype=torch.uint8 if qkv_record_bytes else torch.bfloat16, device=device)
+            for _ in range(n_ranks)]
+    mergeds = [torch.empty(merged_shape, dtype=torch.uint8 if out_record_bytes else out_dtype, device=device)
+               for _ in range(n_ranks)]
     qp, mp = [t.data_ptr() for t in qkvs], [t.data_ptr() for t in mergeds]
     return [PeerBuffers(r, n_ranks, qkvs[r], mergeds[r], qp, mp, lambda: None) for r in range(n_ranks)]
 
@@ -127,17 +137,21 @@ class _HeadGroup:
         self.qkv_send_splits, self.qkv_recv_splits, self.out_send_splits, self.out_recv_splits = xp.splits(count)
         st = (3 * count * D, D)
         self.attn = B.Attn3d(seqs, count, D, rope_dims, theta, device, q_strides=st, k_strides=st, v_strides=st)
-        self.qkv = torch.empty((total, 3, count, D), dtype=torch.bfloat16, device=device)
         if sp.qkv_int8:
+            # records arrive and feed the attention as they are: the rotary producer dequantises (Q~, K~ into the plan's
+            # workspace, V into this scratch); no packed bf16 QKV tensor exists on this side
             self.send = torch.empty((G, n_local, count, sp.rb_in), dtype=torch.uint8, device=device)
             self.qkv_records = torch.empty((total, count, sp.rb_in), dtype=torch.uint8, device=device)
+            self.v_scratch = torch.empty((total, count, D), dtype=torch.bfloat16, device=device)
         else:
+            self.qkv = torch.empty((total, 3, count, D), dtype=torch.bfloat16, device=device)
             self.send = torch.empty((G, n_local, 3, count, D), dtype=torch.bfloat16, device=device)
-        self.out_shard = torch.empty((total, count, D), dtype=sp.out_dtype, device=device)
         if sp.out_int8:
-            self.out_records = torch.empty((total, count, sp.rb_out), dtype=torch.uint8, device=device)
+            # the attention epilogue writes the records that travel back
+            self.out_shard = torch.empty((total, count, sp.rb_out), dtype=torch.uint8, device=device)
             self.recv_out = torch.empty((G, n_local, count, sp.rb_out), dtype=torch.uint8, device=device)
         else:
+            self.out_shard = torch.empty((total, count, D), dtype=sp.out_dtype, device=device)
             self.recv_out = torch.empty((G, n_local, count, D), dtype=sp.out_dtype, device=device)
         self.ev_in = torch.cuda.Event()
         self.ev_out = torch.cuda.Event()
@@ -173,8 +187,8 @@ class SequenceParallelAttn3d:
             raise ValueError("qkv_wire: 'bf16' or 'int8'")
         if transport not in ("collective", "peer"):
             raise ValueError("transport: 'collective' or 'peer'")
-        if transport == "peer" and (qkv_wire != "bf16" or out_format == "int8" or n_groups != 1):
-            raise ValueError("transport 'peer' carries bf16 QKV and bf16 / e4m3 output, in one group")
+        if transport == "peer" and n_groups != 1:
+            raise ValueError("transport 'peer' works in one head group")
         self.fp8 = out_format == "e4m3"
         self.out_int8 = out_format == "int8"
         self.qkv_int8 = qkv_wire == "int8"
@@ -201,30 +215,46 @@ class SequenceParallelAttn3d:
             qkv_strides = (3 * hl * D, D)
             self.attn = B.Attn3d(seqs, hl, D, rope_dims, theta, device, q_strides=qkv_strides, k_strides=qkv_strides,
                                  v_strides=qkv_strides)
+            rb_q = self.rb_in if self.qkv_int8 else 0
+            rb_o = self.rb_out if self.out_int8 else 0
             self.pb = peer_buffers if peer_buffers is not None else symmetric_memory_buffers(
-                total, heads, D, self.out_dtype, device, group)
-            qkv_shape, merged_shape = peer_buffer_shapes(total, heads, D, self.n_ranks)
+                total, heads, D, self.out_dtype, device, group, rb_q, rb_o)
+            qkv_shape, merged_shape = peer_buffer_shapes(total, heads, D, self.n_ranks, rb_q, rb_o)
             if tuple(self.pb.qkv.shape) != qkv_shape or tuple(self.pb.merged.shape) != merged_shape or \
-                    self.pb.merged.dtype != self.out_dtype or len(self.pb.qkv_peers) != self.n_ranks or \
-                    len(self.pb.merged_peers) != self.n_ranks:
+                    self.pb.merged.dtype != (torch.uint8 if rb_o else self.out_dtype) or \
+                    len(self.pb.qkv_peers) != self.n_ranks or len(self.pb.merged_peers) != self.n_ranks:
                 raise ValueError("peer buffers do not fit this problem")
 
     # ---- peer transport, phase by phase (forward() runs them with barriers in between)
     def peer_pack(self, q, k, v):
-        """Phase 1: this rank's Q, K, V rows go straight into every owner's receive buffer."""
-        B.sol_attn3d_exchange_pack_qkv(q, k, v, self.n_ranks, self.pb.qkv_peers, self.xp.first_token)
+        """Phase 1: this rank's Q, K, V rows go straight into every owner's receive buffer (as bf16 rows, or quantised to
+        block-INT8 records on the way)."""
+        pack = B.sol_attn3d_exchange_pack_qkv_int8 if self.qkv_int8 else B.sol_attn3d_exchange_pack_qkv
+        pack(q, k, v, self.n_ranks, self.pb.qkv_peers, self.xp.first_token)
 
     def peer_attend(self, key_mask=None):
         """Phase 2 (after every rank's phase 1): attention over this rank's head shard; the epilogue stores each
         output row into its token owner's merged buffer, at this shard's head offset."""
         qkv = self.pb.qkv
+        fmt = B.OUT_INT8 if self.out_int8 else B.OUT_E4M3 if self.fp8 else B.OUT_BF16
+        if self.qkv_int8:
+            # the scatter entry point takes bf16 views: dequantise the records this rank received (its own buffer) first
+            bf = torch.empty((self.xp.total, 3, self.xp.hl, self.head_dim), dtype=torch.bfloat16, device=qkv.device)
+            B.sol_attn3d_exchange_unpack_qkv_int8(qkv, bf, self.xp.total, self.xp.hl, self.head_dim)
+            qkv = bf
         B.sol_attn3d_forward_scatter(self.attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], key_mask, self.pb.merged_peers,
-                                     self.xp.tok_begin, self.heads, self.rank * self.xp.hl,
-                                     B.OUT_E4M3 if self.fp8 else B.OUT_BF16)
+                                     self.xp.tok_begin, self.heads, self.rank * self.xp.hl, fmt)
 
     def peer_result(self):
-        """Phase 3 (after every rank's phase 2): this rank's token rows, all heads."""
-        return self.pb.merged[:self.xp.n_local]
+        """Phase 3 (after every rank's phase 2): this rank's token rows, all heads (block-INT8 records are dequantised
+        to bf16 rows here, on arrival)."""
+        rows = self.pb.merged[:self.xp.n_local]
+        if not self.out_int8:
+            return rows
+        out = torch.empty((self.xp.n_local, self.heads, self.head_dim), dtype=torch.bfloat16, device=rows.device)
+        if self.xp.n_local:
+            B.sol_attn3d_exchange_dequantize_out_int8(rows.contiguous(), out)
+        return out
 
     def forward(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, key_mask: Optional[torch.Tensor] = None) -> torch.Tensor:
         """q, k, v: [n_local, heads, D] bf16 (any strides, e.g. views into packed QKV); key_mask: uint8 [total] or None."""
@@ -260,7 +290,6 @@ class SequenceParallelAttn3d:
                     B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, G, dsts, 0, group_begin=gr.begin, group_heads=gr.count)
                     self.dist.all_to_all_single(gr.qkv_records.view(-1), gr.send.view(-1), gr.qkv_recv_splits,
                                                 gr.qkv_send_splits, group=self.group)
-                    B.sol_attn3d_exchange_unpack_qkv_int8(gr.qkv_records, gr.qkv, xp.total, gr.count, D)
                 else:
                     B.sol_attn3d_exchange_pack_qkv(q, k, v, G, dsts, 0, group_begin=gr.begin, group_heads=gr.count)
                     self.dist.all_to_all_single(gr.qkv.view(-1), gr.send.view(-1), gr.qkv_recv_splits, gr.qkv_send_splits,
@@ -269,15 +298,18 @@ class SequenceParallelAttn3d:
         # (2) attention group by group on the caller's stream; (3) each group's output returns on the output stream
         for gr in self.groups:
             cur.wait_event(gr.ev_in)
-            qv, kv, vv = gr.qkv[:, 0], gr.qkv[:, 1], gr.qkv[:, 2]
-            if self.fp8:
-                B.sol_attn3d_forward_e4m3(gr.attn.plan, qv, kv, vv, gr.out_shard, key_mask)
+            fmt = B.OUT_INT8 if self.out_int8 else B.OUT_E4M3 if self.fp8 else B.OUT_BF16
+            if self.qkv_int8:
+                B.sol_attn3d_forward_qkv_int8(gr.attn.plan, gr.qkv_records, gr.v_scratch, gr.out_shard, key_mask, fmt)
             else:
-                B.sol_attn3d_forward(gr.attn.plan, qv, kv, vv, gr.out_shard, key_mask)
+                qv, kv, vv = gr.qkv[:, 0], gr.qkv[:, 1], gr.qkv[:, 2]
+                if self.out_int8:
+                    B.sol_attn3d_forward_int8(gr.attn.plan, qv, kv, vv, gr.out_shard, key_mask)
+                elif self.fp8:
+                    B.sol_attn3d_forward_e4m3(gr.attn.plan, qv, kv, vv, gr.out_shard, key_mask)
+                else:
+                    B.sol_attn3d_forward(gr.attn.plan, qv, kv, vv, gr.out_shard, key_mask)
             wire = gr.out_shard
-            if self.out_int8:
-                B.sol_attn3d_exchange_quantize_out_int8(gr.out_shard, gr.out_records)
-                wire = gr.out_records
             gr.ev_out.record(cur)
             with torch.cuda.stream(self.s_out):
                 self.s_out.wait_event(gr.ev_out)

@@ -420,13 +420,10 @@ def test_int8_output_records_are_bit_exact(B, n, heads, D):
     assert torch.equal(back.cpu().view(torch.int16), xo.out_from_records(want, D).to(torch.bfloat16).view(torch.int16))
 
 
-def test_exchange_with_int8_wire_formats(B):
-    """Whole exchange, 4 virtual ranks, block-INT8 both ways.  Approximate by design, so two checks: the GPU
-    pipeline equals the oracle pipeline fed with the same records (attention tolerance), and the end result stays
-    within the quantisation error of the unquantised attention."""
-    w = replace(wl.shrunk("lowres"), heads=8)
-    inp = wl.make_inputs(w, "cuda")
-    G, total, heads, D = 4, w.total_tokens, w.heads, w.head_dim
+def int8_pipeline_by_hand(B, w, inp, G):
+    """Whole exchange with block-INT8 records both ways, G virtual ranks, every kernel called by hand.  Returns (per-rank
+    bf16 rows, per-rank oracle attention of the dequantised inputs)."""
+    total, heads, D = w.total_tokens, w.heads, w.head_dim
     hl = heads // G
     ranges = xo.shard_ranges(total, G)
     rb_in = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)
@@ -452,7 +449,8 @@ def test_exchange_with_int8_wire_formats(B):
         attn.close()
         # oracle attention on the dequantised (bf16-rounded) inputs the GPU attention saw
         dq = [x.to(torch.bfloat16) for x in xo.qkv_from_records(want_rec[:, r * hl:(r + 1) * hl].contiguous(), D)]
-        ref = orc.attn3d_oracle(dq[0], dq[1], dq[2], seq_tuples(w), w.rope_dims, w.theta, None)
+        ref = orc.attn3d_oracle(dq[0], dq[1], dq[2], seq_tuples(w), w.rope_dims, w.theta,
+                                None if inp.key_mask is None else inp.key_mask.cpu())
         max_abs, rel_l2 = orc.compare(shard.cpu(), ref)
         assert max_abs <= TOL_MAX_ABS and rel_l2 <= TOL_REL_L2, (max_abs, rel_l2)
         assert torch.equal(rec.cpu(), xo.out_records(shard.cpu()))
@@ -467,6 +465,17 @@ def test_exchange_with_int8_wire_formats(B):
         B.sol_attn3d_exchange_dequantize_out_int8(merged, rows)
         outs.append(rows)
     torch.cuda.synchronize()
+    return outs, ref_shards
+
+
+def test_exchange_with_int8_wire_formats(B):
+    """Whole exchange, 4 virtual ranks, block-INT8 both ways.  Approximate by design, so two checks: the GPU
+    pipeline equals the oracle pipeline fed with the same records (attention tolerance), and the end result stays
+    within the quantisation error of the unquantised attention."""
+    w = replace(wl.shrunk("lowres"), heads=8)
+    inp = wl.make_inputs(w, "cuda")
+    total, heads, D = w.total_tokens, w.heads, w.head_dim
+    outs, ref_shards = int8_pipeline_by_hand(B, w, inp, 4)
     got = torch.cat(outs, 0).cpu().double()
     # against the oracle of the same pipeline: attention error + half an output step
     ref_pipeline = torch.cat(ref_shards, dim=1)
@@ -536,7 +545,7 @@ def test_full_size_lowres_e4m3_and_scatter_sampled_rows(B):
 
 # ------------------------------------------------------------------------------------------ peer transport, the module's own code
 @pytest.mark.parametrize("name,heads,G,fmt", [("lowres", 8, 4, "bf16"), ("varlen", 6, 3, "bf16"), ("cfg_batch", 8, 8, "bf16"),
-                                              ("lowres", 8, 2, "e4m3")])
+                                              ("lowres", 8, 2, "e4m3"), ("lowres", 8, 4, "int8"), ("cfg_batch", 4, 2, "int8")])
 def test_peer_transport_of_the_module_with_virtual_ranks(B, name, heads, G, fmt):
     """SequenceParallelAttn3d(transport="peer") with all ranks' buffers on this GPU (local_peer_buffers): every rank
     is an instance of the module, and the ranks run its three phases in turn -- all pack, all attend, all read --
@@ -547,12 +556,16 @@ def test_peer_transport_of_the_module_with_virtual_ranks(B, name, heads, G, fmt)
     w = replace(wl.shrunk(name), heads=heads)
     inp = wl.make_inputs(w, "cuda")
     out_dtype = torch.uint8 if fmt == "e4m3" else torch.bfloat16
-    bufs = local_peer_buffers(w.total_tokens, heads, w.head_dim, G, out_dtype, "cuda")
+    int8 = fmt == "int8"                                       # block-INT8 records both ways
+    rb_q = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, w.head_dim) if int8 else 0
+    rb_o = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, w.head_dim) if int8 else 0
+    bufs = local_peer_buffers(w.total_tokens, heads, w.head_dim, G, out_dtype, "cuda", rb_q, rb_o)
     for pb in bufs:                                            # poison: an unwritten element shows
-        pb.qkv.fill_(float("nan"))
+        pb.qkv.view(torch.uint8).fill_(0x7F)
         pb.merged.view(torch.uint8).fill_(0x7F)
+    kw = {"qkv_wire": "int8"} if int8 else {}
     ranks = [SequenceParallelAttn3d(seq_tuples(w), heads, w.head_dim, w.rope_dims, w.theta, transport="peer", out_format=fmt,
-                                    peer_buffers=bufs[r]) for r in range(G)]
+                                    peer_buffers=bufs[r], **kw) for r in range(G)]
     ranges = shard_ranges(w.total_tokens, G)
     for r, (a, b) in enumerate(ranges):
         assert ranks[r].xp.n_local == b - a
@@ -565,6 +578,13 @@ def test_peer_transport_of_the_module_with_virtual_ranks(B, name, heads, G, fmt)
         assert ranks[r].attn.status() == 0
     got = torch.cat([ranks[r].peer_result() for r in range(G)], dim=0)
     assert got.shape[0] == w.total_tokens
+    if int8:
+        # the same records, kernels and arithmetic as the pipeline called by hand: the same bytes
+        by_hand, _ = int8_pipeline_by_hand(B, w, inp, G)
+        assert torch.equal(got, torch.cat(by_hand, dim=0))
+        for r in ranks:
+            r.close()
+        return
     single = B.Attn3d.from_workload(w, "cuda")
     if fmt == "e4m3":
         want = torch.empty((w.total_tokens, heads, w.head_dim), dtype=torch.uint8, device="cuda")
@@ -632,3 +652,108 @@ def test_peer_transport_with_symmetric_memory_one_rank(B):
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     res = subprocess.run([sys.executable, "-c", _PEER_ONE_RANK], cwd=root, env=env, capture_output=True, text=True, timeout=300)
     assert res.returncode == 0 and "PEER_ONE_RANK_OK" in res.stdout, res.stdout[-2000:] + res.stderr[-4000:]
+
+
+# ------------------------------------------------------------------------------------------ wire formats fused into the neighbours
+@pytest.mark.parametrize("name", ["tiny", "cfg_batch", "varlen"])
+def test_int8_epilogue_equals_quantising_the_bf16_rows(B, name):
+    """sol_attn3d_forward_int8: the attention epilogue writes the output records itself.  Byte for byte the records of
+    the two-kernel path (bf16 rows, then the record kernel), and of the oracle's record rule applied to those rows;
+    the rows are pinned against the attention oracle."""
+    w = wl.shrunk(name)
+    inp = wl.make_inputs(w, "cuda")
+    D = w.head_dim
+    rb = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, D)
+    attn = B.Attn3d.from_workload(w, "cuda")
+    rows = attn.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    two = torch.empty((w.total_tokens, w.heads, rb), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_quantize_out_int8(rows, two)
+    fused = torch.full((w.total_tokens + 2, w.heads, rb), 0xAB, dtype=torch.uint8, device="cuda")   # guard rows around
+    B.sol_attn3d_forward_int8(attn.plan, inp.q, inp.k, inp.v, fused[1:-1], inp.key_mask)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert bool((fused[0] == 0xAB).all()) and bool((fused[-1] == 0xAB).all())
+    assert torch.equal(fused[1:-1], two)
+    assert torch.equal(fused[1:-1].cpu(), xo.out_records(rows.cpu()))
+    ma, rl = orc.compare(rows.cpu(), oracle_dense(w, inp))
+    assert ma <= TOL_MAX_ABS and rl <= TOL_REL_L2
+    # scattered to three owners at a head offset, records
+    total = w.total_tokens
+    tb = [0, total // 3, total // 3, total]
+    owners = [torch.full((max(tb[g + 1] - tb[g], 1), w.heads + 1, rb), 0xCD, dtype=torch.uint8, device="cuda") for g in range(3)]
+    B.sol_attn3d_forward_scatter(attn.plan, inp.q, inp.k, inp.v, inp.key_mask, [o.data_ptr() for o in owners], tb,
+                                 w.heads + 1, 1, B.OUT_INT8)
+    torch.cuda.synchronize()
+    got = torch.cat([owners[g][: tb[g + 1] - tb[g], 1:] for g in range(3)])
+    assert torch.equal(got, two)
+    assert all(bool((owners[g][:, 0] == 0xCD).all()) for g in range(3))
+    attn.close()
+
+
+def test_int8_epilogue_writes_zero_records_for_a_sequence_without_keys(B):
+    w = wl.Workload(name="dead", seqs=(wl.SeqSpec(40, 0, 1, 1), wl.SeqSpec(3, 2, 5, 7)), heads=2, head_dim=128,
+                    rope_dims=(32, 48, 48), seed=11)
+    inp = wl.make_inputs(w, "cuda")
+    mask = torch.ones(w.total_tokens, dtype=torch.uint8, device="cuda")
+    mask[40:] = 0
+    attn = B.Attn3d.from_workload(w, "cuda")
+    rows = attn.forward(inp.q, inp.k, inp.v, mask)
+    rb = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, 128)
+    fused = torch.empty((w.total_tokens, w.heads, rb), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_forward_int8(attn.plan, inp.q, inp.k, inp.v, fused, mask)
+    torch.cuda.synchronize()
+    assert torch.equal(fused.cpu(), xo.out_records(rows.cpu()))
+    attn.close()
+
+
+@pytest.mark.parametrize("name,heads", [("tiny", 4), ("lowres", 5), ("cfg_batch", 2), ("varlen", 3)])
+def test_qkv_int8_records_feed_the_attention_directly(B, name, heads):
+    """sol_attn3d_forward_qkv_int8: the rotary producer dequantises the records itself.  Bit for bit the result of
+    unpacking the records into a bf16 QKV tensor and running the plain forward on its views, for every output format;
+    and within the attention tolerance of the oracle run on the oracle's own dequantisation of the oracle's records."""
+    w = replace(wl.shrunk(name), heads=heads)
+    inp = wl.make_inputs(w, "cuda")
+    total, D = w.total_tokens, w.head_dim
+    rb_in = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)
+    rb_out = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, D)
+    rec = torch.empty((total, heads, rb_in), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_pack_qkv_int8(inp.q, inp.k, inp.v, 1, [rec.data_ptr()], 0)
+    torch.cuda.synchronize()
+    assert torch.equal(rec.cpu(), xo.qkv_records(inp.q.cpu(), inp.k.cpu(), inp.v.cpu()))
+    # two-kernel path
+    qkv = torch.empty((total, 3, heads, D), dtype=torch.bfloat16, device="cuda")
+    B.sol_attn3d_exchange_unpack_qkv_int8(rec, qkv, total, heads, D)
+    st = (3 * heads * D, D)
+    a2 = B.Attn3d(seq_tuples(w), heads, D, w.rope_dims, w.theta, "cuda", q_strides=st, k_strides=st, v_strides=st)
+    want = a2.forward(qkv[:, 0], qkv[:, 1], qkv[:, 2], inp.key_mask)
+    want8 = torch.empty(want.shape, dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_forward_e4m3(a2.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], want8, inp.key_mask)
+    wantr = torch.empty((total, heads, rb_out), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_quantize_out_int8(want, wantr)
+    # fused path, on a plan with the default strides (the records carry their own layout)
+    attn = B.Attn3d.from_workload(w, "cuda")
+    v_scratch = torch.full((total, heads, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    got = torch.full_like(want, float("nan"))
+    B.sol_attn3d_forward_qkv_int8(attn.plan, rec, v_scratch, got, inp.key_mask, B.OUT_BF16)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert torch.equal(v_scratch, qkv[:, 2])
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    got8 = torch.empty_like(want8)
+    B.sol_attn3d_forward_qkv_int8(attn.plan, rec, v_scratch, got8, inp.key_mask, B.OUT_E4M3)
+    gotr = torch.empty_like(wantr)
+    B.sol_attn3d_forward_qkv_int8(attn.plan, rec, v_scratch, gotr, inp.key_mask, B.OUT_INT8)
+    torch.cuda.synchronize()
+    assert torch.equal(got8, want8) and torch.equal(gotr, wantr)
+    # the plain forward still works on the same plan afterwards (the cached V map is re-encoded)
+    plain = attn.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    torch.cuda.synchronize()
+    ma, rl = orc.compare(plain.cpu(), oracle_dense(w, inp))
+    assert ma <= TOL_MAX_ABS and rl <= TOL_REL_L2
+    # oracle: its own records, its own dequantisation (rounded to bf16 as the wire tensor would be), its attention
+    dq = [x.to(torch.bfloat16) for x in xo.qkv_from_records(xo.qkv_records(inp.q.cpu(), inp.k.cpu(), inp.v.cpu()), D)]
+    ref = orc.attn3d_oracle(dq[0], dq[1], dq[2], seq_tuples(w), w.rope_dims, w.theta,
+                            None if inp.key_mask is None else inp.key_mask.cpu())
+    ma, rl = orc.compare(got.cpu(), ref)
+    assert ma <= TOL_MAX_ABS and rl <= TOL_REL_L2, (ma, rl)
+    attn.close(); a2.close()
