@@ -265,7 +265,7 @@ def main():
                     help="time sol_attn3d_forward_qknorm (QK RMS-norm fused into the rotary producer) instead")
     ap.add_argument("--exchange", type=int, default=0, metavar="G",
                     help="instead of the forward: time one rank's kernels of a G-way sequence-parallel exchange "
-                         "(Section 3.3) at the workload's shape and print their ms and GB/s")
+                         "(Section 3.2) at the workload's shape and print their ms and GB/s")
     ap.add_argument("--exchange-kernel", default="all",
                     help="with --exchange: run only this kernel (e.g. for a profiler capture)")
     args = ap.parse_args()
@@ -475,14 +475,14 @@ def main():
         q_cpu, k_cpu, v_cpu = inp.q.cpu(), inp.k.cpu(), inp.v.cpu()
         mask_cpu = None if inp.key_mask is None else inp.key_mask.cpu()
         select, picked = [], []
-        for h in sorted({0, w.heads // 2, w.heads - 1}):
+        for h in sorted({0, w.heads - 1}):
             sq0 = w.seqs[0]
             nq, nk = (sq0.n_tokens + 255) // 256, (sq0.n_tokens + 127) // 128
             m = torch.zeros(nq, nk, dtype=torch.bool)
             for i in range(nq):
                 m[i, B.sol_attn3d_sparse_selection(attn.plan, sparse_ws, 0, h, i, nk)] = True
             picked.append(m)
-            select.append((0, h, torch.from_numpy(wl.sample_rows(w, 0, h, 256))))
+            select.append((0, h, torch.from_numpy(wl.sample_rows(w, 0, h, 96))))
         t0 = time.perf_counter()
         ref, _, _ = orc.attn3d_sparse_oracle(q_cpu, k_cpu, v_cpu, seqs, w.rope_dims, w.theta, args.sparse_tau, 256, 128,
                                              mask_cpu, selection=picked, select=select)
@@ -493,7 +493,7 @@ def main():
         kept = sum(float(m.float().mean()) for m in picked) / len(picked)
         fl = sum(4.0 * len(r_) * w.seqs[0].n_tokens * w.head_dim for (_, _, r_) in select) * kept
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "seconds": dt,
-               "sample": f"{len(select)} heads x 256 query rows of sequence 0 over the KV blocks the GPU selected (fp64)"}
+               "sample": f"{len(select)} heads x 96 query rows of sequence 0 over the KV blocks the GPU selected (fp64)"}
         parity = {"max_abs": ma, "rel_l2": rl, "rows": int(got.shape[0]), "tol_max_abs": 2e-2, "tol_rel_l2": 5e-3,
                   "ok": bool(ma <= 2e-2 and rl <= 5e-3), "selection": "the GPU's own, read back per (head, query block)"}
     if not args.no_cpu_baseline and world == 1 and args.sparse_tau is None:

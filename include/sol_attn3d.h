@@ -173,8 +173,8 @@ int sol_attn3d_forward_rect(sol_attn3d_plan_t plan, const void* q, const void* k
                             const uint8_t* key_mask, const uint8_t* query_mask, sol_attn3d_stream_t stream);
 
 /*
- * sol_attn3d_forward with the FP8 output format of Section 3.3 ("Quantized communication": the FP8
- * alternative transmits 128 raw E4M3 bytes per token/head, without scale metadata or padding; "Joint
+ * sol_attn3d_forward with the FP8 output format of Section 3.2 ("Quantized communication": the FP8
+ * alternative transmits 128 raw E4M3 bytes per token/head, without scale metadata or padding; Section 3.3, "Joint
  * optimization with quantized communication": the raw E4M3 values returned by attention feed the quantized
  * output projection with unit scales).  The epilogue converts O/l from fp32 straight to E4M3 (round to
  * nearest even, magnitudes above 448 saturate, no bf16 step in between).
@@ -186,7 +186,7 @@ int sol_attn3d_forward_e4m3(sol_attn3d_plan_t plan, const void* q, const void* k
                             const uint8_t* key_mask, sol_attn3d_stream_t stream);
 
 /*
- * Sequence-parallel exchange around the attention (Section 3.3, "Optimized attention collectives"): ranks
+ * Sequence-parallel exchange around the attention (Section 3.2, "Optimized attention collectives"): ranks
  * hold contiguous ranges of the flat token axis with all heads; attention needs every token for a shard of
  * the heads.  The paper's path is pack -> all-to-all -> attention -> all-to-all -> head merge with ONE
  * collective each way; the two layout kernels below are bit-exact copies of 16-byte chunks.
@@ -234,7 +234,7 @@ int sol_attn3d_exchange_merge_heads(const void* recv, void* out, int64_t n_local
                                     sol_attn3d_stream_t stream);
 
 /*
- * Quantized wire formats of the exchange (Section 3.3, "Quantized communication").  One record per (token,
+ * Quantized wire formats of the exchange (Section 3.2, "Quantized communication").  One record per (token,
  * head); head_dim 64 or 128:
  *   QKV block-INT8   [q int8 x D | k int8 x D | v int8 x D | D/32 q scale codes | D/32 k codes | D/32 v codes |
  *                    zeros to a multiple of 16 bytes]                      D = 128: 384 + 12 + 4 = 400 bytes
@@ -283,9 +283,9 @@ int sol_attn3d_exchange_dequantize_out_int8(const void* records, void* out_rows,
                                             sol_attn3d_stream_t stream);
 
 /*
- * sol_attn3d_forward with the block-INT8 output format of Section 3.3 ("Quantized communication": a 144-byte record
- * per token and head at head_dim 128) written by the attention epilogue itself, the fusion that the paper's "Joint
- * optimization with quantized communication" aims at: the bf16 rows are never written or re-read.  The values are
+ * sol_attn3d_forward with the block-INT8 output format of Section 3.2 ("Quantized communication": a 144-byte record
+ * per token and head at head_dim 128) written by the attention epilogue itself, the kind of fusion that Section 3.3
+ * ("Joint optimization with quantized communication") aims at: the bf16 rows are never written or re-read.  The values are
  * rounded to bf16 and quantised by the rule stated above, so the records are byte for byte those of
  * sol_attn3d_forward followed by sol_attn3d_exchange_quantize_out_int8.
  *   out_records  DEVICE pointer, dense [total_tokens][heads][sol_attn3d_exchange_record_bytes(OUT_INT8, head_dim)]
@@ -296,8 +296,8 @@ int sol_attn3d_forward_int8(sol_attn3d_plan_t plan, const void* q, const void* k
                             const uint8_t* key_mask, sol_attn3d_stream_t stream);
 
 /*
- * sol_attn3d_forward fed by the block-INT8 QKV records of the exchange (Section 3.3, "Quantized communication"): the
- * receiver's dequantisation is fused into the rotary producer ("Joint optimization with quantized communication"),
+ * sol_attn3d_forward fed by the block-INT8 QKV records of the exchange (Section 3.2, "Quantized communication"): the
+ * receiver's dequantisation is fused into the rotary producer (Section 3.3, "Joint optimization with quantized communication"),
  * so the packed bf16 QKV tensor is never written or re-read.  Each value is q * s rounded to bf16, exactly what
  * sol_attn3d_exchange_unpack_qkv_int8 would have stored, and Q, K are rotated from there: the result is bit for bit
  * that of unpack followed by sol_attn3d_forward on the unpacked views.

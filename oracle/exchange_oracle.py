@@ -3,8 +3,8 @@
 Never on the product path: only tests, the smoke check and the benchmark's CPU-baseline leg may import it.  It
 shares no code, tables or constants with the CUDA sources and imports nothing from the package.
 
-What it states (Section 3.3 of the paper, "Optimized attention collectives", "Quantized communication" and
-"Joint optimization with quantized communication"):
+What it states (Section 3.2 of the paper, "Optimized attention collectives" and "Quantized communication", and
+Section 3.3, "Joint optimization with quantized communication"):
 
   X1  sequence-sharded layout: rank g of G holds a contiguous range of the flat token axis, all heads,
       tensors [n_g, heads, D] (the flat (total, heads, head_dim) layout; no batch dimension);
@@ -141,7 +141,7 @@ def ulysses_reference(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, G: int,
 
 # --------------------------------------------------------------------------------------------- block-INT8 wire formats
 #
-# Section 3.3, "Quantized communication".  What the paper fixes: the QKV record of one (token, head) is 384 int8
+# Section 3.2, "Quantized communication".  What the paper fixes: the QKV record of one (token, head) is 384 int8
 # values, twelve scale codes (one per group of 32 values, "finite-positive UE5M3"), four zero bytes = 400 bytes; the
 # output record is 128 values, four scale codes, padded from 132 to 144 bytes; all padding bytes are written.
 # What it leaves open, and the reading taken here (X8-X11):

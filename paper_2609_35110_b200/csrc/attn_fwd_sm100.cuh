@@ -139,7 +139,7 @@ __device__ __forceinline__ void store_rows(const AttnParams& p, const SeqDev& sq
   }
 }
 
-// Epilogue in the block-INT8 wire format of the exchange (Section 3.3, "Quantized communication"): the thread that owns
+// Epilogue in the block-INT8 wire format of the exchange (Section 3.2, "Quantized communication"): the thread that owns
 // an accumulator row writes that row's record, [D int8 | D/32 scale codes | zeros to a multiple of 16 bytes], straight
 // from tensor memory.  A group of 32 values is exactly one 32-column load.  The values are first rounded to bf16 and
 // then quantised by the rule of quantize_records_kernel, so the bytes equal those of the bf16 epilogue followed by that

@@ -1,4 +1,4 @@
-// Layout kernels of the sequence-parallel exchange around the attention (Section 3.3, "Optimized attention
+// Layout kernels of the sequence-parallel exchange around the attention (Section 3.2, "Optimized attention
 // collectives"): the stride-aware QKV pack that writes the exchange buffer in one pass, and the inverse head
 // merge on the return path.  Both move 16-byte chunks and change no byte.
 #pragma once
@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(256) exchange_merge_heads_kernel(const uint8_t
 }
 
 // ---------------------------------------------------------------------------------------------
-// Block-INT8 wire formats (Section 3.3, "Quantized communication").  One (token, head) record:
+// Block-INT8 wire formats (Section 3.2, "Quantized communication").  One (token, head) record:
 //   QKV:    [q int8 x D | k int8 x D | v int8 x D | D/32 q scale codes | D/32 k codes | D/32 v codes | zeros]
 //           padded to a multiple of 16 bytes (D = 128: 384 + 12 + 4 = 400 bytes);
 //   output: [o int8 x D | D/32 scale codes | zeros] padded likewise (D = 128: 128 + 4 + 12 = 144 bytes).

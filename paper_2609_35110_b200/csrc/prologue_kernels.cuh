@@ -207,8 +207,8 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// The same producer fed by the block-INT8 QKV records of the exchange (Section 3.3, "Quantized communication"; the
-// fusion of the receiver's dequantisation into the consumer is what "Joint optimization with quantized
+// The same producer fed by the block-INT8 QKV records of the exchange (Section 3.2, "Quantized communication"; the
+// fusion of the receiver's dequantisation into the consumer is what Section 3.3, "Joint optimization with quantized
 // communication" asks for): records [token][head][q int8 x D | k | v | 3 D/32 scale codes | pad] -> rotated Q~, K~
 // and plain V, all bf16 [token][head][D].  value = q * s is rounded to bf16 first and rotated then, so Q~ and K~ are
 // bit for bit what dequantize_records_kernel followed by rope_qk_kernel produce; the packed bf16 QKV tensor in

@@ -1,4 +1,4 @@
-"""Sequence-parallel attention (Section 3.3 of the paper): every rank holds a contiguous range of the flat token
+"""Sequence-parallel attention (Section 3.2 of the paper): every rank holds a contiguous range of the flat token
 axis with all heads; attention runs head-sharded between two exchanges.
 
 Plumbing only: `torch.distributed` carries the two all-to-alls (NCCL on GPUs), every byte that moves on the

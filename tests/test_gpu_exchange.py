@@ -1,4 +1,4 @@
-"""GPU: E4M3 output epilogue and the sequence-parallel exchange kernels (Section 3.3 of the paper).
+"""GPU: E4M3 output epilogue and the sequence-parallel exchange kernels (Section 3.2 of the paper).
 
 One GPU stands in for the G ranks: their shards and buffers all live on it and the kernels of the "ranks" run one
 after another (nothing waits on anything), which exercises exactly the addresses a real run would use with peer

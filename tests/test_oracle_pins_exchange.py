@@ -1,4 +1,4 @@
-"""Pins for the exchange / FP8-output oracle (Section 3.3: attention collectives and quantized communication).
+"""Pins for the exchange / FP8-output oracle (Section 3.2: attention collectives and quantized communication).
 CPU only.  None of them re-types the oracle's formula: code values are the format's published constants,
 nearest-code is a brute-force search, the cast is re-checked against the library's own, the permutations are
 pure-Python index loops, and the end-to-end identity is checked against the single-device attention."""
