@@ -459,6 +459,8 @@ def main():
     long_step = total_ms > 1000.0
     peak = peaks["sustained"] if long_step else peaks["burst"]
     traffic, traffic_note = load_ncu_traffic(w.name)
+    if args.sparse_tau is not None:         # the capture is of the dense launch; the sparse one was not captured
+        traffic, traffic_note = None, "not captured for the block-sparse launch"
     # cycles of one attention launch at the SM clock sampled during the timed region: separates gains in the
     # dependency chain (fewer cycles) from gains in power (more MHz under the cap)
     sm_mhz = clocks.get("sm_mhz") if clocks else None
@@ -493,7 +495,8 @@ def main():
         kept = sum(float(m.float().mean()) for m in picked) / len(picked)
         fl = sum(4.0 * len(r_) * w.seqs[0].n_tokens * w.head_dim for (_, _, r_) in select) * kept
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle", "seconds": dt,
-               "sample": f"{len(select)} heads x 96 query rows of sequence 0 over the KV blocks the GPU selected (fp64)"}
+               "sample": f"{len(select)} heads x 96 query rows of sequence 0 over the KV blocks the GPU selected (fp64); "
+                         "the time includes rotating every token of those heads"}
         parity = {"max_abs": ma, "rel_l2": rl, "rows": int(got.shape[0]), "tol_max_abs": 2e-2, "tol_rel_l2": 5e-3,
                   "ok": bool(ma <= 2e-2 and rl <= 5e-3), "selection": "the GPU's own, read back per (head, query block)"}
     if not args.no_cpu_baseline and world == 1 and args.sparse_tau is None:
