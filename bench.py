@@ -187,7 +187,11 @@ def exchange_bench(args, w, dev, B, peaks, config):
     rb_out = B.sol_attn3d_exchange_record_bytes(B.WIRE_OUT_INT8, D)
     send8 = torch.empty((G, n_local, hl, rb_in), dtype=torch.uint8, device=dev)
     qkv = torch.randn((total, 3, hl, D), generator=gen, device=dev).to(torch.bfloat16)
-    rec_in = torch.randint(1, 120, (total, hl, rb_in), generator=gen, device=dev, dtype=torch.uint8)
+    v_scratch = torch.empty((total, hl, D), dtype=torch.bfloat16, device=dev)
+    qkv_unpacked = torch.empty_like(qkv)     # the unpack kernel's own output: the attention below keeps its N(0,1) inputs
+    rec_in = torch.empty((total, hl, rb_in), device=dev, dtype=torch.uint8)
+    # realistic records: the N(0,1) QKV shard as a sender would have quantised it
+    B.sol_attn3d_exchange_pack_qkv_int8(qkv[:, 0], qkv[:, 1], qkv[:, 2], 1, [rec_in.data_ptr()], 0)
     shard = (0.1 * torch.randn((total, hl, D), generator=gen, device=dev)).to(torch.bfloat16)
     shard8 = torch.empty((total, hl, D), dtype=torch.uint8, device=dev)
     rec_out = torch.empty((total, hl, rb_out), dtype=torch.uint8, device=dev)
@@ -208,11 +212,16 @@ def exchange_bench(args, w, dev, B, peaks, config):
         "pack_qkv": (lambda: B.sol_attn3d_exchange_pack_qkv(q, k, v, G, sptr, 0), 2 * packed.numel() * bf),
         "merge_heads_bf16": (lambda: B.sol_attn3d_exchange_merge_heads(recv, merged, n_local, heads, D * bf, G), 2 * recv.numel() * bf),
         "pack_qkv_int8": (lambda: B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, G, sptr8, 0), packed.numel() * bf + send8.numel()),
-        "unpack_qkv_int8": (lambda: B.sol_attn3d_exchange_unpack_qkv_int8(rec_in, qkv, total, hl, D), rec_in.numel() + qkv.numel() * bf),
+        "unpack_qkv_int8": (lambda: B.sol_attn3d_exchange_unpack_qkv_int8(rec_in, qkv_unpacked, total, hl, D),
+                            rec_in.numel() + qkv.numel() * bf),
         "quantize_out_int8": (lambda: B.sol_attn3d_exchange_quantize_out_int8(shard, rec_out), shard.numel() * bf + rec_out.numel()),
         "dequantize_out_int8": (lambda: B.sol_attn3d_exchange_dequantize_out_int8(recv_rec, merged), recv_rec.numel() + merged.numel() * bf),
         "attention_shard_bf16": (lambda: B.sol_attn3d_forward(attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], shard, None), None),
         "attention_shard_e4m3": (lambda: B.sol_attn3d_forward_e4m3(attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], shard8, None), None),
+        # the wire formats fused into the neighbours (Section 3.3): INT8 records written by the attention epilogue, and
+        # the attention fed by INT8 QKV records (dequantised inside the rotary producer)
+        "attention_shard_int8_out": (lambda: B.sol_attn3d_forward_int8(attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], rec_out, None), None),
+        "attention_shard_from_int8_records": (lambda: B.sol_attn3d_forward_qkv_int8(attn.plan, rec_in, v_scratch, shard, None), None),
         "attention_shard_scatter": (lambda: B.sol_attn3d_forward_scatter(attn.plan, qkv[:, 0], qkv[:, 1], qkv[:, 2], None,
                                                                          [o.data_ptr() for o in owners], tok_begin, heads, 0), None),
     }
