@@ -339,16 +339,18 @@ int sol_attn3d_forward_scatter(sol_attn3d_plan_t plan, const void* q, const void
  * sol_attn3d_forward on HOST buffers: q, k, v are read from and out is written to host memory (pinned, or the
  * copies will not overlap), through caller-owned device staging memory.  The heads are served in n_groups
  * groups (heads are independent): the host-to-device copy of group g+1 and the device-to-host copy of group
- * g-1 run on two internal streams while the kernels of group g run on `stream`, so that only the first
- * group's inputs and the last group's outputs are exposed.  On return everything is enqueued; `stream` has
- * been made to wait for the last device-to-host copy, so synchronising `stream` is enough before reading out.
+ * g-1 run on two internal streams while the kernels of group g run, so that only the first group's inputs and
+ * the last group's outputs are exposed.  The kernels of even groups run on `stream`, those of odd groups on a
+ * third internal stream, so that a group's kernels fill the SMs that the last wave of its predecessor leaves
+ * idle.  On return everything is enqueued; `stream` has been made to wait for the last device-to-host copy, so
+ * synchronising `stream` is enough before reading out.
  *   q_host, k_host, v_host, out_host   HOST pointers, bf16, dense [total_tokens, heads, head_dim] (the plan must use
  *                  the default strides); key_mask_host HOST uint8 [total_tokens] or NULL.
  *   staging        DEVICE memory, 256-byte aligned, >= sol_attn3d_host_staging_bytes(plan) (four tensors and the
  *                  mask), caller-owned, must stay untouched until `stream` has passed this call.
- *   n_groups       1 .. 8 equal groups (clamped to the number of heads); 0 = default: six groups of growing and then
+ *   n_groups       1 .. 8 equal groups (clamped to the number of heads); 0 = default: eight groups of growing and then
  *                  shrinking size (a small first group, whose inputs are exposed, and a small last one, whose outputs are).
- * The first call creates two streams and a few events (no device memory); sol_attn3d_destroy releases them.
+ * The first call creates three streams and a few events (no device memory); sol_attn3d_destroy releases them.
  * Result: bit-identical to sol_attn3d_forward on device copies of the same tensors.
  * Errors: INVALID_ARG, NO_WORKSPACE (plan workspace or staging), UNSUPPORTED_SHAPE (strided plan), CUDA.
  */

@@ -71,8 +71,8 @@ struct sol_attn3d_plan_s {
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
   bool prof = false, prof_valid = false, prof_bits = false;
   // sol_attn3d_forward_host: copy streams and events, created on first use
-  cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
-  cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[8] = {}, ev_out[8] = {};
+  cudaStream_t s_h2d = nullptr, s_d2h = nullptr, s_alt = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_bits = nullptr, ev_in[8] = {}, ev_out[8] = {};
   bool host_pipe_ready = false;
   int sm_count = 148;                 // of the device the workspace was bound on
   int launches = 0;                   // kernels enqueued by the most recent forward-type call
@@ -90,15 +90,17 @@ int fail_cuda(sol_attn3d_plan_t p, cudaError_t e) {
 void release_host_pipe(sol_attn3d_plan_t p) {
   if (p->s_h2d != nullptr) (void)cudaStreamDestroy(p->s_h2d);
   if (p->s_d2h != nullptr) (void)cudaStreamDestroy(p->s_d2h);
+  if (p->s_alt != nullptr) (void)cudaStreamDestroy(p->s_alt);
   if (p->ev_start != nullptr) (void)cudaEventDestroy(p->ev_start);
   if (p->ev_done != nullptr) (void)cudaEventDestroy(p->ev_done);
+  if (p->ev_bits != nullptr) (void)cudaEventDestroy(p->ev_bits);
   for (int g = 0; g < 8; ++g) {
     if (p->ev_in[g] != nullptr) (void)cudaEventDestroy(p->ev_in[g]);
     if (p->ev_out[g] != nullptr) (void)cudaEventDestroy(p->ev_out[g]);
     p->ev_in[g] = p->ev_out[g] = nullptr;
   }
-  p->s_h2d = p->s_d2h = nullptr;
-  p->ev_start = p->ev_done = nullptr;
+  p->s_h2d = p->s_d2h = p->s_alt = nullptr;
+  p->ev_start = p->ev_done = p->ev_bits = nullptr;
   p->host_pipe_ready = false;
 }
 
@@ -461,6 +463,7 @@ struct FwdOpts {
   const void* qkv_records = nullptr;  // Q, K, V arrive as block-INT8 records (q and k are then NULL, v is a bf16 scratch)
   bool skip_keybits = false;          // the key-validity bits of this mask were built by an earlier call
   bool keep_launch_count = false;     // one of several launch sets of the same API call: keep counting
+  cudaEvent_t bits_done = nullptr;    // recorded on the stream once the key-validity bits are in place (built or kept)
   // Scratch other than the plan's bound workspace (sol_attn3d_forward_noalloc): the caller of forward_impl has put
   // the tables and the sequence table there; nothing about it is cached in the plan.
   unsigned char* ws = nullptr;
@@ -858,6 +861,7 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
     ++p->launches;
     if (own) p->keybits_state = key_mask ? 2 : 1;
   }
+  if (o.bits_done != nullptr && (e = cudaEventRecord(o.bits_done, st)) != cudaSuccess) return fail_cuda(p, e);
 
   if (p->prof && (e = cudaEventRecord(p->ev[1], st)) != cudaSuccess) return fail_cuda(p, e);
 
@@ -1160,12 +1164,12 @@ int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void*
   // head-group boundaries: equal groups when the caller names a count; by default a ramp (small first group:
   // its host-to-device copy is exposed; small last group: its device-to-host copy is) with larger groups between
   int bounds[9];
-  if (n_groups <= 0 && p->heads >= 12) {
-    static const int kRamp[7] = {0, 1, 4, 9, 14, 18, 20};       // cumulative weights 1, 3, 5, 5, 4, 2 (of 20)
-    n_groups = 6;
-    for (int g = 0; g <= 6; ++g) bounds[g] = (int)(((long long)p->heads * kRamp[g] + 10) / 20);
-    for (int g = 1; g <= 6; ++g) bounds[g] = std::max(bounds[g], bounds[g - 1] + 1);
-    bounds[6] = p->heads;
+  if (n_groups <= 0 && p->heads >= 16) {
+    static const int kRamp[9] = {0, 1, 4, 10, 19, 28, 34, 38, 40};      // group weights 1, 3, 6, 9, 9, 6, 4, 2 (of 40)
+    n_groups = 8;
+    for (int g = 0; g <= 8; ++g) bounds[g] = (int)(((long long)p->heads * kRamp[g] + 20) / 40);
+    for (int g = 1; g <= 8; ++g) bounds[g] = std::max(bounds[g], bounds[g - 1] + 1);
+    bounds[8] = p->heads;
   } else {
     if (n_groups <= 0) n_groups = 8;
     n_groups = std::min(std::min(n_groups, 8), p->heads);
@@ -1176,8 +1180,10 @@ int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void*
   if (!p->host_pipe_ready) {
     e = cudaStreamCreateWithFlags(&p->s_h2d, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->s_d2h, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->s_alt, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_start, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_bits, cudaEventDisableTiming);
     for (int g = 0; g < 8 && e == cudaSuccess; ++g) {
       e = cudaEventCreateWithFlags(&p->ev_in[g], cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_out[g], cudaEventDisableTiming);
@@ -1219,15 +1225,25 @@ int sol_attn3d_forward_host(sol_attn3d_plan_t p, const void* q_host, const void*
                                  (size_t)p->total_tokens, cudaMemcpyHostToDevice, p->s_h2d)) != cudaSuccess)
         return fail_cuda(p, e);
     if ((e = cudaEventRecord(p->ev_in[g], p->s_h2d)) != cudaSuccess) return fail_cuda(p, e);
-    if ((e = cudaStreamWaitEvent(st, p->ev_in[g], 0)) != cudaSuccess) return fail_cuda(p, e);
+    // Kernels of even groups run on the caller's stream, those of odd groups on an internal one: neighbouring groups may
+    // then share the GPU, and the last, partly filled wave of one group's attention no longer leaves SMs idle until
+    // the next group's kernels start.  (Different heads: disjoint parts of the workspace and of the output.)
+    cudaStream_t sg = (g & 1) ? p->s_alt : st;
+    if (g == 1) {
+      // the internal stream joins after everything the caller queued before this call, and after group 0's launch set
+      // has got far enough for the key-validity bits (built or kept by group 0) to be in place
+      if ((e = cudaStreamWaitEvent(p->s_alt, p->ev_bits, 0)) != cudaSuccess) return fail_cuda(p, e);
+    }
+    if ((e = cudaStreamWaitEvent(sg, p->ev_in[g], 0)) != cudaSuccess) return fail_cuda(p, e);
     FwdOpts o;
     o.head_begin = h0;
     o.head_end = h1;
     o.skip_keybits = g > 0;
     o.keep_launch_count = g > 0;
-    rc = forward_impl(p, dq, dk, dv, dout, dmask, stream, o);
+    o.bits_done = g == 0 ? p->ev_bits : nullptr;
+    rc = forward_impl(p, dq, dk, dv, dout, dmask, static_cast<sol_attn3d_stream_t>(sg), o);
     if (rc != SOL_ATTN3D_OK) break;
-    if ((e = cudaEventRecord(p->ev_out[g], st)) != cudaSuccess) return fail_cuda(p, e);
+    if ((e = cudaEventRecord(p->ev_out[g], sg)) != cudaSuccess) return fail_cuda(p, e);
     if ((e = cudaStreamWaitEvent(p->s_d2h, p->ev_out[g], 0)) != cudaSuccess) return fail_cuda(p, e);
     if ((e = cudaMemcpy2DAsync(static_cast<unsigned char*>(out_host) + off, pitch, dout + off, pitch, width,
                                (size_t)p->total_tokens, cudaMemcpyDeviceToHost, p->s_d2h)) != cudaSuccess)
