@@ -86,7 +86,7 @@ def _ramp_inputs(w, direction, step_g, a=8.0, single_step_at=None):
     """N(0,1) inputs with dim D-1 of every query set to `a` and of every key to a per-tile level g_t, which adds
     a * g_t / sqrt(D) to the logits of tile t and leaves the within-tile spread alone.  A handful of keys then carry
     each row, so the outputs are as large as single V entries; V is scaled by 1/4 (exact in bf16) to keep them
-    around 1, where the absolute bound of the contract is neither vacuous nor below the bf16 output rounding."""
+    close to 1, where the absolute bound of the contract is neither vacuous nor below the bf16 output rounding."""
     inp = wl.make_inputs(w, "cuda")
     inp.v.mul_(0.25)
     n, D = w.total_tokens, w.head_dim
