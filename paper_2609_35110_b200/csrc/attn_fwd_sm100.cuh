@@ -468,10 +468,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // =========================================================== TMA producer
     if (lane == 0) {
       bool ok = true;
-      // Q tiles are read once: first to go from L2, so that they do not push out the head's K / V, which every
-      // CTA of the head streams (an evict-last hint on K / V was measured too: more DRAM reads, not fewer, because
-      // the previous heads' tiles then linger)
+      // Q tiles are read once: first to go from L2, so that they do not push out the head's K / V, which every CTA of the
+      // head streams.  K / V of a CTA pair are loaded with an evict-last hint on half of the lines: at the high-resolution
+      // size that took the DRAM reads of a launch from 6.9 to 5.6 GB (any share from 0.3 to 1.0 did; evict-first on the rest
+      // instead of the default: 38-48 GB).  Single CTAs keep the default: there the hint was measured to raise the reads,
+      // because the previous heads' tiles then linger.
       const uint64_t pol_once = l2_policy_evict_first();
+      const uint64_t pol_kv = l2_policy_evict_last_half();
       // the leader's barrier counts the bytes of both CTAs' loads
       if (leader) mbar_arrive_expect_tx(bar_q_full, kCtas * 2 * L::kTile);
 #pragma unroll
@@ -496,9 +499,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (kv == 0) {
 #pragma unroll
               for (int hf = 0; hf < L::kHalves; ++hf)
-                tma_load_3d_pair(dst + hf * L::kKBoxBytes, &tm_k, full, hf * 64, head, tok0 + jt * 128 + (int)rank * 64);
+                tma_load_3d_pair_hint(dst + hf * L::kKBoxBytes, &tm_k, full, hf * 64, head, tok0 + jt * 128 + (int)rank * 64, pol_kv);
             } else {
-              tma_load_3d_pair(dst, &tm_v, full, (int)rank * 64, head, tok0 + jt * 128);
+              tma_load_3d_pair_hint(dst, &tm_v, full, (int)rank * 64, head, tok0 + jt * 128, pol_kv);
             }
           } else {
             const CUtensorMap* tm = kv ? &tm_v : &tm_k;
