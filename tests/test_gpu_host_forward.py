@@ -47,6 +47,26 @@ def test_host_forward_equals_device_forward(B, name, groups):
     attn.close()
 
 
+@pytest.mark.parametrize("name", ["varlen", "cfg_batch"])
+def test_host_forward_as_the_first_call_of_a_plan(B, name):
+    """Nothing has run on the plan before: the key-validity bits are built by the first head group's launch set on the
+    caller's stream, and the second group's kernels, which run on an internal stream, must come after them."""
+    w = wl.shrunk(name)
+    inp = wl.make_inputs(w, "cuda")
+    attn = B.Attn3d.from_workload(w, "cuda")
+    hq, hk, hv = (t.cpu().pin_memory() for t in (inp.q, inp.k, inp.v))
+    hmask = None if inp.key_mask is None else inp.key_mask.cpu().pin_memory()
+    hout = torch.full(tuple(inp.q.shape), float("nan"), dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(B.sol_attn3d_host_staging_bytes(attn.plan), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_forward_host(attn.plan, hq, hk, hv, hout, hmask, staging, 0)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    want = attn.forward(inp.q, inp.k, inp.v, inp.key_mask)
+    torch.cuda.synchronize()
+    assert torch.equal(hout.view(torch.int16), want.cpu().view(torch.int16))
+    attn.close()
+
+
 def test_host_forward_rejects_bad_arguments(B):
     w = wl.shrunk("tiny")
     inp = wl.make_inputs(w, "cuda")

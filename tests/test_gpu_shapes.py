@@ -120,3 +120,31 @@ def test_one_very_long_sequence_sampled_rows():
     print("long:", max_abs, rel_l2)
     assert max_abs <= 2e-2 and rel_l2 <= 5e-3
     attn.close()
+
+
+def test_tensors_beyond_four_gib_sampled_groups():
+    """32 sequences of 4,352 tokens with 128 heads: every one of Q, K, V and the output is 4.56 GB, so byte offsets pass
+    2^32 (and element offsets 2^31) in the rotary producer, in the TMA coordinates times strides, and in the epilogue's row
+    addresses.  Whole (sequence, head) groups are checked against the oracle, the last one in memory among them."""
+    from paper_2609_35110_b200 import binding as B
+    spec = wl.SeqSpec(256, 16, 16, 16)
+    w = wl.Workload(name="big", seqs=(spec,) * 32, heads=128, head_dim=128, rope_dims=(32, 48, 48), seed=91)
+    n_seq = 256 + 16 * 16 * 16
+    assert w.total_tokens == 32 * n_seq and w.total_tokens * 128 * 128 * 2 > (1 << 32)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(w.seed)
+    shape = (w.total_tokens, w.heads, w.head_dim)
+    q, k, v = (torch.randn(shape, generator=gen, device="cuda", dtype=torch.bfloat16) for _ in range(3))
+    attn = B.Attn3d.from_workload(w, "cuda")
+    out = torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.sol_attn3d_forward(attn.plan, q, k, v, out, None)
+    torch.cuda.synchronize()
+    assert attn.status() == 0
+    assert not bool(torch.isnan(out[-n_seq:].float()).any()) and not bool(torch.isnan(out[:n_seq].float()).any())
+    for s, h in [(0, 0), (15, 127), (16, 0), (31, 64), (31, 127)]:
+        sl = slice(s * n_seq, (s + 1) * n_seq)
+        ref = orc.attn3d_oracle(q[sl, h:h + 1].cpu(), k[sl, h:h + 1].cpu(), v[sl, h:h + 1].cpu(), [(256, 16, 16, 16)],
+                                w.rope_dims, w.theta, None)
+        max_abs, rel_l2 = orc.compare(out[sl, h:h + 1].cpu(), ref)
+        assert max_abs <= 2e-2 and rel_l2 <= 5e-3, (s, h, max_abs, rel_l2)
+    attn.close()
