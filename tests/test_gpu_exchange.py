@@ -130,6 +130,39 @@ def test_pack_qkv_is_the_reference_permutation(B, G, n_local, heads, D):
         assert torch.equal(send2, send)
 
 
+def test_layout_kernels_beyond_four_gib(B):
+    """One rank of a one-way exchange at 150,000 tokens x 40 heads x 128: the packed destination is 4.6 GB, so chunk and
+    byte offsets pass 2^32 in the pack, the record pack and the merge.  Every kernel works token by token, so slices of
+    tokens (the first, those around the 2^32-byte mark, the last) are compared with the oracle on the same slices."""
+    n, heads, D = 150_000, 40, 128
+    g = torch.Generator(device="cuda").manual_seed(321)
+    q, k, v = (torch.randn((n, heads, D), generator=g, device="cuda", dtype=torch.bfloat16) for _ in range(3))
+    send = torch.empty((1, n, 3, heads, D), dtype=torch.bfloat16, device="cuda")
+    assert send.numel() * 2 > (1 << 32)
+    B.sol_attn3d_exchange_pack_qkv(q, k, v, 1, [send[0].data_ptr()], 0)
+    rb = B.sol_attn3d_exchange_record_bytes(B.WIRE_QKV_INT8, D)
+    send8 = torch.empty((1, n, heads, rb), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_pack_qkv_int8(q, k, v, 1, [send8[0].data_ptr()], 0)
+    # return path: two ranks' results for 440,000 tokens, 4.5 GB in and out
+    n2, hl = 440_000, 20
+    recv = torch.randint(0, 256, (2, n2, hl, 2 * D), generator=g, device="cuda", dtype=torch.uint8)
+    assert recv.numel() > (1 << 32)
+    merged = torch.empty((n2, 2 * hl, 2 * D), dtype=torch.uint8, device="cuda")
+    B.sol_attn3d_exchange_merge_heads(recv, merged, n2, 2 * hl, 2 * D, 2)
+    torch.cuda.synchronize()
+    mark = (1 << 32) // (3 * heads * D * 2)                    # the token whose packed row straddles byte 2^32
+    for t0, t1 in [(0, 64), (mark - 32, mark + 32), (n - 64, n)]:
+        qs, ks, vs = q[t0:t1].cpu(), k[t0:t1].cpu(), v[t0:t1].cpu()
+        want = xo.pack_qkv_reference(qs, ks, vs, 1)
+        assert torch.equal(send[:, t0:t1].cpu().view(torch.int16), want.view(torch.int16)), (t0, t1)
+        want8 = xo.qkv_records(qs, ks, vs)
+        assert torch.equal(send8[0, t0:t1].cpu(), want8), (t0, t1)
+    mark2 = (1 << 32) // (2 * hl * 2 * D)
+    for t0, t1 in [(0, 64), (mark2 - 32, mark2 + 32), (n2 - 64, n2)]:
+        want = xo.merge_heads_reference(recv[:, t0:t1].cpu())
+        assert torch.equal(merged[t0:t1].cpu(), want), (t0, t1)
+
+
 @pytest.mark.parametrize("G,n_local,heads,record", [(2, 300, 8, 256), (4, 77, 8, 128), (8, 33, 40, 144), (1, 5, 3, 64), (2, 129, 4, 16)])
 def test_merge_heads_is_the_reference_permutation(B, G, n_local, heads, record):
     g = torch.Generator(device="cuda").manual_seed(200 + G)
