@@ -232,6 +232,25 @@ __global__ void __launch_bounds__(256) quantize_records_kernel(const QuantArgs a
   }
 }
 
+// sixteen int8 values (one 16-byte load) times one scale -> eight packed bf16 pairs, each value q * s rounded to bf16.
+// The int8 -> float step avoids the conversion unit: byte b xor 0x80 dropped into the mantissa of 2^23 + 2^22 gives
+// m = 12582912 + (q + 128) exactly, and q * s = fma(m, s, -12583040 s): the addend is exact (21 significant bits) and so
+// is the result, because q * s itself is representable (7 + 4 significant bits).
+__device__ __forceinline__ void dequant16(const uint4 v, float s, uint32_t (&out)[8]) {
+  const uint32_t w[4] = {v.x ^ 0x80808080u, v.y ^ 0x80808080u, v.z ^ 0x80808080u, v.w ^ 0x80808080u};
+  const float ns = -12583040.0f * s;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float x0 = __fmaf_rn(__uint_as_float(__byte_perm(w[j], 0x4B400000u, 0x7650)), s, ns);
+    const float x1 = __fmaf_rn(__uint_as_float(__byte_perm(w[j], 0x4B400000u, 0x7651)), s, ns);
+    const float x2 = __fmaf_rn(__uint_as_float(__byte_perm(w[j], 0x4B400000u, 0x7652)), s, ns);
+    const float x3 = __fmaf_rn(__uint_as_float(__byte_perm(w[j], 0x4B400000u, 0x7653)), s, ns);
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(x0, x1), hi = __floats2bfloat162_rn(x2, x3);
+    out[2 * j] = *reinterpret_cast<const uint32_t*>(&lo);
+    out[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&hi);
+  }
+}
+
 // Receiver's side: records [rows][heads][rec_bytes] -> bf16 [rows][NW][heads][D] (NW = 3: the packed QKV tensor
 // the attention reads through strides; NW = 1: output rows).  value = q * s, exact in fp32, one rounding to bf16.
 template <int NW>
@@ -254,19 +273,15 @@ __global__ void __launch_bounds__(256) dequantize_records_kernel(const uint8_t* 
     const uint4* src = reinterpret_cast<const uint4*>(r + which * head_dim + grp * 32);
     const uint4 v0 = __ldg(src), v1 = __ldg(src + 1);
     const float s = ue5m3_value(__ldg(r + NW * head_dim + rem));
-    const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    uint32_t o[16];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float q0 = (float)(int)(int8_t)(w[j] & 0xffu), q1 = (float)(int)(int8_t)((w[j] >> 8) & 0xffu);
-      const float q2 = (float)(int)(int8_t)((w[j] >> 16) & 0xffu), q3 = (float)(int)(int8_t)(w[j] >> 24);
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(q0 * s, q1 * s), hi = __floats2bfloat162_rn(q2 * s, q3 * s);
-      o[2 * j] = *reinterpret_cast<const uint32_t*>(&lo);
-      o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&hi);
-    }
+    uint32_t o0[8], o1[8];
+    dequant16(v0, s, o0);
+    dequant16(v1, s, o1);
     uint4* dst = reinterpret_cast<uint4*>(out + (((t * NW + which) * heads + h) * (long long)head_dim + grp * 32));
 #pragma unroll
-    for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+    for (int j = 0; j < 2; ++j) {
+      dst[j] = make_uint4(o0[4 * j], o0[4 * j + 1], o0[4 * j + 2], o0[4 * j + 3]);
+      dst[2 + j] = make_uint4(o1[4 * j], o1[4 * j + 1], o1[4 * j + 2], o1[4 * j + 3]);
+    }
   }
 }
 

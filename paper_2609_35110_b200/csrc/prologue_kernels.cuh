@@ -228,73 +228,83 @@ struct RopeRecordArgs {
   unsigned int* status;
 };
 
-__global__ void __launch_bounds__(256, 3) rope_records_kernel(const RopeRecordArgs a) {
+// Thread = 16 head dims of one (token, head) record: one 16-byte load per tensor, two 16-byte stores per tensor.  A block
+// is (head_dim / 16) x heads_per_pass x tokens_per_block threads; every thread takes its heads two at a time, the six
+// loads of the pair in flight together.
+__global__ void __launch_bounds__(256, 2) rope_records_kernel(const RopeRecordArgs a, int heads_per_pass) {
   const int D = a.g.head_dim;
-  const int chunks = D >> 3;
-  const int heads_per_pass = blockDim.x / chunks;
-  const int chunk = threadIdx.x % chunks;
-  const int hsub = threadIdx.x / chunks;
+  const int lanes = D >> 4;                       // threads per record
+  const int part = threadIdx.x % lanes;           // which 16 head dims
+  const int hsub = (threadIdx.x / lanes) % heads_per_pass;
+  const int tsub = threadIdx.x / (lanes * heads_per_pass);
+  const int toks_per_block = blockDim.x / (lanes * heads_per_pass);
   const int d1 = a.g.rope[0], d2 = d1 + a.g.rope[1], d3 = d2 + a.g.rope[2];
-  int axis[4], tab[4], step[4];
+  int axis[8], tab[8], step[8];                   // per pair of this thread: which position, which table entries
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const int d = chunk * 8 + 2 * u;
+  for (int u = 0; u < 8; ++u) {
+    const int d = part * 16 + 2 * u;
     if (d < d1)      { axis[u] = 0; tab[u] = a.g.tab_off[0] + (d >> 1);        step[u] = a.g.rope[0] >> 1; }
     else if (d < d2) { axis[u] = 1; tab[u] = a.g.tab_off[1] + ((d - d1) >> 1); step[u] = a.g.rope[1] >> 1; }
     else if (d < d3) { axis[u] = 2; tab[u] = a.g.tab_off[2] + ((d - d2) >> 1); step[u] = a.g.rope[2] >> 1; }
     else             { axis[u] = -1; tab[u] = 0; step[u] = 0; }
   }
-  const int code_off = 3 * D + (chunk >> 2);      // this chunk's scale code inside a tensor's D/32 codes
   const int n_codes = D >> 5;
+  const int code_idx = part >> 1;                 // this thread's group of 32 inside a tensor
 
-  for (long long tok = blockIdx.x; tok < a.total_tokens; tok += gridDim.x) {
+  for (long long tok = (long long)blockIdx.x * toks_per_block + tsub; tok < a.total_tokens;
+       tok += (long long)gridDim.x * toks_per_block) {
     int s = 0;
     while (s + 1 < a.n_seqs && !(tok >= a.seqs[s].tok_start && tok < a.seqs[s].tok_start + a.seqs[s].n_tokens)) ++s;
     const SeqDev sq = a.seqs[s];
     const int local = (int)(tok - sq.tok_start);
     SOL_DEVICE_CHECK(a.status, local >= 0 && local < sq.n_tokens, kCheckTokenSequence);
     const bool rotate = local >= sq.text_len;
-    float2 cs[4];
+    float2 cs[8];
     if (rotate) {
       const int p = local - sq.text_len;
       const int hw = sq.H * sq.W;
       const int pt = p / hw, ph = (p / sq.W) % sq.H, pw = p % sq.W;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 8; ++u) {
         const int pos = axis[u] == 0 ? pt : axis[u] == 1 ? ph : pw;
         cs[u] = axis[u] < 0 ? make_float2(1.f, 0.f) : __ldg(&a.tables[tab[u] + pos * step[u]]);
       }
     }
-    for (int h = hsub; h < a.g.heads; h += heads_per_pass) {
-      const uint8_t* rec = a.records + (tok * a.g.heads + h) * (long long)a.rec_bytes;
-      uint2 v[3];
-      float sc[3];
+    for (int h0 = hsub; h0 < a.g.heads; h0 += 2 * heads_per_pass) {
+      uint4 v[2][3];
+      float sc[2][3];
 #pragma unroll
-      for (int which = 0; which < 3; ++which) {
-        v[which] = __ldg(reinterpret_cast<const uint2*>(rec + which * D + chunk * 8));
-        sc[which] = ue5m3_value(__ldg(rec + code_off + which * n_codes));
+      for (int b = 0; b < 2; ++b) {
+        const int h = h0 + b * heads_per_pass;
+        if (h >= a.g.heads) break;
+        const uint8_t* rec = a.records + (tok * a.g.heads + h) * (long long)a.rec_bytes;
+#pragma unroll
+        for (int which = 0; which < 3; ++which) {
+          v[b][which] = __ldg(reinterpret_cast<const uint4*>(rec + which * D + part * 16));
+          sc[b][which] = ue5m3_value(__ldg(rec + 3 * D + which * n_codes + code_idx));
+        }
       }
 #pragma unroll
-      for (int which = 0; which < 3; ++which) {
-        const uint32_t w[2] = {v[which].x, v[which].y};
-        float f[8];
+      for (int b = 0; b < 2; ++b) {
+        const int h = h0 + b * heads_per_pass;
+        if (h >= a.g.heads) break;
+        const long long row = (tok * a.g.heads + h) * (long long)D + part * 16;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float qv = (float)(int)(int8_t)((w[e >> 2] >> (8 * (e & 3))) & 0xffu);
-          f[e] = __bfloat162float(__float2bfloat16_rn(qv * sc[which]));     // the value the bf16 wire tensor would hold
-        }
-        uint32_t o[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          float re = f[2 * u], ro = f[2 * u + 1];
+        for (int which = 0; which < 3; ++which) {
+          uint32_t o[8];
+          dequant16(v[b][which], sc[b][which], o);            // the values the bf16 wire tensor would hold
           if (which < 2 && rotate) {
-            re = f[2 * u] * cs[u].x - f[2 * u + 1] * cs[u].y;
-            ro = f[2 * u] * cs[u].y + f[2 * u + 1] * cs[u].x;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const float f0 = __uint_as_float(o[u] << 16), f1 = __uint_as_float(o[u] & 0xffff0000u);
+              const __nv_bfloat162 r2 = __floats2bfloat162_rn(f0 * cs[u].x - f1 * cs[u].y, f0 * cs[u].y + f1 * cs[u].x);
+              o[u] = *reinterpret_cast<const uint32_t*>(&r2);
+            }
           }
-          const __nv_bfloat162 r2 = __floats2bfloat162_rn(re, ro);
-          o[u] = *reinterpret_cast<const uint32_t*>(&r2);
+          uint4* dst = reinterpret_cast<uint4*>(a.y[which] + row);
+          dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+          dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
         }
-        *reinterpret_cast<uint4*>(a.y[which] + (tok * a.g.heads + h) * (long long)D + chunk * 8) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   }

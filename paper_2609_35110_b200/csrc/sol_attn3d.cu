@@ -883,12 +883,16 @@ int forward_impl(sol_attn3d_plan_t p, const void* q, const void* k, const void* 
     ra.g.head_dim = p->head_dim;
     ra.g.heads = p->heads;
     ra.status = reinterpret_cast<unsigned int*>(ws + p->off_status);
-    const int chunks = p->head_dim / 8, cap = 256 / chunks;
-    int hpp = std::max(1, std::min(p->heads, cap));
-    for (int d = std::min(p->heads, cap); d >= std::max(1, cap / 2); --d)
+    // a record takes head_dim / 16 threads; heads per pass: the largest divisor of the head count that fits a block, so
+    // that every thread has the same number of heads (two per batch); small shards put several tokens in a block
+    const int lanes = p->head_dim / 16, cap = 256 / lanes;
+    int hpp = 1;
+    for (int d = std::min(p->heads, cap); d >= 1; --d)
       if (p->heads % d == 0) { hpp = d; break; }
-    const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
-    sol::rope_records_kernel<<<(unsigned)blocks, chunks * hpp, 0, st>>>(ra);
+    const int toks = std::max(1, 256 / (lanes * hpp));
+    const long long want = (p->total_tokens + toks - 1) / toks;
+    const long long blocks = std::max<long long>(1, std::min<long long>(want, 148ll * 16));
+    sol::rope_records_kernel<<<(unsigned)blocks, lanes * hpp * toks, 0, st>>>(ra, hpp);
     if ((e = cudaGetLastError()) != cudaSuccess) return fail_cuda(p, e);
     ++p->launches;
   } else {
