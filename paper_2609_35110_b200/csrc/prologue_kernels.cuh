@@ -105,14 +105,7 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
   const int hsub = threadIdx.x / chunks;
   const int d1 = a.g.rope[0], d2 = d1 + a.g.rope[1], d3 = d2 + a.g.rope[2];
   const float inv_d = 1.0f / (float)a.g.head_dim;
-  // the gains of this thread's eight head dims (the plain rotary instantiation carries none)
-  float gn[2][kNorm ? 8 : 1];
-  if (kNorm) {
-#pragma unroll
-    for (int which = 0; which < 2; ++which)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) gn[which][kNorm ? e : 0] = a.gain[which] ? __ldg(a.gain[which] + chunk * 8 + e) : 1.0f;
-  }
+  const unsigned warp_lanes = __activemask();    // the block's last warp may be partial; nothing diverges after this point
   // which table entry each of the thread's four pairs uses (fixed per thread: it depends on the chunk only)
   int axis[4], tab[4], step[4];                 // step: table entries per position of that axis
 #pragma unroll
@@ -134,8 +127,9 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
     const bool rotate = local >= sq.text_len;
     // heads in groups of kBatch per thread and tensor: the loads of Q AND K of a group are all issued before any is
     // used, and the table lookups travel with them
-    constexpr int kBatch = kNorm ? 3 : 4;         // (the normalising instantiation also holds sixteen gains)
-    for (int h0 = a.head_begin + hsub; h0 < a.head_end; h0 += kBatch * heads_per_pass) {
+    constexpr int kBatch = 4;
+    for (int hb = a.head_begin; hb < a.head_end; hb += kBatch * heads_per_pass) {    // the same trip count for every thread
+      const int h0 = hb + hsub;
       uint4 v[2][kBatch];
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
@@ -144,7 +138,8 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
           const int h = h0 + b * heads_per_pass;
-          if (h < a.head_end) v[which][b] = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
+          if (kNorm)                v[which][b] = __ldg(reinterpret_cast<const uint4*>(src + min(h, a.head_end - 1) * a.x_head_stride[which]));
+          else if (h < a.head_end)  v[which][b] = __ldg(reinterpret_cast<const uint4*>(src + h * a.x_head_stride[which]));
         }
       }
       float2 cs[4];
@@ -158,6 +153,37 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
           cs[u] = axis[u] < 0 ? make_float2(1.f, 0.f) : __ldg(&a.tables[tab[u] + pos * step[u]]);
         }
       }
+      // Normalising instantiation: the sums of squares of all rows of the group first, then their shuffle reductions
+      // step by step across the rows (six independent chains instead of six dependent ones one after another), then
+      // the reciprocal roots.  Rows past the head range were loaded from a clamped head and are not stored.
+      float rinv[2][kBatch];
+      if (kNorm) {
+        float ss[2][kBatch];
+#pragma unroll
+        for (int which = 0; which < 2; ++which)
+#pragma unroll
+          for (int b = 0; b < kBatch; ++b) {
+            const uint32_t w[4] = {v[which][b].x, v[which][b].y, v[which][b].z, v[which][b].w};
+            float acc = 0.f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const float lo = __uint_as_float(w[u] << 16), hi = __uint_as_float(w[u] & 0xffff0000u);
+              acc = fmaf(lo, lo, acc);
+              acc = fmaf(hi, hi, acc);
+            }
+            ss[which][b] = acc;
+          }
+        for (int off = chunks >> 1; off > 0; off >>= 1) {
+#pragma unroll
+          for (int which = 0; which < 2; ++which)
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) ss[which][b] += __shfl_xor_sync(warp_lanes, ss[which][b], off);
+        }
+#pragma unroll
+        for (int which = 0; which < 2; ++which)
+#pragma unroll
+          for (int b = 0; b < kBatch; ++b) rinv[which][b] = rsqrtf(ss[which][b] * inv_d + a.eps);
+      }
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
         if (a.x[which] == nullptr) continue;
@@ -166,27 +192,21 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
           const int h = h0 + b * heads_per_pass;
-          if (h >= a.head_end) break;
-          // all lanes of a row enter together (the bound depends on hsub only)
-          const unsigned lanes = __activemask();
+          if (!kNorm && h >= a.head_end) break;
           const uint32_t w[4] = {v[which][b].x, v[which][b].y, v[which][b].z, v[which][b].w};
           float f[8];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162*>(&w[u]);
-            f[2 * u] = __low2float(b2);
-            f[2 * u + 1] = __high2float(b2);
+            f[2 * u] = __uint_as_float(w[u] << 16);
+            f[2 * u + 1] = __uint_as_float(w[u] & 0xffff0000u);
           }
           if (norm) {
-            float ss = 0.f;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
-            for (int off = chunks >> 1; off > 0; off >>= 1) ss += __shfl_xor_sync(lanes, ss, off);
-            const float r = rsqrtf(ss * inv_d + a.eps);
-            // the gains of this thread's eight head dims: 32 bytes that stay in L1 (not kept in registers: the
-            // plain rotary path has no use for them)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] = f[e] * r * gn[which][kNorm ? e : 0];
+            // the gains of this thread's eight head dims: 32 bytes that stay in L1
+            const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.gain[which] + chunk * 8));
+            const float4 g1 = __ldg(reinterpret_cast<const float4*>(a.gain[which] + chunk * 8) + 1);
+            const float r = rinv[which][b];
+            f[0] *= r * g0.x; f[1] *= r * g0.y; f[2] *= r * g0.z; f[3] *= r * g0.w;
+            f[4] *= r * g1.x; f[5] *= r * g1.y; f[6] *= r * g1.z; f[7] *= r * g1.w;
           }
           uint32_t o[4];
 #pragma unroll
@@ -199,7 +219,7 @@ __global__ void __launch_bounds__(256, 3) rope_qk_kernel(const RopeArgs a) {
             const __nv_bfloat162 r2 = __floats2bfloat162_rn(re, ro);
             o[u] = *reinterpret_cast<const uint32_t*>(&r2);
           }
-          *reinterpret_cast<uint4*>(dst + (long long)h * a.g.head_dim) = make_uint4(o[0], o[1], o[2], o[3]);
+          if (h < a.head_end) *reinterpret_cast<uint4*>(dst + (long long)h * a.g.head_dim) = make_uint4(o[0], o[1], o[2], o[3]);
         }
       }
     }

@@ -335,8 +335,8 @@ int launch_rope(sol_attn3d_plan_t p, const unsigned char* ws, const void* q, con
   const int n_heads = a.head_end - a.head_begin, cap = 256 / chunks;
   const bool norm = q_gain != nullptr || k_gain != nullptr;
   int hpp = std::max(1, std::min(n_heads, cap));
-  for (int d = std::min(n_heads, cap); !norm && d >= std::max(1, cap / 2); --d)   // (the normalising variant, bound by its
-    if (n_heads % d == 0) { hpp = d; break; }                                      //  reductions, measured better with full blocks)
+  for (int d = std::min(n_heads, cap); d >= std::max(1, cap / 2); --d)
+    if (n_heads % d == 0) { hpp = d; break; }
   const int threads = chunks * hpp;
   const long long blocks = std::min<long long>(p->total_tokens, 148ll * 16);
   if (norm) sol::rope_qk_kernel<true><<<(unsigned)blocks, threads, 0, st>>>(a);
